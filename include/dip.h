@@ -1,0 +1,262 @@
+/*
+ * dip.h — C ABI of the B200 (sm_100a) sparse SwiGLU decode-MLP library for
+ * Dynamic Input Pruning (DIP) and its cache-aware variant (DIP-CA),
+ * arxiv 2412.01380.
+ *
+ * The library computes, per decode token and per MLP block, the sparse MLP of
+ * Eq. 3 with the input-pruning masks of Eq. 7-8:
+ *
+ *     m_x = topK(score(x))            keep k_x of the d_model input columns
+ *     h   = (W~u x) * silu(W~g x)     gate/up read only the kept columns of W^g, W^u
+ *     m_h = topK(score(h))            keep k_h of the d_ff columns of W^d
+ *     y   = W~d h                     down reads only the kept columns of W^d
+ *
+ * where score is |.| (DIP) or the cache-aware re-weighting of Eq. 10 with the
+ * column-cache update of Algorithm 1 (DIP-CA).
+ *
+ * Conventions
+ *  - Every data pointer is DEVICE memory owned by the caller unless a comment
+ *    says "host".  Structs and the context handle are host memory.
+ *  - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and
+ *    return without synchronising.  Results are valid once the stream reaches
+ *    the end of the enqueued work.
+ *  - Calls on the same context must not overlap on the GPU (they share the
+ *    context's scratch workspace): use one context per concurrently running
+ *    stream.
+ *  - Arguments are validated on the host before anything is launched; a failed
+ *    validation returns an error code and launches nothing.
+ *  - Data pointers must be 16-byte aligned.
+ *  - Float vectors are binary32.  Masks are bit sets: bit (i & 31) of word
+ *    (i >> 5) is column i.  Kept-index lists are int32 in ascending order.
+ *  - Top-k ties are resolved in favour of the lower column index, so every
+ *    result is unique; the paper does not fix a tie rule.
+ *  - Floating-point sums run in a fixed order: results are bit-reproducible
+ *    from run to run on the same device and library build.
+ */
+#ifndef DIP_H
+#define DIP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DIP_OK = 0,
+    DIP_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, k or capacity out of range, bad size   */
+    DIP_ERR_UNSUPPORTED = 2,   /* valid request the library does not implement (see each call)      */
+    DIP_ERR_CUDA = 3,          /* a CUDA runtime call failed; see dip_last_error                     */
+    DIP_ERR_WORKSPACE = 4      /* problem larger than the context's scratch workspace allows         */
+} dip_status;
+
+typedef enum {
+    DIP_W_F32 = 0,             /* binary32 weights                                                   */
+    DIP_W_BF16 = 1,            /* bfloat16 weights                                                   */
+    DIP_W_INT4_G128 = 2        /* 4-bit symmetric codes, one binary16 scale per 128 input indices    */
+} dip_wtype;
+
+enum {
+    DIP_MAX_D = 32768,         /* largest masked dimension (d_model or d_ff)                         */
+    DIP_MAX_BATCH = 16,
+    DIP_INT4_GROUP = 128,
+    DIP_CACHE_META_INTS = 8    /* length of dip_cache_state.meta                                     */
+};
+
+typedef struct dip_ctx dip_ctx;   /* opaque; owns scratch workspace on one device */
+
+/* Create a context on `device` (a CUDA ordinal).  Allocates the scratch
+ * workspace (a few MB) with cudaMalloc; no other call allocates.  *out is
+ * NULL on failure. */
+dip_status dip_create(dip_ctx **out, int device);
+/* Frees the workspace.  The caller makes sure no work of this context is in flight. */
+dip_status dip_destroy(dip_ctx *ctx);
+/* Static description of a status code (host string, never NULL). */
+const char *dip_status_string(dip_status s);
+/* Text of the last CUDA failure seen by this context (host string owned by the
+ * context; empty if none). */
+const char *dip_last_error(const dip_ctx *ctx);
+/* Number of streaming multiprocessors of the context's device. */
+int dip_sm_count(const dip_ctx *ctx);
+
+/* ------------------------------------------------------------------------
+ * Weights.  The paper's unit of selection is a column W[:, i] of a matrix
+ * W in R^{d_out x d_in} (Eq. 4, 7, 8), so the library stores each matrix
+ * column-contiguous: row i of the packed array holds column i.  Gate and up
+ * always share one mask (Eq. 7), so their columns are bundled: packed row i
+ * holds W^g[:, i] and W^u[:, i] interleaved in 16-byte pieces
+ * (piece 2c = gate outputs of chunk c, piece 2c+1 = up outputs of chunk c;
+ * a chunk is 4 outputs for F32, 8 for BF16, 32 for INT4).
+ *
+ *   gate_up        [d_model][2 * d_ff] elements, interleaved as above
+ *   down           [d_ff][d_model]     elements
+ *   INT4 codes     two per byte, output j in bits 4*(j&1).. of byte j>>1 within a row
+ *                  (within a 16-byte piece for gate_up); value = (code - 8) * scale
+ *   gate_up_scales [d_model/128][2 * d_ff] binary16, interleaved in 16-byte pieces
+ *                  (8 gate scales, 8 up scales)
+ *   down_scales    [d_ff/128][d_model] binary16
+ *
+ * Requirements: d_model % 32 == 0, d_ff % 32 == 0 (all formats); INT4 also
+ * needs d_model % 128 == 0 and d_ff % 128 == 0.
+ * ------------------------------------------------------------------------ */
+typedef struct {
+    int32_t wtype;               /* dip_wtype */
+    int32_t d_model;
+    int32_t d_ff;
+    int32_t reserved;
+    const void *gate_up;
+    const void *gate_up_scales;  /* NULL unless INT4 */
+    const void *down;
+    const void *down_scales;     /* NULL unless INT4 */
+} dip_mlp_weights;
+
+/* Bytes of a packed array: which = 0 gate_up, 1 down, 2 gate_up_scales,
+ * 3 down_scales.  Returns 0 for scales of non-INT4 types and for invalid
+ * arguments. */
+size_t dip_packed_bytes(int wtype, int d_model, int d_ff, int which);
+
+/* Repack canonical matrices (row-major [d_out][d_in]: Wg, Wu are
+ * [d_ff][d_model], Wd is [d_model][d_ff]; INT4 codes two per byte along d_in
+ * with the even index in the low nibble; INT4 scales Sg, Su [d_model/128][d_ff],
+ * Sd [d_ff/128][d_model]) into the packed layout above.  `out` names
+ * caller-allocated device buffers of dip_packed_bytes() bytes each.  A one-off
+ * set-up step; values are copied bit for bit. */
+dip_status dip_pack_weights(dip_ctx *ctx, int wtype, int d_model, int d_ff,
+                            const void *Wg, const void *Wu, const void *Wd,
+                            const void *Sg, const void *Su, const void *Sd,
+                            const dip_mlp_weights *out, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Column-cache state of ONE masked linear-layer input (Algorithm 1's c):
+ * gate and up share one cache over the d_model input columns, down has one
+ * over its d_ff input columns.  Eviction policy: LRU (Sec. 5.1: the column
+ * whose last use lies farthest in the past is evicted).
+ *
+ *   stamp[i]  -1 if column i is not resident, else the update number at which
+ *             it was last used while resident
+ *   meta[0]   number of resident columns        meta[1]  updates so far
+ *   meta[2..5] accumulated hits, misses, evictions, bypassed columns
+ *   meta[6..7] reserved (kept zero)
+ * A cold cache is stamp = -1 everywhere and meta = 0.  The state is updated
+ * in place; saving and restoring it is a copy of the two buffers.
+ *
+ * One update with mask m (k ones): hits are counted against the state the
+ * score used; columns of m are never evicted by the same update; the number
+ * of evictions is max(0, misses - free slots), limited by the resident columns
+ * outside m, taking the smallest (stamp, index) first; missed columns become
+ * resident in ascending index while room remains, the rest are used without
+ * being cached ("bypassed", the case of Sec. 6.3 where the active set exceeds
+ * the cache).
+ * ------------------------------------------------------------------------ */
+typedef struct {
+    int32_t d;          /* number of columns (input dimension of the layer) */
+    int32_t capacity;   /* cache size in columns, 0 <= capacity <= d        */
+    int32_t *stamp;     /* device int32[d]                                  */
+    int32_t *meta;      /* device int32[DIP_CACHE_META_INTS]                */
+} dip_cache_state;
+
+/* ------------------------------------------------------------------------
+ * dip_mask_topk — per-token magnitude top-k (Sec. 3.1; the masks of Eq. 7-8).
+ * For each of `batch` rows of x[batch][d]: keep the k columns of largest |x|.
+ *   mask_bits [batch][ceil(d/32)] out (may be NULL)
+ *   kept_idx  [batch][k]          out, ascending (may be NULL)
+ * 1 <= k <= d <= DIP_MAX_D, 1 <= batch <= DIP_MAX_BATCH.
+ * ------------------------------------------------------------------------ */
+dip_status dip_mask_topk(dip_ctx *ctx, const float *x, int batch, int d, int k,
+                         uint32_t *mask_bits, int32_t *kept_idx, void *stream);
+
+/* ------------------------------------------------------------------------
+ * dip_ca_mask — Algorithm 1 for one linear-layer input and one token:
+ *     s = |x| (c + gamma (1 - c)) / ||x||_inf      (Eq. 10)
+ *     m = topK(s, k);   c' = cache_update(c, m)    (LRU, see dip_cache_state)
+ * The ranking uses the numerator of Eq. 10 evaluated as ONE binary32
+ * round-to-nearest product |x_i| * (c_i ? 1 : gamma); the positive constant
+ * 1/||x||_inf cannot change the order and is not applied.  gamma == 1 gives
+ * the DIP mask while still tracking the cache.
+ *   st        cache state, updated in place (required)
+ *   mask_bits [ceil(d/32)] out (may be NULL);  kept_idx [k] out (may be NULL)
+ * 1 <= k <= d <= DIP_MAX_D, gamma finite and >= 0, st->d == d.
+ * ------------------------------------------------------------------------ */
+dip_status dip_ca_mask(dip_ctx *ctx, const float *x, int d, int k, float gamma,
+                       const dip_cache_state *st,
+                       uint32_t *mask_bits, int32_t *kept_idx, void *stream);
+
+/* ------------------------------------------------------------------------
+ * dip_sparse_gemv_gate_up — h = (W~u x) * silu(W~g x) over the kept columns
+ * (Eq. 2 inside Eq. 3 with the mask of Eq. 7), binary32 accumulation.
+ *   x        [batch][d_model]
+ *   kept_idx [n_kept] ascending columns to read.  batch == 1: the token's mask.
+ *            batch > 1: the union of the tokens' masks, each row read once.
+ *   mask_bits batch > 1 only: [batch][ceil(d_model/32)] per-token masks; token
+ *            b uses column i only if its bit is set.  NULL for batch == 1.
+ *   h        [batch][d_ff] out
+ * 1 <= n_kept <= d_model.
+ * ------------------------------------------------------------------------ */
+dip_status dip_sparse_gemv_gate_up(dip_ctx *ctx, const dip_mlp_weights *w,
+                                   const float *x, int batch,
+                                   const int32_t *kept_idx, int n_kept,
+                                   const uint32_t *mask_bits,
+                                   float *h, void *stream);
+
+/* ------------------------------------------------------------------------
+ * dip_sparse_gemv_down — y = W~d h over the kept columns of W^d (Eq. 1 inside
+ * Eq. 3 with the mask of Eq. 8).  Arguments as above with h [batch][d_ff] in,
+ * y [batch][d_model] out, kept_idx over the d_ff columns, 1 <= n_kept <= d_ff.
+ * ------------------------------------------------------------------------ */
+dip_status dip_sparse_gemv_down(dip_ctx *ctx, const dip_mlp_weights *w,
+                                const float *h, int batch,
+                                const int32_t *kept_idx, int n_kept,
+                                const uint32_t *mask_bits,
+                                float *y, void *stream);
+
+/* Optional outputs of a step; any pointer may be NULL (the step then keeps the
+ * intermediate in its own workspace). */
+typedef struct {
+    uint32_t *mask_x;   /* [batch][ceil(d_model/32)] */
+    int32_t *idx_x;     /* [batch][k_x]              */
+    float *h;           /* [batch][d_ff]             */
+    uint32_t *mask_h;   /* [batch][ceil(d_ff/32)]    */
+    int32_t *idx_h;     /* [batch][k_h]              */
+    int32_t *union_counts; /* batch > 1: int32[2] = |union of m_x|, |union of m_h| */
+} dip_step_outputs;
+
+/* ------------------------------------------------------------------------
+ * dip_mlp_step — the whole sparse MLP step of Eq. 3 / 7 / 8 for one block:
+ * mask x, gate/up + silu*up, mask h, down.  h stays binary32 between the
+ * halves.  cache_gu / cache_d NULL = DIP (|.| ranking, no cache); non-NULL =
+ * DIP-CA (Algorithm 1) on that input, batch must then be 1.
+ *   x [batch][d_model] in;  y [batch][d_model] out;  out may be NULL.
+ * batch > 1 computes one mask per token and reads the union of the kept
+ * columns once.
+ * ------------------------------------------------------------------------ */
+dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
+                        const float *x, int batch, int k_x, int k_h, float gamma,
+                        const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                        float *y, const dip_step_outputs *out, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Layer chaining for multi-layer workloads (not part of the paper's method):
+ * x_next = (x + y) / rms(x + y), per row, binary32 out.  x, y, x_next are
+ * [batch][d]; x_next may alias x.
+ * ------------------------------------------------------------------------ */
+dip_status dip_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y,
+                                int batch, int d, float *x_next, void *stream);
+
+/* ------------------------------------------------------------------------
+ * dip_stack_step — one decode token (or batch) through n_layers blocks:
+ * for each layer l: y = dip_mlp_step(layer l, x_l); x_{l+1} = residual_rmsnorm(x_l, y).
+ *   layers    host array [n_layers] of weights (all with the same shapes)
+ *   cache_gu, cache_d  host arrays [n_layers] or NULL (DIP)
+ *   x_in  [batch][d_model] in;  x_out [batch][d_model] out = x_{n_layers}
+ *   y_last [batch][d_model] out, the last layer's MLP output (may be NULL)
+ * ------------------------------------------------------------------------ */
+dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *layers,
+                          const float *x_in, int batch, int k_x, int k_h, float gamma,
+                          const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                          float *x_out, float *y_last, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIP_H */
