@@ -1,0 +1,75 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "dip.h"
+
+// Scratch workspace of a context.  All device memory the library itself owns.
+struct dip_ctx {
+    int device;
+    int sm_count;
+    // split-row partial sums of the two GEMVs (binary32)
+    float *partials;
+    size_t partials_floats;
+    // one arrival counter per output slab; zero between launches
+    unsigned int *tickets;
+    int n_tickets;
+    // intermediates of dip_mlp_step when the caller does not ask for them
+    float *h;            // [DIP_MAX_BATCH][DIP_MAX_D]
+    float *y;            // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner)
+    float *xa;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner ping)
+    float *xb;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner pong)
+    uint32_t *mask;      // [DIP_MAX_BATCH][DIP_MAX_D/32]
+    int32_t *idx;        // [DIP_MAX_BATCH][DIP_MAX_D]
+    int32_t *union_idx;  // [DIP_MAX_D]
+    int32_t *counts;     // [8] device scalars (union sizes)
+    char err[256];
+};
+
+#define DIP_CUDA_TRY(ctx, call)                                                        \
+    do {                                                                               \
+        cudaError_t e_ = (call);                                                       \
+        if (e_ != cudaSuccess) {                                                       \
+            snprintf((ctx)->err, sizeof((ctx)->err), "%s: %s", #call,                  \
+                     cudaGetErrorString(e_));                                          \
+            return DIP_ERR_CUDA;                                                       \
+        }                                                                              \
+    } while (0)
+
+static inline bool dip_aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
+
+// ---- launchers implemented in the kernel files (host functions) -----------------
+
+// topk.cu: one CTA per row.  stamp == nullptr: plain |x| ranking, no cache.
+dip_status dip_launch_mask(dip_ctx *ctx, const float *x, int batch, int d, int k, float gamma,
+                           int32_t *stamp, int32_t *meta, int capacity,
+                           uint32_t *mask_bits, int32_t *kept_idx, cudaStream_t stream);
+
+// topk.cu: per-device set-up of the mask kernels (dynamic shared memory limit).
+dip_status dip_init_mask_kernels(dip_ctx *ctx);
+
+// topk.cu: union of `batch` bit masks -> ascending index list and its length (device scalar).
+dip_status dip_launch_union(dip_ctx *ctx, const uint32_t *mask_bits, int batch, int d,
+                            int32_t *union_idx, int32_t *union_count, cudaStream_t stream);
+
+// topk.cu: x_next = (x + y) / rms(x + y) per row.
+dip_status dip_launch_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y, int batch, int d,
+                                       float *x_next, cudaStream_t stream);
+
+// gemv.cu: gather GEMV over kept rows of a packed matrix.
+//   which = 0: gate/up bundle with the silu*up epilogue, out = h[batch][d_ff]
+//   which = 1: down, out = y[batch][d_model]
+// n_kept_dev != nullptr: the row count is read on the device (at most n_kept_max).
+dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
+                           const float *v, int batch,
+                           const int32_t *kept_idx, int n_kept_max, const int32_t *n_kept_dev,
+                           const uint32_t *mask_bits, float *out, cudaStream_t stream);
+
+// pack.cu
+dip_status dip_launch_pack(dip_ctx *ctx, int wtype, int d_model, int d_ff,
+                           const void *Wg, const void *Wu, const void *Wd,
+                           const void *Sg, const void *Su, const void *Sd,
+                           const dip_mlp_weights *out, cudaStream_t stream);
