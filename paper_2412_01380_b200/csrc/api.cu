@@ -1,0 +1,287 @@
+// C ABI of the library (see include/dip.h): context, argument validation, and the
+// composition of the kernels into the sparse MLP step of Eq. 3 / 7 / 8.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr size_t PARTIALS_FLOATS = (size_t)8 << 20;   // 32 MB of split-row partial sums
+constexpr int N_TICKETS = 4096;
+
+bool dims_ok(int wtype, int d_model, int d_ff)
+{
+    if (wtype != DIP_W_F32 && wtype != DIP_W_BF16 && wtype != DIP_W_INT4_G128) return false;
+    if (d_model < 32 || d_ff < 32 || d_model > DIP_MAX_D || d_ff > DIP_MAX_D) return false;
+    if (d_model % 32 || d_ff % 32) return false;
+    if (wtype == DIP_W_INT4_G128 && (d_model % DIP_INT4_GROUP || d_ff % DIP_INT4_GROUP)) return false;
+    return true;
+}
+
+bool weights_ok(const dip_mlp_weights *w)
+{
+    if (!w || !dims_ok(w->wtype, w->d_model, w->d_ff)) return false;
+    if (!w->gate_up || !w->down || !dip_aligned16(w->gate_up) || !dip_aligned16(w->down)) return false;
+    if (w->wtype == DIP_W_INT4_G128 &&
+        (!w->gate_up_scales || !w->down_scales || !dip_aligned16(w->gate_up_scales) ||
+         !dip_aligned16(w->down_scales)))
+        return false;
+    return true;
+}
+
+bool cache_ok(const dip_cache_state *c, int d)
+{
+    return c && c->d == d && c->capacity >= 0 && c->capacity <= d && c->stamp && c->meta &&
+           dip_aligned16(c->stamp) && dip_aligned16(c->meta);
+}
+
+template <typename T> dip_status dev_alloc(dip_ctx *ctx, T **p, size_t n)
+{
+    DIP_CUDA_TRY(ctx, cudaMalloc((void **)p, n * sizeof(T)));
+    return DIP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *dip_status_string(dip_status s)
+{
+    switch (s) {
+    case DIP_OK: return "ok";
+    case DIP_ERR_INVALID_ARG: return "invalid argument";
+    case DIP_ERR_UNSUPPORTED: return "unsupported request";
+    case DIP_ERR_CUDA: return "CUDA runtime failure";
+    case DIP_ERR_WORKSPACE: return "problem exceeds the context workspace";
+    }
+    return "unknown status";
+}
+
+const char *dip_last_error(const dip_ctx *ctx) { return ctx ? ctx->err : ""; }
+int dip_sm_count(const dip_ctx *ctx) { return ctx ? ctx->sm_count : 0; }
+
+dip_status dip_create(dip_ctx **out, int device)
+{
+    if (!out) return DIP_ERR_INVALID_ARG;
+    *out = nullptr;
+    dip_ctx *ctx = new (std::nothrow) dip_ctx();
+    if (!ctx) return DIP_ERR_CUDA;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->device = device;
+    dip_status st = DIP_OK;
+    auto fail = [&](dip_status s) {
+        // keep the message readable through a static copy: the context is about to go
+        dip_destroy(ctx);
+        return s;
+    };
+    if (cudaSetDevice(device) != cudaSuccess) return fail(DIP_ERR_CUDA);
+    if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+        return fail(DIP_ERR_CUDA);
+    ctx->partials_floats = PARTIALS_FLOATS;
+    ctx->n_tickets = N_TICKETS;
+    const size_t vec = (size_t)DIP_MAX_BATCH * DIP_MAX_D;
+    if ((st = dev_alloc(ctx, &ctx->partials, ctx->partials_floats)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->tickets, (size_t)N_TICKETS)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->h, vec)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->y, vec)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->xa, vec)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->xb, vec)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->mask, vec / 32)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->idx, vec)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->mask_h, vec / 32)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->idx_h, vec)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->union_idx, (size_t)DIP_MAX_D)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->counts, (size_t)8)) != DIP_OK) return fail(st);
+    if (cudaMemset(ctx->tickets, 0, N_TICKETS * sizeof(unsigned int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
+    if (cudaMemset(ctx->counts, 0, 8 * sizeof(int32_t)) != cudaSuccess) return fail(DIP_ERR_CUDA);
+    if ((st = dip_init_mask_kernels(ctx)) != DIP_OK) return fail(st);
+    *out = ctx;
+    return DIP_OK;
+}
+
+dip_status dip_destroy(dip_ctx *ctx)
+{
+    if (!ctx) return DIP_ERR_INVALID_ARG;
+    cudaFree(ctx->partials);
+    cudaFree(ctx->tickets);
+    cudaFree(ctx->h);
+    cudaFree(ctx->y);
+    cudaFree(ctx->xa);
+    cudaFree(ctx->xb);
+    cudaFree(ctx->mask);
+    cudaFree(ctx->idx);
+    cudaFree(ctx->mask_h);
+    cudaFree(ctx->idx_h);
+    cudaFree(ctx->union_idx);
+    cudaFree(ctx->counts);
+    delete ctx;
+    return DIP_OK;
+}
+
+size_t dip_packed_bytes(int wtype, int d_model, int d_ff, int which)
+{
+    if (!dims_ok(wtype, d_model, d_ff) || which < 0 || which > 3) return 0;
+    const size_t n_gu = (size_t)d_model * 2 * (size_t)d_ff, n_d = (size_t)d_ff * (size_t)d_model;
+    if (which == 0) return wtype == DIP_W_F32 ? n_gu * 4 : wtype == DIP_W_BF16 ? n_gu * 2 : n_gu / 2;
+    if (which == 1) return wtype == DIP_W_F32 ? n_d * 4 : wtype == DIP_W_BF16 ? n_d * 2 : n_d / 2;
+    if (wtype != DIP_W_INT4_G128) return 0;
+    if (which == 2) return (size_t)(d_model / DIP_INT4_GROUP) * 2 * (size_t)d_ff * 2;
+    return (size_t)(d_ff / DIP_INT4_GROUP) * (size_t)d_model * 2;
+}
+
+dip_status dip_pack_weights(dip_ctx *ctx, int wtype, int d_model, int d_ff,
+                            const void *Wg, const void *Wu, const void *Wd,
+                            const void *Sg, const void *Su, const void *Sd,
+                            const dip_mlp_weights *out, void *stream)
+{
+    if (!ctx || !Wg || !Wu || !Wd || !out) return DIP_ERR_INVALID_ARG;
+    if (!weights_ok(out) || out->wtype != wtype || out->d_model != d_model || out->d_ff != d_ff)
+        return DIP_ERR_INVALID_ARG;
+    if (wtype == DIP_W_INT4_G128 && (!Sg || !Su || !Sd)) return DIP_ERR_INVALID_ARG;
+    return dip_launch_pack(ctx, wtype, d_model, d_ff, Wg, Wu, Wd, Sg, Su, Sd, out, (cudaStream_t)stream);
+}
+
+dip_status dip_mask_topk(dip_ctx *ctx, const float *x, int batch, int d, int k,
+                         uint32_t *mask_bits, int32_t *kept_idx, void *stream)
+{
+    if (!ctx || !x || !dip_aligned16(x)) return DIP_ERR_INVALID_ARG;
+    if (batch < 1 || batch > DIP_MAX_BATCH || d < 1 || d > DIP_MAX_D || k < 1 || k > d) return DIP_ERR_INVALID_ARG;
+    return dip_launch_mask(ctx, x, batch, d, k, 1.0f, nullptr, nullptr, 0, mask_bits, kept_idx,
+                           (cudaStream_t)stream);
+}
+
+dip_status dip_ca_mask(dip_ctx *ctx, const float *x, int d, int k, float gamma,
+                       const dip_cache_state *st,
+                       uint32_t *mask_bits, int32_t *kept_idx, void *stream)
+{
+    if (!ctx || !x || !dip_aligned16(x)) return DIP_ERR_INVALID_ARG;
+    if (d < 1 || d > DIP_MAX_D || k < 1 || k > d) return DIP_ERR_INVALID_ARG;
+    if (!(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
+    if (!cache_ok(st, d)) return DIP_ERR_INVALID_ARG;
+    return dip_launch_mask(ctx, x, 1, d, k, gamma, st->stamp, st->meta, st->capacity, mask_bits, kept_idx,
+                           (cudaStream_t)stream);
+}
+
+static dip_status gemv_entry(dip_ctx *ctx, const dip_mlp_weights *w, int which, const float *v, int batch,
+                             const int32_t *kept_idx, int n_kept, const uint32_t *mask_bits,
+                             float *out, void *stream)
+{
+    if (!ctx || !weights_ok(w) || !v || !kept_idx || !out) return DIP_ERR_INVALID_ARG;
+    if (!dip_aligned16(v) || !dip_aligned16(out)) return DIP_ERR_INVALID_ARG;
+    const int d_in = which == 0 ? w->d_model : w->d_ff;
+    if (batch < 1 || batch > DIP_MAX_BATCH || n_kept < 1 || n_kept > d_in) return DIP_ERR_INVALID_ARG;
+    if (batch > 1 && !mask_bits) return DIP_ERR_INVALID_ARG;
+    return dip_launch_gemv(ctx, w, which, v, batch, kept_idx, n_kept, nullptr,
+                           batch > 1 ? mask_bits : nullptr, out, (cudaStream_t)stream);
+}
+
+dip_status dip_sparse_gemv_gate_up(dip_ctx *ctx, const dip_mlp_weights *w, const float *x, int batch,
+                                   const int32_t *kept_idx, int n_kept, const uint32_t *mask_bits,
+                                   float *h, void *stream)
+{
+    return gemv_entry(ctx, w, 0, x, batch, kept_idx, n_kept, mask_bits, h, stream);
+}
+
+dip_status dip_sparse_gemv_down(dip_ctx *ctx, const dip_mlp_weights *w, const float *h, int batch,
+                                const int32_t *kept_idx, int n_kept, const uint32_t *mask_bits,
+                                float *y, void *stream)
+{
+    return gemv_entry(ctx, w, 1, h, batch, kept_idx, n_kept, mask_bits, y, stream);
+}
+
+dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
+                        const float *x, int batch, int k_x, int k_h, float gamma,
+                        const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                        float *y, const dip_step_outputs *out, void *stream)
+{
+    if (!ctx || !weights_ok(w) || !x || !y || !dip_aligned16(x) || !dip_aligned16(y)) return DIP_ERR_INVALID_ARG;
+    if (batch < 1 || batch > DIP_MAX_BATCH) return DIP_ERR_INVALID_ARG;
+    if (k_x < 1 || k_x > w->d_model || k_h < 1 || k_h > w->d_ff) return DIP_ERR_INVALID_ARG;
+    if (!(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
+    if (cache_gu && !cache_ok(cache_gu, w->d_model)) return DIP_ERR_INVALID_ARG;
+    if (cache_d && !cache_ok(cache_d, w->d_ff)) return DIP_ERR_INVALID_ARG;
+    if (batch > 1 && (cache_gu || cache_d)) return DIP_ERR_UNSUPPORTED;   // Algorithm 1 is per token
+
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t *mask_x = out && out->mask_x ? out->mask_x : ctx->mask;
+    int32_t *idx_x = out && out->idx_x ? out->idx_x : ctx->idx;
+    float *h = out && out->h ? out->h : ctx->h;
+    uint32_t *mask_h = out && out->mask_h ? out->mask_h : ctx->mask_h;
+    int32_t *idx_h = out && out->idx_h ? out->idx_h : ctx->idx_h;
+    dip_status st;
+
+    // m_x = topK(score(x))            (Eq. 7; Algorithm 1 when a cache is given)
+    st = dip_launch_mask(ctx, x, batch, w->d_model, k_x, gamma,
+                         cache_gu ? cache_gu->stamp : nullptr, cache_gu ? cache_gu->meta : nullptr,
+                         cache_gu ? cache_gu->capacity : 0, mask_x, idx_x, s);
+    if (st != DIP_OK) return st;
+    // h = (W~u x) * silu(W~g x)       (Eq. 2 inside Eq. 3)
+    if (batch == 1) {
+        st = dip_launch_gemv(ctx, w, 0, x, 1, idx_x, k_x, nullptr, nullptr, h, s);
+    } else {
+        st = dip_launch_union(ctx, mask_x, batch, w->d_model, ctx->union_idx, ctx->counts + 0, s);
+        if (st != DIP_OK) return st;
+        const long long cap = (long long)batch * k_x;
+        st = dip_launch_gemv(ctx, w, 0, x, batch, ctx->union_idx, cap < w->d_model ? (int)cap : w->d_model,
+                             ctx->counts + 0, mask_x, h, s);
+    }
+    if (st != DIP_OK) return st;
+    // m_h = topK(score(h))            (Eq. 8: the GLU of the already sparsified gate/up)
+    st = dip_launch_mask(ctx, h, batch, w->d_ff, k_h, gamma,
+                         cache_d ? cache_d->stamp : nullptr, cache_d ? cache_d->meta : nullptr,
+                         cache_d ? cache_d->capacity : 0, mask_h, idx_h, s);
+    if (st != DIP_OK) return st;
+    // y = W~d h                       (Eq. 1 inside Eq. 3)
+    if (batch == 1) {
+        st = dip_launch_gemv(ctx, w, 1, h, 1, idx_h, k_h, nullptr, nullptr, y, s);
+    } else {
+        st = dip_launch_union(ctx, mask_h, batch, w->d_ff, ctx->union_idx, ctx->counts + 1, s);
+        if (st != DIP_OK) return st;
+        const long long cap = (long long)batch * k_h;
+        st = dip_launch_gemv(ctx, w, 1, h, batch, ctx->union_idx, cap < w->d_ff ? (int)cap : w->d_ff,
+                             ctx->counts + 1, mask_h, y, s);
+        if (st == DIP_OK && out && out->union_counts)
+            DIP_CUDA_TRY(ctx, cudaMemcpyAsync(out->union_counts, ctx->counts, 2 * sizeof(int32_t),
+                                              cudaMemcpyDeviceToDevice, s));
+    }
+    return st;
+}
+
+dip_status dip_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y,
+                                int batch, int d, float *x_next, void *stream)
+{
+    if (!ctx || !x || !y || !x_next) return DIP_ERR_INVALID_ARG;
+    if (batch < 1 || batch > DIP_MAX_BATCH || d < 1 || d > DIP_MAX_D) return DIP_ERR_INVALID_ARG;
+    return dip_launch_residual_rmsnorm(ctx, x, y, batch, d, x_next, (cudaStream_t)stream);
+}
+
+dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *layers,
+                          const float *x_in, int batch, int k_x, int k_h, float gamma,
+                          const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                          float *x_out, float *y_last, void *stream)
+{
+    if (!ctx || n_layers < 1 || !layers || !x_in || !x_out) return DIP_ERR_INVALID_ARG;
+    if (batch < 1 || batch > DIP_MAX_BATCH) return DIP_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!weights_ok(&layers[l])) return DIP_ERR_INVALID_ARG;
+        if (layers[l].d_model != layers[0].d_model || layers[l].d_ff != layers[0].d_ff) return DIP_ERR_INVALID_ARG;
+    }
+    const int d = layers[0].d_model;
+    const float *cur = x_in;
+    for (int l = 0; l < n_layers; ++l) {
+        float *y = (l == n_layers - 1 && y_last) ? y_last : ctx->y;
+        dip_status st = dip_mlp_step(ctx, &layers[l], cur, batch, k_x, k_h, gamma,
+                                     cache_gu ? &cache_gu[l] : nullptr, cache_d ? &cache_d[l] : nullptr,
+                                     y, nullptr, stream);
+        if (st != DIP_OK) return st;
+        float *next = l == n_layers - 1 ? x_out : ((l & 1) ? ctx->xb : ctx->xa);
+        st = dip_residual_rmsnorm(ctx, cur, y, batch, d, next, stream);
+        if (st != DIP_OK) return st;
+        cur = next;
+    }
+    return DIP_OK;
+}
+
+}  // extern "C"

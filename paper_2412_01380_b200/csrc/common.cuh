@@ -22,8 +22,10 @@ struct dip_ctx {
     float *y;            // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner)
     float *xa;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner ping)
     float *xb;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner pong)
-    uint32_t *mask;      // [DIP_MAX_BATCH][DIP_MAX_D/32]
-    int32_t *idx;        // [DIP_MAX_BATCH][DIP_MAX_D]
+    uint32_t *mask;      // [DIP_MAX_BATCH][DIP_MAX_D/32]  masks of x
+    int32_t *idx;        // [DIP_MAX_BATCH][DIP_MAX_D]     kept indices of x
+    uint32_t *mask_h;    // same for h
+    int32_t *idx_h;
     int32_t *union_idx;  // [DIP_MAX_D]
     int32_t *counts;     // [8] device scalars (union sizes)
     char err[256];
