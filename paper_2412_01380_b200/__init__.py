@@ -1,0 +1,246 @@
+"""Thin Python binding of the sm_100a DIP / DIP-CA sparse decode-MLP library (include/dip.h).
+
+Argument marshalling only: every step of the method runs in the CUDA kernels of
+`libdip.so`.  PyTorch supplies device memory and streams.  There is no CPU
+fallback: importing this package without the built library raises ImportError.
+
+Functions carry the names of the C entry points they call.
+"""
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdip.so")
+
+W_F32, W_BF16, W_INT4_G128 = 0, 1, 2
+MAX_D, MAX_BATCH, INT4_GROUP, CACHE_META_INTS = 32768, 16, 128, 8
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_WORKSPACE = 0, 1, 2, 3, 4
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "%s is missing: build it with `python paper_2412_01380_b200/build.py` "
+        "(nvcc, sm_100a).  This package has no fallback path." % LIB_PATH)
+_lib = C.CDLL(LIB_PATH)
+
+_vp, _i32, _f32 = C.c_void_p, C.c_int, C.c_float
+
+
+class MlpWeightsStruct(C.Structure):
+    _fields_ = [("wtype", C.c_int32), ("d_model", C.c_int32), ("d_ff", C.c_int32), ("reserved", C.c_int32),
+                ("gate_up", _vp), ("gate_up_scales", _vp), ("down", _vp), ("down_scales", _vp)]
+
+
+class CacheStateStruct(C.Structure):
+    _fields_ = [("d", C.c_int32), ("capacity", C.c_int32), ("stamp", _vp), ("meta", _vp)]
+
+
+class StepOutputsStruct(C.Structure):
+    _fields_ = [("mask_x", _vp), ("idx_x", _vp), ("h", _vp), ("mask_h", _vp), ("idx_h", _vp),
+                ("union_counts", _vp)]
+
+
+_lib.dip_create.restype = _i32
+_lib.dip_create.argtypes = [C.POINTER(_vp), _i32]
+_lib.dip_destroy.restype = _i32
+_lib.dip_destroy.argtypes = [_vp]
+_lib.dip_status_string.restype = C.c_char_p
+_lib.dip_status_string.argtypes = [_i32]
+_lib.dip_last_error.restype = C.c_char_p
+_lib.dip_last_error.argtypes = [_vp]
+_lib.dip_sm_count.restype = _i32
+_lib.dip_sm_count.argtypes = [_vp]
+_lib.dip_packed_bytes.restype = C.c_size_t
+_lib.dip_packed_bytes.argtypes = [_i32, _i32, _i32, _i32]
+_lib.dip_pack_weights.restype = _i32
+_lib.dip_pack_weights.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
+                                  C.POINTER(MlpWeightsStruct), _vp]
+_lib.dip_mask_topk.restype = _i32
+_lib.dip_mask_topk.argtypes = [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp]
+_lib.dip_ca_mask.restype = _i32
+_lib.dip_ca_mask.argtypes = [_vp, _vp, _i32, _i32, _f32, C.POINTER(CacheStateStruct), _vp, _vp, _vp]
+for _name in ("dip_sparse_gemv_gate_up", "dip_sparse_gemv_down"):
+    getattr(_lib, _name).restype = _i32
+    getattr(_lib, _name).argtypes = [_vp, C.POINTER(MlpWeightsStruct), _vp, _i32, _vp, _i32, _vp, _vp, _vp]
+_lib.dip_mlp_step.restype = _i32
+_lib.dip_mlp_step.argtypes = [_vp, C.POINTER(MlpWeightsStruct), _vp, _i32, _i32, _i32, _f32,
+                              C.POINTER(CacheStateStruct), C.POINTER(CacheStateStruct), _vp,
+                              C.POINTER(StepOutputsStruct), _vp]
+_lib.dip_residual_rmsnorm.restype = _i32
+_lib.dip_residual_rmsnorm.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp, _vp]
+_lib.dip_stack_step.restype = _i32
+_lib.dip_stack_step.argtypes = [_vp, _i32, C.POINTER(MlpWeightsStruct), _vp, _i32, _i32, _i32, _f32,
+                                C.POINTER(CacheStateStruct), C.POINTER(CacheStateStruct), _vp, _vp, _vp]
+
+EXPORTED = ["dip_create", "dip_destroy", "dip_status_string", "dip_last_error", "dip_sm_count",
+            "dip_packed_bytes", "dip_pack_weights", "dip_mask_topk", "dip_ca_mask",
+            "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_mlp_step",
+            "dip_residual_rmsnorm", "dip_stack_step"]
+
+
+class DipError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        msg = _lib.dip_status_string(status).decode()
+        super().__init__("%s (status %d)%s" % (msg, status, (": " + detail) if detail else ""))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Context:
+    """A dip_ctx: scratch workspace on one device.  Not for concurrent use from several streams."""
+
+    def __init__(self, device: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_2412_01380_b200 needs a CUDA device; there is no CPU path")
+        h = _vp()
+        st = _lib.dip_create(C.byref(h), int(device))
+        if st != OK:
+            raise DipError(st, "dip_create")
+        self.handle = h
+        self.device = int(device)
+
+    def check(self, st: int) -> None:
+        if st != OK:
+            raise DipError(st, _lib.dip_last_error(self.handle).decode())
+
+    @property
+    def sm_count(self) -> int:
+        return _lib.dip_sm_count(self.handle)
+
+    def close(self) -> None:
+        if self.handle:
+            _lib.dip_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class MlpWeights:
+    """Packed weights of one MLP block (device tensors owned here) plus the C struct naming them."""
+
+    def __init__(self, wtype: int, d_model: int, d_ff: int, device):
+        self.wtype, self.d_model, self.d_ff = int(wtype), int(d_model), int(d_ff)
+        sizes = [_lib.dip_packed_bytes(wtype, d_model, d_ff, w) for w in range(4)]
+        if sizes[0] == 0:
+            raise DipError(ERR_INVALID_ARG, "unsupported weight type or shape")
+        self.gate_up = torch.empty(sizes[0], dtype=torch.uint8, device=device)
+        self.down = torch.empty(sizes[1], dtype=torch.uint8, device=device)
+        self.gate_up_scales = torch.empty(sizes[2], dtype=torch.uint8, device=device) if sizes[2] else None
+        self.down_scales = torch.empty(sizes[3], dtype=torch.uint8, device=device) if sizes[3] else None
+        self.struct = MlpWeightsStruct(self.wtype, self.d_model, self.d_ff, 0, _ptr(self.gate_up),
+                                       _ptr(self.gate_up_scales), _ptr(self.down), _ptr(self.down_scales))
+
+    @property
+    def nbytes(self) -> int:
+        return sum(t.numel() for t in (self.gate_up, self.down, self.gate_up_scales, self.down_scales)
+                   if t is not None)
+
+
+class CacheState:
+    """Column-cache state of one masked layer input: stamp int32[d], meta int32[8] on the device."""
+
+    def __init__(self, d: int, capacity: int, device):
+        self.d, self.capacity = int(d), int(capacity)
+        self.stamp = torch.full((d,), -1, dtype=torch.int32, device=device)
+        self.meta = torch.zeros(CACHE_META_INTS, dtype=torch.int32, device=device)
+        self.struct = CacheStateStruct(self.d, self.capacity, _ptr(self.stamp), _ptr(self.meta))
+
+    def load(self, stamp, n_resident: int, step: int, counters=(0, 0, 0, 0)) -> None:
+        self.stamp.copy_(torch.as_tensor(stamp, dtype=torch.int32))
+        self.meta.copy_(torch.tensor([n_resident, step, *counters, 0, 0], dtype=torch.int32))
+
+
+def dip_packed_bytes(wtype: int, d_model: int, d_ff: int, which: int) -> int:
+    return int(_lib.dip_packed_bytes(wtype, d_model, d_ff, which))
+
+
+def dip_pack_weights(ctx: Context, wtype: int, d_model: int, d_ff: int,
+                     Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor,
+                     Sg: Optional[torch.Tensor] = None, Su: Optional[torch.Tensor] = None,
+                     Sd: Optional[torch.Tensor] = None, out: Optional[MlpWeights] = None) -> MlpWeights:
+    """Canonical device tensors ([d_out, d_in] row-major) -> packed MlpWeights."""
+    if out is None:
+        out = MlpWeights(wtype, d_model, d_ff, Wg.device)
+    for t in (Wg, Wu, Wd, Sg, Su, Sd):
+        assert t is None or (t.is_cuda and t.is_contiguous())
+    ctx.check(_lib.dip_pack_weights(ctx.handle, wtype, d_model, d_ff, _ptr(Wg), _ptr(Wu), _ptr(Wd),
+                                    _ptr(Sg), _ptr(Su), _ptr(Sd), C.byref(out.struct), _stream()))
+    return out
+
+
+def dip_mask_topk(ctx: Context, x: torch.Tensor, k: int, mask_bits: Optional[torch.Tensor],
+                  kept_idx: Optional[torch.Tensor]) -> None:
+    batch, d = (1, x.numel()) if x.dim() == 1 else x.shape
+    ctx.check(_lib.dip_mask_topk(ctx.handle, _ptr(x), batch, d, int(k), _ptr(mask_bits), _ptr(kept_idx),
+                                 _stream()))
+
+
+def dip_ca_mask(ctx: Context, x: torch.Tensor, k: int, gamma: float, st: CacheState,
+                mask_bits: Optional[torch.Tensor], kept_idx: Optional[torch.Tensor]) -> None:
+    ctx.check(_lib.dip_ca_mask(ctx.handle, _ptr(x), x.numel(), int(k), float(gamma), C.byref(st.struct),
+                               _ptr(mask_bits), _ptr(kept_idx), _stream()))
+
+
+def dip_sparse_gemv_gate_up(ctx: Context, w: MlpWeights, x: torch.Tensor, kept_idx: torch.Tensor, n_kept: int,
+                            mask_bits: Optional[torch.Tensor], h: torch.Tensor) -> None:
+    batch = 1 if x.dim() == 1 else x.shape[0]
+    ctx.check(_lib.dip_sparse_gemv_gate_up(ctx.handle, C.byref(w.struct), _ptr(x), batch, _ptr(kept_idx),
+                                           int(n_kept), _ptr(mask_bits), _ptr(h), _stream()))
+
+
+def dip_sparse_gemv_down(ctx: Context, w: MlpWeights, h: torch.Tensor, kept_idx: torch.Tensor, n_kept: int,
+                         mask_bits: Optional[torch.Tensor], y: torch.Tensor) -> None:
+    batch = 1 if h.dim() == 1 else h.shape[0]
+    ctx.check(_lib.dip_sparse_gemv_down(ctx.handle, C.byref(w.struct), _ptr(h), batch, _ptr(kept_idx),
+                                        int(n_kept), _ptr(mask_bits), _ptr(y), _stream()))
+
+
+def dip_mlp_step(ctx: Context, w: MlpWeights, x: torch.Tensor, k_x: int, k_h: int, gamma: float,
+                 cache_gu: Optional[CacheState], cache_d: Optional[CacheState], y: torch.Tensor,
+                 mask_x=None, idx_x=None, h=None, mask_h=None, idx_h=None, union_counts=None) -> None:
+    batch = 1 if x.dim() == 1 else x.shape[0]
+    outs = StepOutputsStruct(_ptr(mask_x), _ptr(idx_x), _ptr(h), _ptr(mask_h), _ptr(idx_h), _ptr(union_counts))
+    ctx.check(_lib.dip_mlp_step(ctx.handle, C.byref(w.struct), _ptr(x), batch, int(k_x), int(k_h), float(gamma),
+                                C.byref(cache_gu.struct) if cache_gu else None,
+                                C.byref(cache_d.struct) if cache_d else None,
+                                _ptr(y), C.byref(outs), _stream()))
+
+
+def dip_residual_rmsnorm(ctx: Context, x: torch.Tensor, y: torch.Tensor, x_next: torch.Tensor) -> None:
+    batch, d = (1, x.numel()) if x.dim() == 1 else x.shape
+    ctx.check(_lib.dip_residual_rmsnorm(ctx.handle, _ptr(x), _ptr(y), batch, d, _ptr(x_next), _stream()))
+
+
+class Stack:
+    """Host arrays naming the layers (and caches) of an MLP stack for dip_stack_step."""
+
+    def __init__(self, layers: Sequence[MlpWeights], cache_gu: Optional[Sequence[CacheState]] = None,
+                 cache_d: Optional[Sequence[CacheState]] = None):
+        self.layers: List[MlpWeights] = list(layers)
+        self.cache_gu = list(cache_gu) if cache_gu is not None else None
+        self.cache_d = list(cache_d) if cache_d is not None else None
+        n = len(self.layers)
+        self.w_arr = (MlpWeightsStruct * n)(*[l.struct for l in self.layers])
+        self.gu_arr = (CacheStateStruct * n)(*[c.struct for c in self.cache_gu]) if self.cache_gu else None
+        self.d_arr = (CacheStateStruct * n)(*[c.struct for c in self.cache_d]) if self.cache_d else None
+
+
+def dip_stack_step(ctx: Context, stack: Stack, x_in: torch.Tensor, k_x: int, k_h: int, gamma: float,
+                   x_out: torch.Tensor, y_last: Optional[torch.Tensor] = None) -> None:
+    batch = 1 if x_in.dim() == 1 else x_in.shape[0]
+    ctx.check(_lib.dip_stack_step(ctx.handle, len(stack.layers), stack.w_arr, _ptr(x_in), batch, int(k_x),
+                                  int(k_h), float(gamma), stack.gu_arr, stack.d_arr, _ptr(x_out),
+                                  _ptr(y_last), _stream()))

@@ -1,0 +1,70 @@
+"""Helpers shared by the GPU parity tests: upload synthetic layers, wrap oracle matrices, error metric."""
+import numpy as np
+import torch
+
+import dip_inputs as di
+import oracle
+
+REL_TOL = 2e-3   # max relative error, bf16/fp32 weights with binary32 accumulation vs the fp64 oracle
+
+
+def rel_err(got: np.ndarray, ref: np.ndarray) -> float:
+    """max_j |got_j - ref_j| / max(|ref_j|, rms(ref)): element-wise relative error with the
+    denominator floored at the vector's RMS so that near-zero outputs do not dominate."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    den = np.maximum(np.abs(ref), max(rms, 1e-300))
+    return float(np.max(np.abs(got - ref) / den))
+
+
+def oracle_mats(lw: di.LayerWeights):
+    t = lw.wtype
+    return (oracle.Matrix(t, lw.gate, lw.gate_scales, lw.d_ff, lw.d_model),
+            oracle.Matrix(t, lw.up, lw.up_scales, lw.d_ff, lw.d_model),
+            oracle.Matrix(t, lw.down, lw.down_scales, lw.d_model, lw.d_ff))
+
+
+def _dev(a, dtype=None):
+    if a is None:
+        return None
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.view(dtype)
+    return t.cuda()
+
+
+def upload_layer(dip, ctx, lw: di.LayerWeights):
+    """Canonical host arrays -> device -> dip_pack_weights."""
+    if lw.wtype == di.W_BF16:
+        args = [_dev(lw.gate.view(np.int16)), _dev(lw.up.view(np.int16)), _dev(lw.down.view(np.int16))]
+        sc = [None, None, None]
+    elif lw.wtype == di.W_F32:
+        args = [_dev(lw.gate), _dev(lw.up), _dev(lw.down)]
+        sc = [None, None, None]
+    else:
+        args = [_dev(lw.gate), _dev(lw.up), _dev(lw.down)]
+        sc = [_dev(lw.gate_scales.view(np.int16)), _dev(lw.up_scales.view(np.int16)),
+              _dev(lw.down_scales.view(np.int16))]
+    w = dip.dip_pack_weights(ctx, lw.wtype, lw.d_model, lw.d_ff, *args, *sc)
+    torch.cuda.synchronize()
+    return w
+
+
+def bits_to_mask(bits: torch.Tensor, d: int) -> np.ndarray:
+    """uint32 words (as int32 tensor) -> uint8 [.., d] 0/1 array."""
+    w = bits.cpu().numpy().view(np.uint32)
+    m = ((w[..., :, None] >> np.arange(32, dtype=np.uint32)) & 1).astype(np.uint8)
+    return m.reshape(*w.shape[:-1], -1)[..., :d]
+
+
+def gpu_cache_from_oracle(dip, c: "oracle.Cache"):
+    g = dip.CacheState(c.d, c.capacity, "cuda")
+    g.load(c.stamp, int(c.n_resident[0]), int(c.step[0]), tuple(int(v) for v in c.counters))
+    return g
+
+
+def cache_equal(g, c: "oracle.Cache") -> bool:
+    meta = g.meta.cpu().numpy()
+    return (np.array_equal(g.stamp.cpu().numpy(), c.stamp) and meta[0] == c.n_resident[0]
+            and meta[1] == c.step[0] and np.array_equal(meta[2:6], c.counters))
