@@ -91,7 +91,7 @@ def test_mask_topk_adversarial_ties(dip, ctx):
 ])
 def test_ca_mask_and_cache_state_bit_exact(dip, ctx, d, k, cap, gamma):
     w = di.WORKLOADS["phi3_mini"].scaled(seed=d + k + cap)
-    n_tok = 24 if d <= 8192 else 10
+    n_tok = 24
     xs = di.token_inputs(w, n_tokens=n_tok, batch=1, d=d)[:, 0]
     # correlate successive tokens a little so that hits, misses and evictions all occur
     for t in range(1, n_tok):
@@ -111,7 +111,8 @@ def test_ca_mask_and_cache_state_bit_exact(dip, ctx, d, k, cap, gamma):
     c = ref.counters
     assert c[0] + c[1] == n_tok * k
     if 0 < cap < d and k <= cap:
-        assert c[0] > 0 and c[2] > 0          # the trace exercised hits and evictions
+        assert c[0] > 0                       # the trace exercised hits
+        assert c[2] > 0 or c[1] <= cap        # and evictions, once the misses exceed the cache
     if k > cap:
         assert c[3] > 0                       # and the bypass rule
 
