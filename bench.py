@@ -1,0 +1,441 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse SwiGLU decode-MLP path (DIP / DIP-CA) on B200.
+
+A step is one decode token through the whole MLP stack of the workload (n_layers MLP-steps:
+mask x, gate/up GEMV + silu*up, mask h, down GEMV, residual + rmsnorm per layer).  The layers
+are distinct and the stack is far larger than L2, so every step streams its kept weight
+columns from HBM.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload NAME] [--keep-ratio R] [--cache-budget B] [--no-sweep]
+
+With N > 1 (torchrun) every rank runs an independent replica of the stack on its own
+sequence ("replicas only": the path has no exchange step); value = MLP-steps of all ranks
+divided by the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import dip_inputs as di  # noqa: E402
+
+METRIC = "sparse_swiglu_decode_mlp_steps_per_s"
+UNIT = "MLP-steps/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="phi3_medium", choices=sorted(di.WORKLOADS))
+    ap.add_argument("--keep-ratio", type=float, default=None)
+    ap.add_argument("--cache-budget", type=float, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging; not a valid bench)")
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def weight_bytes(wtype):
+    return {di.W_F32: 4.0, di.W_BF16: 2.0, di.W_INT4_G128: 0.5}[wtype]
+
+
+def algorithmic_bytes(w, k_x, k_h, ca):
+    """Bytes the method has to move per MLP-step: the kept weight columns plus activations,
+    index lists and (cache-aware masking on) the cache stamps.  INT4 adds the scale rows of the
+    groups touched (bounded by all groups)."""
+    bw = weight_bytes(w.wtype)
+    gu = k_x * 2 * w.d_ff * bw + 4 * w.d_model + 4 * k_x + 4 * w.d_ff
+    dn = k_h * w.d_model * bw + 4 * w.d_ff + 4 * k_h + 4 * w.d_model
+    if w.wtype == di.W_INT4_G128:
+        gu += min(k_x, w.d_model // di.GROUP) * 2 * w.d_ff * 2
+        dn += min(k_h, w.d_ff // di.GROUP) * w.d_model * 2
+    masks = 4 * (w.d_model + w.d_ff) + 4 * (k_x + k_h)
+    if ca:
+        masks += 8 * (w.d_model + w.d_ff)
+    return {"gate_up": gu, "down": dn, "step": gu + dn + masks}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_stack(dip, ctx, torch, w, n_layers, rank):
+    """Draw and pack the stack's weights on the device (one canonical layer at a time)."""
+    from dip_inputs import device as dd
+    dev = "cuda"
+    layers = []
+    for l in range(n_layers):
+        g, gs = dd.matrix(w, l, "gate", w.d_ff, w.d_model, dev, rank)
+        u, us = dd.matrix(w, l, "up", w.d_ff, w.d_model, dev, rank)
+        d_, ds = dd.matrix(w, l, "down", w.d_model, w.d_ff, dev, rank)
+        layers.append(dip.dip_pack_weights(ctx, w.wtype, w.d_model, w.d_ff, g, u, d_, gs, us, ds))
+        torch.cuda.synchronize()
+        del g, u, d_, gs, us, ds
+    return layers
+
+
+def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, warmup, use_graph=True,
+               kernel_pass=True, e2e_pass=True, sampler=None, dist=None):
+    """Time `steps` decode tokens through the stack at one (keep ratio, cache budget)."""
+    L, d_model, d_ff = len(layers), w.d_model, w.d_ff
+    k_x, k_h = di.keep_count(keep_ratio, d_model), di.keep_count(keep_ratio, d_ff)
+    ca = budget is not None
+    gamma = w.gamma if ca else 1.0
+
+    def fresh_stack():
+        if not ca:
+            return dip.Stack(layers)
+        cg = [dip.CacheState(d_model, di.cache_capacity(budget, d_model), "cuda") for _ in range(L)]
+        cd = [dip.CacheState(d_ff, di.cache_capacity(budget, d_ff), "cuda") for _ in range(L)]
+        return dip.Stack(layers, cg, cd)
+
+    n_tok = xs_host.shape[0]
+    xs_dev = xs_host.cuda()
+    x_cur = torch.empty(d_model, device="cuda")
+    x_out = torch.empty(d_model, device="cuda")
+    out_host = torch.empty(d_model).pin_memory()
+    stack = fresh_stack()
+    stream = torch.cuda.current_stream()
+
+    graph = None
+    if use_graph:
+        # capture one token through the stack; replays read x_cur and update the caches in place
+        x_cur.copy_(xs_dev[0])
+        dip.dip_stack_step(ctx, stack, x_cur, k_x, k_h, gamma, x_out)      # prime outside capture
+        torch.cuda.synchronize()
+        stack = fresh_stack()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            dip.dip_stack_step(ctx, stack, x_cur, k_x, k_h, gamma, x_out)
+
+    def one_step(t):
+        x_cur.copy_(xs_dev[t % n_tok], non_blocking=True)
+        if graph is not None:
+            graph.replay()
+        else:
+            dip.dip_stack_step(ctx, stack, x_cur, k_x, k_h, gamma, x_out)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing ----
+    for t in range(warmup):
+        one_step(t)
+    barrier()
+    if sampler:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for t in range(steps):
+        one_step(warmup + t)
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tms = torch.tensor([ms], device="cuda")
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+        ms = float(tms.item())
+    res = {"keep_ratio": keep_ratio, "cache_budget": budget, "k_x": k_x, "k_h": k_h, "ms_total": ms,
+           "ms_per_step": ms / steps, "mlp_steps_per_s": L * steps / (ms * 1e-3), "clocks": clocks,
+           "bytes": algorithmic_bytes(w, k_x, k_h, ca)}
+    res["step_gbs"] = res["bytes"]["step"] * L * steps / (ms * 1e-3) / 1e9
+    if ca:
+        meta = torch.stack([c.meta for c in stack.cache_gu + stack.cache_d]).sum(0).cpu().tolist()
+        res["hit_rate"] = meta[2] / max(1, meta[2] + meta[3])
+
+    # ---- end to end: host buffers in, host result out, every step ----
+    if e2e_pass:
+        xs_pin = xs_host.pin_memory()
+        n_e2e = min(steps, 128)
+        for t in range(3):
+            one_step(t)
+        barrier()
+        t0 = time.perf_counter()
+        e0.record(stream)
+        for t in range(n_e2e):
+            x_cur.copy_(xs_pin[(warmup + t) % n_tok], non_blocking=True)
+            if graph is not None:
+                graph.replay()
+            else:
+                dip.dip_stack_step(ctx, stack, x_cur, k_x, k_h, gamma, x_out)
+            out_host.copy_(x_out, non_blocking=True)
+            stream.synchronize()          # a decode loop needs the result before the next token
+        e1.record(stream)
+        barrier()
+        ms_e = e0.elapsed_time(e1)
+        if dist is not None:
+            tms = torch.tensor([ms_e], device="cuda")
+            dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+            ms_e = float(tms.item())
+        res["e2e"] = {"value": L * n_e2e / (ms_e * 1e-3), "unit": UNIT, "steps": n_e2e,
+                      "h2d_bytes_per_step": 4 * d_model, "d2h_bytes_per_step": 4 * d_model,
+                      "wall_ms": (time.perf_counter() - t0) * 1e3}
+
+    # ---- per-kernel durations (separate instrumented pass, one event pair per launch) ----
+    if kernel_pass:
+        st2 = fresh_stack()
+        mask_x = torch.zeros((d_model + 31) // 32, dtype=torch.int32, device="cuda")
+        idx_x = torch.zeros(k_x, dtype=torch.int32, device="cuda")
+        mask_h = torch.zeros((d_ff + 31) // 32, dtype=torch.int32, device="cuda")
+        idx_h = torch.zeros(k_h, dtype=torch.int32, device="cuda")
+        h = torch.empty(d_ff, device="cuda")
+        y = torch.empty(d_model, device="cuda")
+        n_pass_tok = 6
+        names = ["mask_x", "gate_up", "mask_h", "down", "rmsnorm"]
+        evs = []
+        for t in range(n_pass_tok):
+            cur = xs_dev[t % n_tok].clone()
+            for l in range(L):
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+                ev[0].record(stream)
+                if ca:
+                    dip.dip_ca_mask(ctx, cur, k_x, gamma, st2.cache_gu[l], mask_x, idx_x)
+                else:
+                    dip.dip_mask_topk(ctx, cur, k_x, mask_x, idx_x)
+                ev[1].record(stream)
+                dip.dip_sparse_gemv_gate_up(ctx, layers[l], cur, idx_x, k_x, None, h)
+                ev[2].record(stream)
+                if ca:
+                    dip.dip_ca_mask(ctx, h, k_h, gamma, st2.cache_d[l], mask_h, idx_h)
+                else:
+                    dip.dip_mask_topk(ctx, h, k_h, mask_h, idx_h)
+                ev[3].record(stream)
+                dip.dip_sparse_gemv_down(ctx, layers[l], h, idx_h, k_h, None, y)
+                ev[4].record(stream)
+                dip.dip_residual_rmsnorm(ctx, cur, y, cur)
+                ev[5].record(stream)
+                if t >= 2:
+                    evs.append(ev)
+        torch.cuda.synchronize()
+        kern = {}
+        for i, n in enumerate(names):
+            kern[n + "_us"] = float(np.mean([e[i].elapsed_time(e[i + 1]) for e in evs])) * 1e3
+        res["kernels"] = kern
+    return res
+
+
+def oracle_rate(w, keep_ratio, budget, n_layers_sample, n_steps, warmup=0):
+    """The CPU oracle as it stands, timed on this machine's host cores on a bounded sample of the
+    workload: `n_steps` MLP-steps cycling over `n_layers_sample` host-generated layers."""
+    import oracle
+    k_x, k_h = di.keep_count(keep_ratio, w.d_model), di.keep_count(keep_ratio, w.d_ff)
+    ca = budget is not None
+    gamma = w.gamma if ca else 1.0
+    lws = [di.layer_weights(w, l) for l in range(n_layers_sample)]
+    mats = [(oracle.Matrix(lw.wtype, lw.gate, lw.gate_scales, w.d_ff, w.d_model),
+             oracle.Matrix(lw.wtype, lw.up, lw.up_scales, w.d_ff, w.d_model),
+             oracle.Matrix(lw.wtype, lw.down, lw.down_scales, w.d_model, w.d_ff)) for lw in lws]
+    cg = [oracle.Cache(w.d_model, di.cache_capacity(budget, w.d_model)) if ca else None for _ in lws]
+    cd = [oracle.Cache(w.d_ff, di.cache_capacity(budget, w.d_ff)) if ca else None for _ in lws]
+    n_tok = (warmup + n_steps + n_layers_sample - 1) // n_layers_sample + 1
+    xs = di.token_inputs(w, n_tokens=n_tok, batch=1)[:, 0]
+    cur, t_idx, times = xs[0], 0, []
+    for s in range(warmup + n_steps):
+        l = s % n_layers_sample
+        if l == 0:
+            t_idx += 1
+            cur = xs[t_idx % n_tok]
+        t0 = time.perf_counter()
+        r = oracle.mlp_step(*mats[l], cur, k_x, k_h, gamma, cg[l], cd[l])
+        cur = oracle.residual_rmsnorm(cur, r.y)
+        if s >= warmup:
+            times.append(time.perf_counter() - t0)
+    total = float(np.sum(times))
+    return {"value": n_steps / total, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "%d MLP-steps over %d host-generated layer(s) of %s, keep ratio %g, cache budget %s"
+                      % (n_steps, n_layers_sample, w.name, keep_ratio, budget),
+            "ms_per_mlp_step": total / n_steps * 1e3}
+
+
+def main_reference(args, w, keep_ratio, budget):
+    """The reference arm: the CPU oracle timed on the host cores; a step is one MLP-step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    r = oracle_rate(w, keep_ratio, budget, 1, args.steps, args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_mlp_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic",
+            "config": {"workload": w.name, "keep_ratio": keep_ratio, "cache_budget": budget,
+                       "d_model": w.d_model, "d_ff": w.d_ff, "step": "one MLP-step (1 layer x 1 token) of the CPU oracle"},
+            "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    w = di.WORKLOADS[args.workload]
+    keep_ratio = args.keep_ratio if args.keep_ratio is not None else w.keep_ratio
+    budget = args.cache_budget if args.cache_budget is not None else w.cache_budget
+    if args.impl == "reference":
+        return main_reference(args, w, keep_ratio, budget)
+
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+
+    import paper_2412_01380_b200 as dip
+    ctx = dip.Context(local)
+    L = args.layers if args.layers else w.n_layers
+    layers = build_stack(dip, ctx, torch, w, L, rank)
+    n_tok = min(w.n_tokens, args.steps + args.warmup)
+    wl_rank = w.scaled(seed=w.seed + 1000 * rank)
+    xs_host = torch.from_numpy(di.token_inputs(wl_rank, n_tokens=n_tok, batch=1)[:, 0].copy())
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
+                           else int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])) if rank == 0 else None
+    head = run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, args.steps, args.warmup,
+                      sampler=sampler, dist=dist)
+
+    sweep = []
+    if not args.no_sweep and world == 1 and w.name == "phi3_medium":
+        for rho in di.PHI3_MEDIUM_KEEP_RATIOS:
+            for beta in di.PHI3_MEDIUM_CACHE_BUDGETS:
+                r = run_config(dip, ctx, torch, w, layers, xs_host, rho, beta, min(args.steps, 64), 4,
+                               kernel_pass=True, e2e_pass=False)
+                sweep.append(r)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    gu_bytes = head["bytes"]["gate_up"]
+    gu_us = head["kernels"]["gate_up_us"]
+    achieved = gu_bytes / (gu_us * 1e-6) / 1e9
+    launches_per_step = L * 5
+    line = {
+        "metric": METRIC, "value": head["mlp_steps_per_s"] * world, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": {di.W_F32: "f32", di.W_BF16: "bf16 weights, f32 accumulate", di.W_INT4_G128: "int4 weights, f32 accumulate"}[w.wtype],
+        "data": "synthetic",
+        "config": {"workload": w.name, "n_layers": L, "d_model": w.d_model, "d_ff": w.d_ff,
+                   "keep_ratio": keep_ratio, "k_x": head["k_x"], "k_h": head["k_h"], "cache_budget": budget,
+                   "gamma": w.gamma if budget is not None else 1.0, "batch": 1,
+                   "step": "one decode token through %d layers = %d MLP-steps" % (L, L),
+                   "l2": "inputs larger than L2: %.1f GB of distinct layer weights cycled" % (sum(l.nbytes for l in layers) / 1e9),
+                   "launch": "CUDA graph of dip_stack_step", "parallelism": "replicas only"},
+        "mlp_step_us": head["ms_per_step"] * 1e3 / L,
+        "step_gbs": head["step_gbs"] * world,
+        "step_frac_of_measured_hbm": head["step_gbs"] / peak,
+        "step_frac_of_nominal_8tbs": head["step_gbs"] / NOMINAL_HBM_GBS,
+        "hit_rate": head.get("hit_rate"),
+        "clocks": head["clocks"],
+        "e2e": {k: head["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "gemv_kernel (gate/up bundle)", "achieved": achieved, "peak": peak,
+                     "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS, "bytes_per_launch": gu_bytes,
+                     "us_per_launch": gu_us, "traffic": None},
+        "kernels_us": head["kernels"],
+    }
+    line["e2e"]["value"] *= world
+    if sweep:
+        line["sweep"] = [{"keep_ratio": r["keep_ratio"], "cache_budget": r["cache_budget"],
+                          "mlp_steps_per_s": r["mlp_steps_per_s"], "mlp_step_us": r["ms_per_step"] * 1e3 / L,
+                          "step_gbs": r["step_gbs"], "frac_of_measured": r["step_gbs"] / peak,
+                          "frac_of_nominal_8tbs": r["step_gbs"] / NOMINAL_HBM_GBS, "hit_rate": r.get("hit_rate"),
+                          "gate_up_gbs": r["bytes"]["gate_up"] / (r["kernels"]["gate_up_us"] * 1e-6) / 1e9,
+                          "down_gbs": r["bytes"]["down"] / (r["kernels"]["down_us"] * 1e-6) / 1e9,
+                          "kernels_us": r["kernels"]} for r in sweep]
+    if world == 1 and not args.no_cpu_baseline:
+        del layers
+        torch.cuda.empty_cache()
+        line["cpu_baseline"] = {k: v for k, v in oracle_rate(w, keep_ratio, budget, 1, 60).items()
+                                if k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
