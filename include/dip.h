@@ -256,6 +256,45 @@ dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *lay
                           const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
                           float *x_out, float *y_last, void *stream);
 
+/* ------------------------------------------------------------------------
+ * dip_sparse_gemv_down_noalloc — the down product y = W~d h of
+ * dip_sparse_gemv_down (batch 1, F32 or BF16 weights) for callers that are not
+ * allowed to allocate device memory.  The paper has no counterpart of this
+ * call; it exists for integration only.
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits — inside a
+ * framework that owns the whole memory pool and forbids foreign allocations,
+ * in a latency-critical serving loop where an allocation (an implicit device
+ * synchronisation) is not acceptable, or in a process that has handed all of
+ * the device's free memory to its own allocator, so that creating a dip_ctx
+ * (which allocates its workspace) would fail.  This call takes no context:
+ * the split-row partial sums and arrival counters that the context-based call
+ * keeps in its workspace live in a fixed array of about 4 MB inside the
+ * library image instead.  Every GPU that loads the library holds that array
+ * until the process exits, whether or not this call is used.
+ *
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.  The
+ * first call on a device looks up the array's device address and the device's
+ * SM count (once per device, with that device current); make that first call
+ * before any stream capture.  The device used is the calling thread's current
+ * device; w, h, kept_idx and y must live there.
+ *
+ * Limits: d_model <= 16384 (DIP_ERR_WORKSPACE beyond it: the fixed array
+ * cannot hold the partial sums), d_model % 32 == 0, 1 <= n_kept <= d_ff <=
+ * DIP_MAX_D; INT4 weights return DIP_ERR_UNSUPPORTED.  Only w->wtype,
+ * w->d_model, w->d_ff and w->down are read.
+ *
+ * All calls on a device share the one array, which keeps the previous call's
+ * contents (each call clears the counters it needs on `stream` first).  Two
+ * calls that overlap on the GPU — different streams, or different host
+ * threads without ordering — race on it and give wrong results: serialise them.
+ * The result equals dip_sparse_gemv_down's up to the order of the binary32
+ * sums (the split into row parts may differ).
+ * ------------------------------------------------------------------------ */
+dip_status dip_sparse_gemv_down_noalloc(const dip_mlp_weights *w, const float *h,
+                                        const int32_t *kept_idx, int n_kept,
+                                        float *y, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

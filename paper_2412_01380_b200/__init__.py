@@ -74,10 +74,13 @@ _lib.dip_stack_step.restype = _i32
 _lib.dip_stack_step.argtypes = [_vp, _i32, C.POINTER(MlpWeightsStruct), _vp, _i32, _i32, _i32, _f32,
                                 C.POINTER(CacheStateStruct), C.POINTER(CacheStateStruct), _vp, _vp, _vp]
 
+_lib.dip_sparse_gemv_down_noalloc.restype = _i32
+_lib.dip_sparse_gemv_down_noalloc.argtypes = [C.POINTER(MlpWeightsStruct), _vp, _vp, _i32, _vp, _vp]
+
 EXPORTED = ["dip_create", "dip_destroy", "dip_status_string", "dip_last_error", "dip_sm_count",
             "dip_packed_bytes", "dip_pack_weights", "dip_mask_topk", "dip_ca_mask",
             "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_mlp_step",
-            "dip_residual_rmsnorm", "dip_stack_step"]
+            "dip_residual_rmsnorm", "dip_stack_step", "dip_sparse_gemv_down_noalloc"]
 
 
 class DipError(RuntimeError):
@@ -244,3 +247,23 @@ def dip_stack_step(ctx: Context, stack: Stack, x_in: torch.Tensor, k_x: int, k_h
     ctx.check(_lib.dip_stack_step(ctx.handle, len(stack.layers), stack.w_arr, _ptr(x_in), batch, int(k_x),
                                   int(k_h), float(gamma), stack.gu_arr, stack.d_arr, _ptr(x_out),
                                   _ptr(y_last), _stream()))
+
+
+def dip_sparse_gemv_down_noalloc(w: MlpWeights, h: torch.Tensor, kept_idx: torch.Tensor, n_kept: int,
+                                 y: torch.Tensor) -> None:
+    """y = W~d h without a Context and without any device allocation by the library.
+
+    For callers that cannot let this library allocate: hosts whose memory pool is owned by a
+    framework, serving loops that cannot afford the synchronisation an allocation implies, or
+    processes with no free device memory left for a Context's workspace.  Scratch comes from a
+    fixed ~4 MB array inside the library image, shared by every call on the device, so calls
+    that overlap on the GPU race: keep them on one stream.  d_model is limited to 16384
+    (ERR_WORKSPACE beyond); F32 and BF16 weights only.  The first call on a device does a
+    one-off address look-up and should come before any stream capture.
+    """
+    st = _lib.dip_sparse_gemv_down_noalloc(C.byref(w.struct), _ptr(h), _ptr(kept_idx), int(n_kept), _ptr(y),
+                                           _stream())
+    if st == ERR_WORKSPACE:
+        raise DipError(st, "d_model exceeds the no-allocation entry point's fixed scratch (max 16384)")
+    if st != OK:
+        raise DipError(st, "dip_sparse_gemv_down_noalloc")
