@@ -86,6 +86,7 @@ dip_status dip_create(dip_ctx **out, int device)
     if ((st = dev_alloc(ctx, &ctx->tickets, (size_t)N_TICKETS)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->h, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->y, vec)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->y2, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->xa, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->xb, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask, vec / 32)) != DIP_OK) return fail(st);
@@ -108,6 +109,7 @@ dip_status dip_destroy(dip_ctx *ctx)
     cudaFree(ctx->tickets);
     cudaFree(ctx->h);
     cudaFree(ctx->y);
+    cudaFree(ctx->y2);
     cudaFree(ctx->xa);
     cudaFree(ctx->xb);
     cudaFree(ctx->mask);
@@ -191,12 +193,17 @@ dip_status dip_sparse_gemv_down(dip_ctx *ctx, const dip_mlp_weights *w, const fl
     return gemv_entry(ctx, w, 1, h, batch, kept_idx, n_kept, mask_bits, y, stream);
 }
 
-dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
-                        const float *x, int batch, int k_x, int k_h, float gamma,
-                        const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
-                        float *y, const dip_step_outputs *out, void *stream)
+// One sparse MLP step.  xb != nullptr: the step's input is formed first as
+// x = (xa + xb) / rms(xa + xb), written to x_norm, in the same launch as its mask.
+static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
+                            const float *xa, const float *xb, float *x_norm,
+                            int batch, int k_x, int k_h, float gamma,
+                            const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                            float *y, const dip_step_outputs *out, void *stream)
 {
-    if (!ctx || !weights_ok(w) || !x || !y || !dip_aligned16(x) || !dip_aligned16(y)) return DIP_ERR_INVALID_ARG;
+    const float *x = xb ? x_norm : xa;
+    if (!ctx || !weights_ok(w) || !xa || !x || !y || !dip_aligned16(xa) || !dip_aligned16(x) || !dip_aligned16(y))
+        return DIP_ERR_INVALID_ARG;
     if (batch < 1 || batch > DIP_MAX_BATCH) return DIP_ERR_INVALID_ARG;
     if (k_x < 1 || k_x > w->d_model || k_h < 1 || k_h > w->d_ff) return DIP_ERR_INVALID_ARG;
     if (!(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
@@ -213,9 +220,14 @@ dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
     dip_status st;
 
     // m_x = topK(score(x))            (Eq. 7; Algorithm 1 when a cache is given)
-    st = dip_launch_mask(ctx, x, batch, w->d_model, k_x, gamma,
-                         cache_gu ? cache_gu->stamp : nullptr, cache_gu ? cache_gu->meta : nullptr,
-                         cache_gu ? cache_gu->capacity : 0, mask_x, idx_x, s);
+    if (xb)
+        st = dip_launch_norm_mask(ctx, xa, xb, x_norm, batch, w->d_model, k_x, gamma,
+                                  cache_gu ? cache_gu->stamp : nullptr, cache_gu ? cache_gu->meta : nullptr,
+                                  cache_gu ? cache_gu->capacity : 0, mask_x, idx_x, s);
+    else
+        st = dip_launch_mask(ctx, x, batch, w->d_model, k_x, gamma,
+                             cache_gu ? cache_gu->stamp : nullptr, cache_gu ? cache_gu->meta : nullptr,
+                             cache_gu ? cache_gu->capacity : 0, mask_x, idx_x, s);
     if (st != DIP_OK) return st;
     // h = (W~u x) * silu(W~g x)       (Eq. 2 inside Eq. 3)
     if (batch == 1) {
@@ -249,6 +261,14 @@ dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
     return st;
 }
 
+dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
+                        const float *x, int batch, int k_x, int k_h, float gamma,
+                        const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                        float *y, const dip_step_outputs *out, void *stream)
+{
+    return step_impl(ctx, w, x, nullptr, nullptr, batch, k_x, k_h, gamma, cache_gu, cache_d, y, out, stream);
+}
+
 dip_status dip_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y,
                                 int batch, int d, float *x_next, void *stream)
 {
@@ -269,19 +289,21 @@ dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *lay
         if (layers[l].d_model != layers[0].d_model || layers[l].d_ff != layers[0].d_ff) return DIP_ERR_INVALID_ARG;
     }
     const int d = layers[0].d_model;
-    const float *cur = x_in;
+    // x_0 = x_in; for l > 0 the chaining x_l = rmsnorm(x_{l-1} + y_{l-1}) runs inside layer l's
+    // first mask launch.  x and y ping-pong between two workspace buffers each.
+    const float *x_prev = x_in;
+    const float *y_prev = nullptr;
     for (int l = 0; l < n_layers; ++l) {
-        float *y = (l == n_layers - 1 && y_last) ? y_last : ctx->y;
-        dip_status st = dip_mlp_step(ctx, &layers[l], cur, batch, k_x, k_h, gamma,
-                                     cache_gu ? &cache_gu[l] : nullptr, cache_d ? &cache_d[l] : nullptr,
-                                     y, nullptr, stream);
+        float *y = (l == n_layers - 1 && y_last) ? y_last : ((l & 1) ? ctx->y2 : ctx->y);
+        float *x_l = (l & 1) ? ctx->xb : ctx->xa;
+        dip_status st = step_impl(ctx, &layers[l], x_prev, y_prev, y_prev ? x_l : nullptr, batch, k_x, k_h, gamma,
+                                  cache_gu ? &cache_gu[l] : nullptr, cache_d ? &cache_d[l] : nullptr,
+                                  y, nullptr, stream);
         if (st != DIP_OK) return st;
-        float *next = l == n_layers - 1 ? x_out : ((l & 1) ? ctx->xb : ctx->xa);
-        st = dip_residual_rmsnorm(ctx, cur, y, batch, d, next, stream);
-        if (st != DIP_OK) return st;
-        cur = next;
+        if (y_prev) x_prev = x_l;
+        y_prev = y;
     }
-    return DIP_OK;
+    return dip_residual_rmsnorm(ctx, x_prev, y_prev, batch, d, x_out, stream);
 }
 
 }  // extern "C"

@@ -19,7 +19,8 @@ struct dip_ctx {
     int n_tickets;
     // intermediates of dip_mlp_step when the caller does not ask for them
     float *h;            // [DIP_MAX_BATCH][DIP_MAX_D]
-    float *y;            // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner)
+    float *y;            // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner, even layers)
+    float *y2;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner, odd layers)
     float *xa;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner ping)
     float *xb;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner pong)
     uint32_t *mask;      // [DIP_MAX_BATCH][DIP_MAX_D/32]  masks of x
@@ -49,6 +50,11 @@ static inline bool dip_aligned16(const void *p) { return (((uintptr_t)p) & 15u) 
 dip_status dip_launch_mask(dip_ctx *ctx, const float *x, int batch, int d, int k, float gamma,
                            int32_t *stamp, int32_t *meta, int capacity,
                            uint32_t *mask_bits, int32_t *kept_idx, cudaStream_t stream);
+
+// topk.cu: x_out = (xa + xb) / rms(xa + xb) followed by the mask of x_out, in one launch.
+dip_status dip_launch_norm_mask(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d,
+                                int k, float gamma, int32_t *stamp, int32_t *meta, int capacity,
+                                uint32_t *mask_bits, int32_t *kept_idx, cudaStream_t stream);
 
 // topk.cu: per-device set-up of the mask kernels (dynamic shared memory limit).
 dip_status dip_init_mask_kernels(dip_ctx *ctx);

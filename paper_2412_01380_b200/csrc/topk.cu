@@ -3,7 +3,7 @@
 // decode, and the residual + RMS re-normalisation that chains layers.
 //
 // One CTA of 1024 threads handles one input row.  The row's rank keys live in shared memory;
-// the k-th largest key is found by an 8-bit-per-pass radix select, then one ordered sweep
+// the k-th largest key is found by an 11-bit-per-pass radix select, then one ordered sweep
 // (warp ballots over 32 consecutive columns = one mask word) emits the bit mask and the
 // ascending index list.  Everything here is integer work on bit patterns, so results are
 // exact and unique (ties go to the lower column index).
@@ -13,13 +13,17 @@ namespace {
 
 constexpr int TK_THREADS = 1024;
 constexpr int TK_WARPS = TK_THREADS / 32;
+constexpr int RADIX_BITS = 11;
+constexpr int RADIX_BINS = 1 << RADIX_BITS;   // two bins per thread
 
 struct TkShared {
-    unsigned int hist[256];
+    unsigned int hist[RADIX_BINS];
     int bcast[4];
     int wa[TK_WARPS];   // per-warp counts for ordered prefix sums
     int wb[TK_WARPS];
     int wc[TK_WARPS];
+    float wf[TK_WARPS];
+    float scale;
 };
 
 __device__ __forceinline__ unsigned lanemask_lt()
@@ -44,60 +48,87 @@ __device__ __forceinline__ int warp_array_prefix(const int *arr, int warp, int l
     return __shfl_sync(0xffffffffu, excl, warp);
 }
 
-// k-th largest of keys[0..d) (31-bit patterns).  All threads of the CTA take part and get the
-// same answer: keep every key > T and the first `quota` columns (by index) with key == T.
-// Requires 1 <= k <= d.  A caller that wants to exclude a column gives it key 0 and makes
-// sure k does not reach the zeros.
-__device__ void block_radix_select(const uint32_t *keys, int d, int k, TkShared &s, uint32_t &T, int &quota)
+// k-th largest of (keys[e] & keymask), e in [0, d).  All threads of the CTA take part and get
+// the same answer: keep every key > T and the first `quota` columns (by index) with key == T.
+// Requires 1 <= k <= d and every masked key < 2^top_bit.  A caller that wants to exclude a
+// column gives it key 0 and makes sure k does not reach the zeros.
+//
+// Radix select from the top bit down, up to 11 bits per pass: a shared-memory histogram of the
+// current digit over the keys that match the prefix found so far, then a suffix scan over the
+// bins (two per thread) to find the bin holding the k-th key.  The four smallest digits, which
+// are by far the most frequent ones when the keys are ages of cache lines, are counted in
+// registers instead of with contended atomics.
+__device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask, int top_bit, int k,
+                                   TkShared &s, uint32_t &T, int &quota)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t prefix = 0, prefmask = 0;
     int krem = k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        if (tid < 256) s.hist[tid] = 0;
+    int hi = top_bit;
+    while (hi > 0) {
+        const int w = hi < RADIX_BITS ? hi : RADIX_BITS;
+        const int shift = hi - w;
+        const uint32_t dmask = (1u << w) - 1u;
+        s.hist[2 * tid] = 0;
+        s.hist[2 * tid + 1] = 0;
         __syncthreads();
-        for (int e0 = warp * 32; e0 < d; e0 += TK_THREADS) {
-            int e = e0 + lane;
-            uint32_t digit = 0xffffffffu;
-            if (e < d) {
-                uint32_t key = keys[e];
-                if ((key & prefmask) == prefix) digit = (key >> shift) & 255u;
+        int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+        for (int e = tid; e < d; e += TK_THREADS) {
+            const uint32_t key = keys[e] & keymask;
+            if ((key & prefmask) == prefix) {
+                const uint32_t dg = (key >> shift) & dmask;
+                if (dg >= 4u) atomicAdd(&s.hist[dg], 1u);
+                c0 += dg == 0u;
+                c1 += dg == 1u;
+                c2 += dg == 2u;
+                c3 += dg == 3u;
             }
-            // lanes with the same digit add once
-            unsigned peers = __match_any_sync(0xffffffffu, digit);
-            if (digit != 0xffffffffu && (peers & lanemask_lt()) == 0)
-                atomicAdd(&s.hist[digit], (unsigned)__popc(peers));
+        }
+        c0 = __reduce_add_sync(0xffffffffu, c0);
+        c1 = __reduce_add_sync(0xffffffffu, c1);
+        c2 = __reduce_add_sync(0xffffffffu, c2);
+        c3 = __reduce_add_sync(0xffffffffu, c3);
+        if (lane == 0) {
+            if (c0) atomicAdd(&s.hist[0], (unsigned)c0);
+            if (c1) atomicAdd(&s.hist[1], (unsigned)c1);
+            if (c2) atomicAdd(&s.hist[2], (unsigned)c2);
+            if (c3) atomicAdd(&s.hist[3], (unsigned)c3);
         }
         __syncthreads();
-        if (warp == 0) {
-            unsigned c[8];
-            unsigned sum = 0;
+        // suffix scan: thread t owns bins 2t and 2t+1
+        const unsigned h0 = s.hist[2 * tid], h1 = s.hist[2 * tid + 1];
+        const int own = (int)(h0 + h1);
+        int suf = own;   // inclusive suffix within the warp
 #pragma unroll
-            for (int b = 0; b < 8; ++b) {
-                c[b] = s.hist[lane * 8 + b];
-                sum += c[b];
-            }
-            // number of matching keys in the bins above this lane's 8 bins
-            unsigned incl = sum;
+        for (int o = 1; o < 32; o <<= 1) {
+            int n = __shfl_down_sync(0xffffffffu, suf, o);
+            if (lane + o < 32) suf += n;
+        }
+        if (lane == 0) s.wa[warp] = suf;
+        __syncthreads();
+        int wv = s.wa[lane];
+        int wsuf = wv;   // inclusive suffix over warps
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                unsigned n = __shfl_down_sync(0xffffffffu, incl, o);
-                if (lane + o < 32) incl += n;
-            }
-            unsigned cum = incl - sum;
-#pragma unroll
-            for (int b = 7; b >= 0; --b) {
-                if (cum < (unsigned)krem && (unsigned)krem <= cum + c[b]) {
-                    s.bcast[0] = lane * 8 + b;
-                    s.bcast[1] = krem - (int)cum;
-                }
-                cum += c[b];
-            }
+        for (int o = 1; o < 32; o <<= 1) {
+            int n = __shfl_down_sync(0xffffffffu, wsuf, o);
+            if (lane + o < 32) wsuf += n;
+        }
+        const int above_warp = __shfl_sync(0xffffffffu, wsuf - wv, warp);
+        int cum = above_warp + suf - own;             // keys in bins above 2t+1
+        if (cum < krem && krem <= cum + (int)h1) {
+            s.bcast[0] = 2 * tid + 1;
+            s.bcast[1] = krem - cum;
+        }
+        cum += (int)h1;
+        if (cum < krem && krem <= cum + (int)h0) {
+            s.bcast[0] = 2 * tid;
+            s.bcast[1] = krem - cum;
         }
         __syncthreads();
         prefix |= (uint32_t)s.bcast[0] << shift;
-        prefmask |= 255u << shift;
+        prefmask |= dmask << shift;
         krem = s.bcast[1];
+        hi = shift;
     }
     T = prefix;
     quota = krem;
@@ -108,12 +139,15 @@ __device__ void block_radix_select(const uint32_t *keys, int d, int k, TkShared 
 //   CA == false: key = bits(|x|)                              (DIP, Eq. 7-8)
 //   CA == true : key = bits(|x| * (resident ? 1 : gamma))     (numerator of Eq. 10), then the
 //                LRU cache update c' = cache_update(c, m).
+//   NORM == true: the row is first formed as x = (xa + xb) / rms(xa + xb) (the layer chaining
+//                of a stack) and written to x_out; the summation order is that of
+//                residual_rmsnorm_kernel, so both give the same bits.
 // keys[] is dynamic shared memory: d words.
 // ---------------------------------------------------------------------------------------
-template <bool CA>
+template <bool CA, bool NORM>
 __global__ void __launch_bounds__(TK_THREADS, 1)
-mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
-            int32_t *stamp, int32_t *meta, int capacity,
+mask_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *__restrict__ x_out,
+            int d, int k, float gamma, int32_t *stamp, int32_t *meta, int capacity,
             uint32_t *__restrict__ mask_bits, int32_t *__restrict__ kept_idx)
 {
     extern __shared__ uint32_t keys[];
@@ -122,23 +156,59 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x;
     const int n_words = (d + 31) >> 5;
-    x += (size_t)row * d;
+    xa += (size_t)row * d;
+    if (NORM) {
+        xb += (size_t)row * d;
+        x_out += (size_t)row * d;
+    }
     if (mask_bits) mask_bits += (size_t)row * n_words;
     if (kept_idx) kept_idx += (size_t)row * k;
 
-    for (int e = tid; e < d; e += TK_THREADS) {
-        float a = fabsf(x[e]);
-        if (CA) {
-            float w = stamp[e] >= 0 ? 1.0f : gamma;
-            a = __fmul_rn(a, w);
+    int n_res = 0, t_now = 0;
+    if (CA) {
+        n_res = meta[0];
+        t_now = meta[1] + 1;
+    }
+
+    if (NORM) {
+        float ss = 0.f;
+        for (int e = tid; e < d; e += TK_THREADS) {
+            float r = xa[e] + xb[e];
+            keys[e] = __float_as_uint(r);
+            ss = fmaf(r, r, ss);
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) s.wf[warp] = ss;
+        __syncthreads();
+        if (warp == 0) {
+            float v = s.wf[lane];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == 0) {
+                float rms = sqrtf(v / (float)d);
+                s.scale = rms > 0.f ? 1.0f / rms : 1.0f;
+            }
+        }
+        __syncthreads();
+    }
+    for (int e = tid; e < d; e += TK_THREADS) {
+        float v;
+        if (NORM) {
+            v = __uint_as_float(keys[e]) * s.scale;
+            x_out[e] = v;
+        } else {
+            v = xa[e];
+        }
+        float a = fabsf(v);
+        if (CA) a = __fmul_rn(a, stamp[e] >= 0 ? 1.0f : gamma);
         keys[e] = __float_as_uint(a) & 0x7fffffffu;
     }
     __syncthreads();
 
     uint32_t T;
     int quota;
-    block_radix_select(keys, d, k, s, T, quota);
+    block_radix_select(keys, d, 0x7fffffffu, 31, k, s, T, quota);
 
     // ordered sweeps: warp w owns columns [w*span, (w+1)*span), span a multiple of 32
     const int span = ((d + TK_THREADS - 1) / TK_THREADS) * 32;
@@ -163,8 +233,8 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
     int eq_before = warp_array_prefix(s.wb, warp, lane, tot);
     __syncthreads();   // wa/wb are reused below
 
-    // second sweep: emit the mask and the index list; for CA also turn keys[] into the
-    // eviction keys and count hits and misses
+    // second sweep: emit the mask and the index list; for CA also turn keys[] into
+    // (resident flag << 31) | eviction key and count hits and misses
     int hits = 0, misses = 0;
     for (int it = 0; it < span; it += 32) {
         int e = base + it + lane;
@@ -178,7 +248,7 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
         unsigned bk = __ballot_sync(0xffffffffu, keep);
         if (base + it < d) {
             if (lane == 0) {
-                s_mask[(base + it) >> 5] = bk;
+                if (CA) s_mask[(base + it) >> 5] = bk;
                 if (mask_bits) mask_bits[(base + it) >> 5] = bk;
             }
             if (kept_idx && keep) {
@@ -189,9 +259,9 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
         if (CA) {
             int st = valid ? stamp[e] : -1;
             bool res = st >= 0;
-            // eviction key: an older stamp gives a larger key; columns that cannot be
-            // evicted (not resident, or in the current mask) get 0
-            if (valid) keys[e] = (res && !keep) ? (0x7fffffffu - (uint32_t)st) : 0u;
+            // eviction key = age of the last use: an older column has a larger key; columns
+            // that cannot be evicted (not resident, or in the current mask) get 0
+            if (valid) keys[e] = (res ? 0x80000000u : 0u) | ((res && !keep) ? (uint32_t)(t_now - st) : 0u);
             hits += __popc(__ballot_sync(0xffffffffu, keep && res));
             misses += __popc(__ballot_sync(0xffffffffu, keep && !res));
         }
@@ -209,13 +279,11 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
     int total_hits, total_misses;
     (void)warp_array_prefix(s.wa, warp, lane, total_hits);
     int miss_before = warp_array_prefix(s.wc, warp, lane, total_misses);
-    const int n_res = meta[0];
-    const int t = meta[1] + 1;
     const int free_slots = capacity - n_res;
     const int evictable = n_res - total_hits;
     const int n_evict = min(max(0, total_misses - free_slots), evictable);
     const int room = free_slots + n_evict;
-    __syncthreads();   // everyone has read meta[] and the warp arrays
+    __syncthreads();   // the warp arrays are reused by the select
 
     // victims: the n_evict largest eviction keys (oldest stamps), lower index first among equals
     uint32_t T2 = 0x7fffffffu;   // no key exceeds it: no victim
@@ -224,7 +292,7 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
         if (n_evict == evictable)
             T2 = 0u;             // every evictable column (key > 0) goes
         else
-            block_radix_select(keys, d, n_evict, s, T2, quota2);
+            block_radix_select(keys, d, 0x7fffffffu, 32 - __clz(t_now), n_evict, s, T2, quota2);
     }
 
     // ordered rank of the eviction-key ties
@@ -233,7 +301,7 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
         int veq = 0;
         for (int it = 0; it < span; it += 32) {
             int e = base + it + lane;
-            veq += __popc(__ballot_sync(0xffffffffu, e < d && keys[e] == T2));
+            veq += __popc(__ballot_sync(0xffffffffu, e < d && (keys[e] & 0x7fffffffu) == T2));
         }
         if (lane == 0) s.wb[warp] = veq;
         __syncthreads();
@@ -243,19 +311,21 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
     for (int it = 0; it < span; it += 32) {
         int e = base + it + lane;
         bool valid = e < d;
-        uint32_t vkey = valid ? keys[e] : 0u;
+        uint32_t kv = valid ? keys[e] : 0u;
+        uint32_t vkey = kv & 0x7fffffffu;
+        bool res = (kv >> 31) != 0u;
         bool keep = valid && ((s_mask[e >> 5] >> lane) & 1u);
         bool vq = valid && quota2 > 0 && vkey == T2;
         unsigned bvq = __ballot_sync(0xffffffffu, vq);
         bool evict = valid && (vkey > T2 || (vq && (veq_before + __popc(bvq & lt)) < quota2));
-        bool miss = keep && stamp[e] < 0;
+        bool miss = keep && !res;
         unsigned bm = __ballot_sync(0xffffffffu, miss);
         if (valid) {
             if (evict) {
                 stamp[e] = -1;
             } else if (keep) {
                 // a hit, or a miss that still finds room (ascending index order)
-                if (!miss || (miss_before + __popc(bm & lt)) < room) stamp[e] = t;
+                if (!miss || (miss_before + __popc(bm & lt)) < room) stamp[e] = t_now;
             }
         }
         veq_before += __popc(bvq);
@@ -264,7 +334,7 @@ mask_kernel(const float *__restrict__ x, int d, int k, float gamma,
     if (tid == 0) {
         const int inserted = min(total_misses, room);
         meta[0] = n_res - n_evict + inserted;
-        meta[1] = t;
+        meta[1] = t_now;
         meta[2] += total_hits;
         meta[3] += total_misses;
         meta[4] += n_evict;
@@ -350,11 +420,28 @@ dip_status dip_launch_mask(dip_ctx *ctx, const float *x, int batch, int d, int k
 {
     const size_t smem = (size_t)d * sizeof(uint32_t);
     if (stamp)
-        mask_kernel<true><<<batch, TK_THREADS, smem, stream>>>(x, d, k, gamma, stamp, meta, capacity,
-                                                               mask_bits, kept_idx);
+        mask_kernel<true, false><<<batch, TK_THREADS, smem, stream>>>(x, nullptr, nullptr, d, k, gamma, stamp, meta,
+                                                                      capacity, mask_bits, kept_idx);
     else
-        mask_kernel<false><<<batch, TK_THREADS, smem, stream>>>(x, d, k, 1.0f, nullptr, nullptr, 0,
-                                                                mask_bits, kept_idx);
+        mask_kernel<false, false><<<batch, TK_THREADS, smem, stream>>>(x, nullptr, nullptr, d, k, 1.0f, nullptr,
+                                                                       nullptr, 0, mask_bits, kept_idx);
+    DIP_CUDA_TRY(ctx, cudaGetLastError());
+    return DIP_OK;
+}
+
+// x_out = (xa + xb) / rms(xa + xb), then the mask of x_out: one launch for the layer chaining
+// and the first mask of the next layer.
+dip_status dip_launch_norm_mask(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d,
+                                int k, float gamma, int32_t *stamp, int32_t *meta, int capacity,
+                                uint32_t *mask_bits, int32_t *kept_idx, cudaStream_t stream)
+{
+    const size_t smem = (size_t)d * sizeof(uint32_t);
+    if (stamp)
+        mask_kernel<true, true><<<batch, TK_THREADS, smem, stream>>>(xa, xb, x_out, d, k, gamma, stamp, meta,
+                                                                     capacity, mask_bits, kept_idx);
+    else
+        mask_kernel<false, true><<<batch, TK_THREADS, smem, stream>>>(xa, xb, x_out, d, k, 1.0f, nullptr, nullptr,
+                                                                      0, mask_bits, kept_idx);
     DIP_CUDA_TRY(ctx, cudaGetLastError());
     return DIP_OK;
 }
@@ -363,8 +450,10 @@ dip_status dip_launch_mask(dip_ctx *ctx, const float *x, int batch, int d, int k
 dip_status dip_init_mask_kernels(dip_ctx *ctx)
 {
     const int bytes = DIP_MAX_D * (int)sizeof(uint32_t);
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     return DIP_OK;
 }
 
