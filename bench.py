@@ -256,7 +256,7 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
         h = torch.empty(d_ff, device="cuda")
         y = torch.empty(d_model, device="cuda")
         n_pass_tok = 6
-        names = ["mask_x", "gate_up", "mask_h", "down", "rmsnorm"]
+        names = ["mask_x", "gate_up", "mask_h", "down", "rmsnorm"]   # mask_* = select (+ cache update when on)
         evs = []
         for t in range(n_pass_tok):
             cur = xs_dev[t % n_tok].clone()
@@ -264,18 +264,18 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
                 ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
                 ev[0].record(stream)
                 if ca:
-                    dip.dip_ca_mask(ctx, cur, k_x, gamma, st2.cache_gu[l], mask_x, idx_x)
+                    dip.dip_ca_mask(ctx, cur, k_x, gamma, st2.cache_gu[l], mask_x, None)
                 else:
-                    dip.dip_mask_topk(ctx, cur, k_x, mask_x, idx_x)
+                    dip.dip_mask_topk(ctx, cur, k_x, mask_x, None)
                 ev[1].record(stream)
-                dip.dip_sparse_gemv_gate_up(ctx, layers[l], cur, idx_x, k_x, None, h)
+                dip.dip_sparse_gemv_gate_up(ctx, layers[l], cur, None, k_x, mask_x, h)
                 ev[2].record(stream)
                 if ca:
-                    dip.dip_ca_mask(ctx, h, k_h, gamma, st2.cache_d[l], mask_h, idx_h)
+                    dip.dip_ca_mask(ctx, h, k_h, gamma, st2.cache_d[l], mask_h, None)
                 else:
-                    dip.dip_mask_topk(ctx, h, k_h, mask_h, idx_h)
+                    dip.dip_mask_topk(ctx, h, k_h, mask_h, None)
                 ev[3].record(stream)
-                dip.dip_sparse_gemv_down(ctx, layers[l], h, idx_h, k_h, None, y)
+                dip.dip_sparse_gemv_down(ctx, layers[l], h, None, k_h, mask_h, y)
                 ev[4].record(stream)
                 dip.dip_residual_rmsnorm(ctx, cur, y, cur)
                 ev[5].record(stream)
@@ -391,7 +391,7 @@ def main():
     gu_bytes = head["bytes"]["gate_up"]
     gu_us = head["kernels"]["gate_up_us"]
     achieved = gu_bytes / (gu_us * 1e-6) / 1e9
-    launches_per_step = L * 5
+    launches_per_step = L * (4 + (2 if budget is not None else 0)) + 1
     line = {
         "metric": METRIC, "value": head["mlp_steps_per_s"] * world, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["ms_per_step"],

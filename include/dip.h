@@ -22,7 +22,9 @@
  *    the end of the enqueued work.
  *  - Calls on the same context must not overlap on the GPU (they share the
  *    context's scratch workspace): use one context per concurrently running
- *    stream.
+ *    stream.  With a column cache the state update of Algorithm 1 runs on a
+ *    stream of the context's own, beside the products that do not depend on
+ *    it, and is joined back into `stream` before the call's work ends.
  *  - Arguments are validated on the host before anything is launched; a failed
  *    validation returns an error code and launches nothing.
  *  - Data pointers must be 16-byte aligned.
@@ -79,6 +81,11 @@ const char *dip_status_string(dip_status s);
 const char *dip_last_error(const dip_ctx *ctx);
 /* Number of streaming multiprocessors of the context's device. */
 int dip_sm_count(const dip_ctx *ctx);
+/* Every wait inside a kernel (on the arrival of an asynchronous copy) is bounded.  If one runs
+ * out, the kernel stops early, its outputs are invalid and a sticky status word on the device
+ * becomes non-zero.  This call waits for `stream`, then copies the word to *status_out (host):
+ * 0 = no kernel of this context has given up a wait. */
+dip_status dip_device_status(dip_ctx *ctx, int *status_out, void *stream);
 
 /* ------------------------------------------------------------------------
  * Weights.  The paper's unit of selection is a column W[:, i] of a matrix
@@ -188,8 +195,11 @@ dip_status dip_ca_mask(dip_ctx *ctx, const float *x, int d, int k, float gamma,
  *   x        [batch][d_model]
  *   kept_idx [n_kept] ascending columns to read.  batch == 1: the token's mask.
  *            batch > 1: the union of the tokens' masks, each row read once.
- *   mask_bits batch > 1 only: [batch][ceil(d_model/32)] per-token masks; token
- *            b uses column i only if its bit is set.  NULL for batch == 1.
+ *   mask_bits [batch][ceil(d_model/32)] per-token masks; token b uses column i
+ *            only if its bit is set.  Required for batch > 1, where the rows read
+ *            are the union of the masks.  For batch == 1 it may be NULL (the list
+ *            is used), or given with kept_idx == NULL (the bit set is used and
+ *            n_kept is an upper bound on its size).
  *   h        [batch][d_ff] out
  * 1 <= n_kept <= d_model.
  * ------------------------------------------------------------------------ */

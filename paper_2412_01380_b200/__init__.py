@@ -52,6 +52,8 @@ _lib.dip_last_error.restype = C.c_char_p
 _lib.dip_last_error.argtypes = [_vp]
 _lib.dip_sm_count.restype = _i32
 _lib.dip_sm_count.argtypes = [_vp]
+_lib.dip_device_status.restype = _i32
+_lib.dip_device_status.argtypes = [_vp, C.POINTER(C.c_int), _vp]
 _lib.dip_packed_bytes.restype = C.c_size_t
 _lib.dip_packed_bytes.argtypes = [_i32, _i32, _i32, _i32]
 _lib.dip_pack_weights.restype = _i32
@@ -78,6 +80,7 @@ _lib.dip_sparse_gemv_down_noalloc.restype = _i32
 _lib.dip_sparse_gemv_down_noalloc.argtypes = [C.POINTER(MlpWeightsStruct), _vp, _vp, _i32, _vp, _vp]
 
 EXPORTED = ["dip_create", "dip_destroy", "dip_status_string", "dip_last_error", "dip_sm_count",
+            "dip_device_status",
             "dip_packed_bytes", "dip_pack_weights", "dip_mask_topk", "dip_ca_mask",
             "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_mlp_step",
             "dip_residual_rmsnorm", "dip_stack_step", "dip_sparse_gemv_down_noalloc"]
@@ -118,6 +121,12 @@ class Context:
     @property
     def sm_count(self) -> int:
         return _lib.dip_sm_count(self.handle)
+
+    def device_status(self) -> int:
+        """Waits for the current stream; 0 unless a kernel gave up a bounded wait."""
+        out = C.c_int(-1)
+        self.check(_lib.dip_device_status(self.handle, C.byref(out), _stream()))
+        return out.value
 
     def close(self) -> None:
         if self.handle:

@@ -95,6 +95,15 @@ dip_status dip_create(dip_ctx **out, int device)
     if ((st = dev_alloc(ctx, &ctx->idx_h, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->union_idx, (size_t)DIP_MAX_D)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->counts, (size_t)8)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->mask_ring, (size_t)2 * DIP_RING_LAYERS * (DIP_MAX_D / 32))) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->mask_tmp, (size_t)(DIP_MAX_D / 32))) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->status, (size_t)1)) != DIP_OK) return fail(st);
+    if (cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
+    for (int i = 0; i < 2; ++i) {
+        if (cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking) != cudaSuccess) return fail(DIP_ERR_CUDA);
+        if (cudaEventCreateWithFlags(&ctx->ev_fork[i], cudaEventDisableTiming) != cudaSuccess) return fail(DIP_ERR_CUDA);
+        if (cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming) != cudaSuccess) return fail(DIP_ERR_CUDA);
+    }
     if (cudaMemset(ctx->tickets, 0, N_TICKETS * sizeof(unsigned int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if (cudaMemset(ctx->counts, 0, 8 * sizeof(int32_t)) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if ((st = dip_init_mask_kernels(ctx)) != DIP_OK) return fail(st);
@@ -118,6 +127,14 @@ dip_status dip_destroy(dip_ctx *ctx)
     cudaFree(ctx->idx_h);
     cudaFree(ctx->union_idx);
     cudaFree(ctx->counts);
+    cudaFree(ctx->mask_ring);
+    cudaFree(ctx->mask_tmp);
+    cudaFree(ctx->status);
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->side[i]) cudaStreamDestroy(ctx->side[i]);
+        if (ctx->ev_fork[i]) cudaEventDestroy(ctx->ev_fork[i]);
+        if (ctx->ev_join[i]) cudaEventDestroy(ctx->ev_join[i]);
+    }
     delete ctx;
     return DIP_OK;
 }
@@ -145,13 +162,47 @@ dip_status dip_pack_weights(dip_ctx *ctx, int wtype, int d_model, int d_ff,
     return dip_launch_pack(ctx, wtype, d_model, d_ff, Wg, Wu, Wd, Sg, Su, Sd, out, (cudaStream_t)stream);
 }
 
+dip_status dip_device_status(dip_ctx *ctx, int *status_out, void *stream)
+{
+    if (!ctx || !status_out) return DIP_ERR_INVALID_ARG;
+    DIP_CUDA_TRY(ctx, cudaMemcpyAsync(status_out, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    DIP_CUDA_TRY(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+    return DIP_OK;
+}
+
+// Run the cache update of one masked input beside the main stream (side stream `which`).
+static dip_status fork_cache_update(dip_ctx *ctx, int which, const uint32_t *mask_bits, const dip_cache_state *c,
+                                    cudaStream_t main)
+{
+    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork[which], main));
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side[which], ctx->ev_fork[which], 0));
+    dip_status st = dip_launch_cache_update(ctx, mask_bits, c->d, c->stamp, c->meta, c->capacity, ctx->side[which]);
+    ctx->side_busy[which] = true;
+    return st;
+}
+
+// Make the main stream wait for the side streams' updates.
+static dip_status join_cache_updates(dip_ctx *ctx, cudaStream_t main)
+{
+    for (int i = 0; i < 2; ++i) {
+        if (!ctx->side_busy[i]) continue;
+        DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join[i], ctx->side[i]));
+        DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(main, ctx->ev_join[i], 0));
+        ctx->side_busy[i] = false;
+    }
+    return DIP_OK;
+}
+
 dip_status dip_mask_topk(dip_ctx *ctx, const float *x, int batch, int d, int k,
                          uint32_t *mask_bits, int32_t *kept_idx, void *stream)
 {
     if (!ctx || !x || !dip_aligned16(x)) return DIP_ERR_INVALID_ARG;
     if (batch < 1 || batch > DIP_MAX_BATCH || d < 1 || d > DIP_MAX_D || k < 1 || k > d) return DIP_ERR_INVALID_ARG;
-    return dip_launch_mask(ctx, x, batch, d, k, 1.0f, nullptr, nullptr, 0, mask_bits, kept_idx,
-                           (cudaStream_t)stream);
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t *m = mask_bits ? mask_bits : ctx->mask;
+    dip_status st = dip_launch_select(ctx, x, nullptr, nullptr, batch, d, k, 1.0f, nullptr, m, s);
+    if (st == DIP_OK && kept_idx) st = dip_launch_mask_to_idx(ctx, m, batch, 1, d, kept_idx, k, nullptr, s);
+    return st;
 }
 
 dip_status dip_ca_mask(dip_ctx *ctx, const float *x, int d, int k, float gamma,
@@ -162,21 +213,32 @@ dip_status dip_ca_mask(dip_ctx *ctx, const float *x, int d, int k, float gamma,
     if (d < 1 || d > DIP_MAX_D || k < 1 || k > d) return DIP_ERR_INVALID_ARG;
     if (!(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
     if (!cache_ok(st, d)) return DIP_ERR_INVALID_ARG;
-    return dip_launch_mask(ctx, x, 1, d, k, gamma, st->stamp, st->meta, st->capacity, mask_bits, kept_idx,
-                           (cudaStream_t)stream);
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t *m = mask_bits ? mask_bits : ctx->mask;
+    dip_status rc = dip_launch_select(ctx, x, nullptr, nullptr, 1, d, k, gamma, st->stamp, m, s);
+    if (rc == DIP_OK) rc = dip_launch_cache_update(ctx, m, d, st->stamp, st->meta, st->capacity, s);
+    if (rc == DIP_OK && kept_idx) rc = dip_launch_mask_to_idx(ctx, m, 1, 1, d, kept_idx, k, nullptr, s);
+    return rc;
 }
 
 static dip_status gemv_entry(dip_ctx *ctx, const dip_mlp_weights *w, int which, const float *v, int batch,
                              const int32_t *kept_idx, int n_kept, const uint32_t *mask_bits,
                              float *out, void *stream)
 {
-    if (!ctx || !weights_ok(w) || !v || !kept_idx || !out) return DIP_ERR_INVALID_ARG;
+    if (!ctx || !weights_ok(w) || !v || !out) return DIP_ERR_INVALID_ARG;
+    if (!kept_idx && !mask_bits) return DIP_ERR_INVALID_ARG;
     if (!dip_aligned16(v) || !dip_aligned16(out)) return DIP_ERR_INVALID_ARG;
     const int d_in = which == 0 ? w->d_model : w->d_ff;
     if (batch < 1 || batch > DIP_MAX_BATCH || n_kept < 1 || n_kept > d_in) return DIP_ERR_INVALID_ARG;
     if (batch > 1 && !mask_bits) return DIP_ERR_INVALID_ARG;
-    return dip_launch_gemv(ctx, w, which, v, batch, kept_idx, n_kept, nullptr,
-                           batch > 1 ? mask_bits : nullptr, out, (cudaStream_t)stream);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (batch == 1 && kept_idx) {
+        // the kernels take the kept columns as a bit set
+        dip_status st = dip_launch_idx_to_mask(ctx, kept_idx, n_kept, d_in, ctx->mask_tmp, s);
+        if (st != DIP_OK) return st;
+        mask_bits = ctx->mask_tmp;
+    }
+    return dip_launch_gemv(ctx, w, which, v, batch, mask_bits, n_kept, out, s);
 }
 
 dip_status dip_sparse_gemv_gate_up(dip_ctx *ctx, const dip_mlp_weights *w, const float *x, int batch,
@@ -195,11 +257,14 @@ dip_status dip_sparse_gemv_down(dip_ctx *ctx, const dip_mlp_weights *w, const fl
 
 // One sparse MLP step.  xb != nullptr: the step's input is formed first as
 // x = (xa + xb) / rms(xa + xb), written to x_norm, in the same launch as its mask.
+// slot_x / slot_h: where the masks go when the caller did not ask for them.  defer_join: leave
+// the cache updates running on the side streams (the caller joins them later).
 static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
                             const float *xa, const float *xb, float *x_norm,
                             int batch, int k_x, int k_h, float gamma,
                             const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
-                            float *y, const dip_step_outputs *out, void *stream)
+                            float *y, const dip_step_outputs *out,
+                            uint32_t *slot_x, uint32_t *slot_h, bool defer_join, void *stream)
 {
     const float *x = xb ? x_norm : xa;
     if (!ctx || !weights_ok(w) || !xa || !x || !y || !dip_aligned16(xa) || !dip_aligned16(x) || !dip_aligned16(y))
@@ -212,53 +277,41 @@ static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
     if (batch > 1 && (cache_gu || cache_d)) return DIP_ERR_UNSUPPORTED;   // Algorithm 1 is per token
 
     cudaStream_t s = (cudaStream_t)stream;
-    uint32_t *mask_x = out && out->mask_x ? out->mask_x : ctx->mask;
-    int32_t *idx_x = out && out->idx_x ? out->idx_x : ctx->idx;
+    uint32_t *mask_x = out && out->mask_x ? out->mask_x : slot_x;
     float *h = out && out->h ? out->h : ctx->h;
-    uint32_t *mask_h = out && out->mask_h ? out->mask_h : ctx->mask_h;
-    int32_t *idx_h = out && out->idx_h ? out->idx_h : ctx->idx_h;
+    uint32_t *mask_h = out && out->mask_h ? out->mask_h : slot_h;
+    const long long cap_x = (long long)batch * k_x, cap_h = (long long)batch * k_h;
+    const int nmax_x = cap_x < w->d_model ? (int)cap_x : w->d_model;
+    const int nmax_h = cap_h < w->d_ff ? (int)cap_h : w->d_ff;
     dip_status st;
 
-    // m_x = topK(score(x))            (Eq. 7; Algorithm 1 when a cache is given)
-    if (xb)
-        st = dip_launch_norm_mask(ctx, xa, xb, x_norm, batch, w->d_model, k_x, gamma,
-                                  cache_gu ? cache_gu->stamp : nullptr, cache_gu ? cache_gu->meta : nullptr,
-                                  cache_gu ? cache_gu->capacity : 0, mask_x, idx_x, s);
-    else
-        st = dip_launch_mask(ctx, x, batch, w->d_model, k_x, gamma,
-                             cache_gu ? cache_gu->stamp : nullptr, cache_gu ? cache_gu->meta : nullptr,
-                             cache_gu ? cache_gu->capacity : 0, mask_x, idx_x, s);
+    // m_x = topK(score(x))            (Eq. 7; the ranking of Algorithm 1 when a cache is given)
+    st = dip_launch_select(ctx, xa, xb, x_norm, batch, w->d_model, k_x, gamma,
+                           cache_gu ? cache_gu->stamp : nullptr, mask_x, s);
     if (st != DIP_OK) return st;
+    // c' = cache_update(c, m_x)       (Algorithm 1; beside the products, which do not need it)
+    if (cache_gu && (st = fork_cache_update(ctx, 0, mask_x, cache_gu, s)) != DIP_OK) return st;
     // h = (W~u x) * silu(W~g x)       (Eq. 2 inside Eq. 3)
-    if (batch == 1) {
-        st = dip_launch_gemv(ctx, w, 0, x, 1, idx_x, k_x, nullptr, nullptr, h, s);
-    } else {
-        st = dip_launch_union(ctx, mask_x, batch, w->d_model, ctx->union_idx, ctx->counts + 0, s);
-        if (st != DIP_OK) return st;
-        const long long cap = (long long)batch * k_x;
-        st = dip_launch_gemv(ctx, w, 0, x, batch, ctx->union_idx, cap < w->d_model ? (int)cap : w->d_model,
-                             ctx->counts + 0, mask_x, h, s);
-    }
+    st = dip_launch_gemv(ctx, w, 0, x, batch, mask_x, nmax_x, h, s);
     if (st != DIP_OK) return st;
     // m_h = topK(score(h))            (Eq. 8: the GLU of the already sparsified gate/up)
-    st = dip_launch_mask(ctx, h, batch, w->d_ff, k_h, gamma,
-                         cache_d ? cache_d->stamp : nullptr, cache_d ? cache_d->meta : nullptr,
-                         cache_d ? cache_d->capacity : 0, mask_h, idx_h, s);
+    st = dip_launch_select(ctx, h, nullptr, nullptr, batch, w->d_ff, k_h, gamma,
+                           cache_d ? cache_d->stamp : nullptr, mask_h, s);
     if (st != DIP_OK) return st;
+    if (cache_d && (st = fork_cache_update(ctx, 1, mask_h, cache_d, s)) != DIP_OK) return st;
     // y = W~d h                       (Eq. 1 inside Eq. 3)
-    if (batch == 1) {
-        st = dip_launch_gemv(ctx, w, 1, h, 1, idx_h, k_h, nullptr, nullptr, y, s);
-    } else {
-        st = dip_launch_union(ctx, mask_h, batch, w->d_ff, ctx->union_idx, ctx->counts + 1, s);
-        if (st != DIP_OK) return st;
-        const long long cap = (long long)batch * k_h;
-        st = dip_launch_gemv(ctx, w, 1, h, batch, ctx->union_idx, cap < w->d_ff ? (int)cap : w->d_ff,
-                             ctx->counts + 1, mask_h, y, s);
-        if (st == DIP_OK && out && out->union_counts)
-            DIP_CUDA_TRY(ctx, cudaMemcpyAsync(out->union_counts, ctx->counts, 2 * sizeof(int32_t),
-                                              cudaMemcpyDeviceToDevice, s));
+    st = dip_launch_gemv(ctx, w, 1, h, batch, mask_h, nmax_h, y, s);
+    if (st != DIP_OK) return st;
+
+    if (out && out->idx_x && (st = dip_launch_mask_to_idx(ctx, mask_x, batch, 1, w->d_model, out->idx_x, k_x, nullptr, s)) != DIP_OK)
+        return st;
+    if (out && out->idx_h && (st = dip_launch_mask_to_idx(ctx, mask_h, batch, 1, w->d_ff, out->idx_h, k_h, nullptr, s)) != DIP_OK)
+        return st;
+    if (out && out->union_counts && batch > 1) {
+        if ((st = dip_launch_mask_to_idx(ctx, mask_x, 1, batch, w->d_model, nullptr, 0, out->union_counts, s)) != DIP_OK) return st;
+        if ((st = dip_launch_mask_to_idx(ctx, mask_h, 1, batch, w->d_ff, nullptr, 0, out->union_counts + 1, s)) != DIP_OK) return st;
     }
-    return st;
+    return defer_join ? DIP_OK : join_cache_updates(ctx, s);
 }
 
 dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
@@ -266,7 +319,9 @@ dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
                         const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
                         float *y, const dip_step_outputs *out, void *stream)
 {
-    return step_impl(ctx, w, x, nullptr, nullptr, batch, k_x, k_h, gamma, cache_gu, cache_d, y, out, stream);
+    if (!ctx) return DIP_ERR_INVALID_ARG;
+    return step_impl(ctx, w, x, nullptr, nullptr, batch, k_x, k_h, gamma, cache_gu, cache_d, y, out,
+                     ctx->mask, ctx->mask_h, false, stream);
 }
 
 dip_status dip_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y,
@@ -293,17 +348,26 @@ dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *lay
     // first mask launch.  x and y ping-pong between two workspace buffers each.
     const float *x_prev = x_in;
     const float *y_prev = nullptr;
+    const bool ca = cache_gu || cache_d;
     for (int l = 0; l < n_layers; ++l) {
         float *y = (l == n_layers - 1 && y_last) ? y_last : ((l & 1) ? ctx->y2 : ctx->y);
         float *x_l = (l & 1) ? ctx->xb : ctx->xa;
+        // with caches each layer's masks get their own slot: the updates that read them run
+        // beside later layers
+        const int slot = ca ? l % DIP_RING_LAYERS : 0;
+        uint32_t *slot_x = batch == 1 ? ctx->mask_ring + (size_t)slot * (DIP_MAX_D / 32) : ctx->mask;
+        uint32_t *slot_h = batch == 1 ? ctx->mask_ring + (size_t)(DIP_RING_LAYERS + slot) * (DIP_MAX_D / 32) : ctx->mask_h;
         dip_status st = step_impl(ctx, &layers[l], x_prev, y_prev, y_prev ? x_l : nullptr, batch, k_x, k_h, gamma,
                                   cache_gu ? &cache_gu[l] : nullptr, cache_d ? &cache_d[l] : nullptr,
-                                  y, nullptr, stream);
+                                  y, nullptr, slot_x, slot_h, true, stream);
         if (st != DIP_OK) return st;
+        if (ca && slot == DIP_RING_LAYERS - 1 && (st = join_cache_updates(ctx, (cudaStream_t)stream)) != DIP_OK) return st;
         if (y_prev) x_prev = x_l;
         y_prev = y;
     }
-    return dip_residual_rmsnorm(ctx, x_prev, y_prev, batch, d, x_out, stream);
+    dip_status st = dip_residual_rmsnorm(ctx, x_prev, y_prev, batch, d, x_out, stream);
+    if (st != DIP_OK) return st;
+    return join_cache_updates(ctx, (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -29,8 +29,17 @@ struct dip_ctx {
     int32_t *idx_h;
     int32_t *union_idx;  // [DIP_MAX_D]
     int32_t *counts;     // [8] device scalars (union sizes)
+    uint32_t *mask_ring; // [2][DIP_RING_LAYERS][DIP_MAX_D/32] per-layer mask slots of the stack runner
+    uint32_t *mask_tmp;  // [DIP_MAX_D/32] list-based GEMV entry points
+    int *status;         // sticky device status word (0 = fine)
+    // the cache updates run beside the GEMVs: one side stream per cache kind
+    cudaStream_t side[2];
+    cudaEvent_t ev_fork[2], ev_join[2];
+    bool side_busy[2];
     char err[256];
 };
+
+constexpr int DIP_RING_LAYERS = 128;
 
 #define DIP_CUDA_TRY(ctx, call)                                                        \
     do {                                                                               \
@@ -46,35 +55,37 @@ static inline bool dip_aligned16(const void *p) { return (((uintptr_t)p) & 15u) 
 
 // ---- launchers implemented in the kernel files (host functions) -----------------
 
-// topk.cu: one CTA per row.  stamp == nullptr: plain |x| ranking, no cache.
-dip_status dip_launch_mask(dip_ctx *ctx, const float *x, int batch, int d, int k, float gamma,
-                           int32_t *stamp, int32_t *meta, int capacity,
-                           uint32_t *mask_bits, int32_t *kept_idx, cudaStream_t stream);
+// topk.cu: mask of each row: k largest rank keys (|x|, or |x| * (resident ? 1 : gamma) when stamp
+// is given).  xb != nullptr: the row is first formed as (xa + xb) / rms(xa + xb), written to x_out.
+dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d, int k,
+                             float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream);
 
-// topk.cu: x_out = (xa + xb) / rms(xa + xb) followed by the mask of x_out, in one launch.
-dip_status dip_launch_norm_mask(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d,
-                                int k, float gamma, int32_t *stamp, int32_t *meta, int capacity,
-                                uint32_t *mask_bits, int32_t *kept_idx, cudaStream_t stream);
+// topk.cu: LRU cache update from (mask, state).
+dip_status dip_launch_cache_update(dip_ctx *ctx, const uint32_t *mask_bits, int d, int32_t *stamp, int32_t *meta,
+                                   int capacity, cudaStream_t stream);
 
 // topk.cu: per-device set-up of the mask kernels (dynamic shared memory limit).
 dip_status dip_init_mask_kernels(dip_ctx *ctx);
 
-// topk.cu: union of `batch` bit masks -> ascending index list and its length (device scalar).
-dip_status dip_launch_union(dip_ctx *ctx, const uint32_t *mask_bits, int batch, int d,
-                            int32_t *union_idx, int32_t *union_count, cudaStream_t stream);
+// topk.cu: `rows` index lists, each from the OR of `nb` consecutive masks; lengths to count_out.
+dip_status dip_launch_mask_to_idx(dip_ctx *ctx, const uint32_t *mask_bits, int rows, int nb, int d,
+                                  int32_t *idx_out, int out_stride, int32_t *count_out, cudaStream_t stream);
 
 // topk.cu: x_next = (x + y) / rms(x + y) per row.
 dip_status dip_launch_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y, int batch, int d,
                                        float *x_next, cudaStream_t stream);
 
-// gemv.cu: gather GEMV over kept rows of a packed matrix.
+// gemv.cu: gather GEMV over the rows named by the mask bits (OR over the batch; token b uses a
+// row only if its own bit is set).
 //   which = 0: gate/up bundle with the silu*up epilogue, out = h[batch][d_ff]
 //   which = 1: down, out = y[batch][d_model]
-// n_kept_dev != nullptr: the row count is read on the device (at most n_kept_max).
+// n_kept_max bounds the number of rows (sizes the row parts).
 dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
-                           const float *v, int batch,
-                           const int32_t *kept_idx, int n_kept_max, const int32_t *n_kept_dev,
-                           const uint32_t *mask_bits, float *out, cudaStream_t stream);
+                           const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
+                           float *out, cudaStream_t stream);
+
+// gemv.cu: bit set from an ascending index list.
+dip_status dip_launch_idx_to_mask(dip_ctx *ctx, const int32_t *idx, int n, int d, uint32_t *mask, cudaStream_t stream);
 
 // pack.cu
 dip_status dip_launch_pack(dip_ctx *ctx, int wtype, int d_model, int d_ff,

@@ -1,200 +1,344 @@
 // Sparse vector-matrix products over the kept weight columns (Eq. 3 with the masks of Eq. 7-8).
 //
-// A packed matrix stores column i of W as row i (see dip.h), so a kept column is one
-// contiguous row.  The kernel is a gather-GEMV: grid = (output slabs) x (row parts).
-// A warp reads one kept row's slab segment per step, 32 bytes per lane (two 16-byte loads,
-// a full 1 KB contiguous piece per warp), and keeps E binary32 accumulators per lane and
-// token.  The warps of a CTA take different rows; their sums are combined through shared
-// memory in warp order, the row parts through a scratch buffer in part order by the last
-// CTA to arrive at the slab (an arrival counter).  The order of every sum is fixed, so the
-// result is bit-reproducible; no floating-point atomics are used.
+// A packed matrix stores column i of W as row i (see dip.h), so a kept column is one contiguous
+// row.  The kernel is a gather-GEMV: grid = (output slabs of 2 KB of row) x (row parts), sized to
+// one CTA per SM.  Each CTA
+//   1. reads the mask bits, prefix-sums their popcounts and extracts the kept rows whose rank
+//      falls in its part (so parts are balanced whatever the mask looks like);
+//   2. streams its rows' 2 KB slab segments from HBM into a ring of shared-memory stages with
+//      bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts), issued by one
+//      producer warp, so that ~160 KB per SM are in flight independent of register pressure;
+//   3. eight consumer warps (4 column groups x 2 row groups) multiply-accumulate from shared
+//      memory, 16 bytes of a row per lane, in binary32;
+//   4. the row groups are combined through shared memory, the parts through a scratch buffer in
+//      part order by the last CTA to arrive at the slab (an arrival counter).
+// The order of every sum is fixed, so results are bit-reproducible; no float atomics.
 //
-// which = 0 (gate/up bundle): a lane's 32 bytes are [gate chunk | up chunk] of the same
-// outputs, so the silu(gate) * up epilogue (Eq. 2) needs no data exchange.
-// which = 1 (down): plain sums.
+// which = 0 (gate/up bundle): the epilogue applies silu(gate) * up (Eq. 2).  which = 1: down.
+// Every wait on an mbarrier is bounded; on expiry the kernel records a status word and leaves.
 #include "common.cuh"
 
 namespace {
 
-constexpr int GV_THREADS = 256;
-constexpr int GV_WARPS = GV_THREADS / 32;
-constexpr int GV_UNROLL = 8;     // rows in flight per warp
+constexpr int GV_CONSUMER_WARPS = 8;
+constexpr int GV_THREADS = (GV_CONSUMER_WARPS + 1) * 32;   // + one producer warp
+constexpr int GV_SEG_BYTES = 2048;                         // bytes of one row handled by a CTA
+constexpr int GV_STAGE_ROWS = 16;
+constexpr int GV_STAGES = 5;
+constexpr int GV_MAX_ROWS = 1536;                          // kept rows per CTA (index list in smem)
+constexpr int GV_SCAN_THREADS = 256;                       // threads that scan the mask words
+constexpr unsigned long long GV_WAIT_LIMIT_NS = 1000000000ull;   // a wait gives up after one second
+
+struct GemvParams {
+    const char *W;             // packed rows
+    size_t row_bytes;          // bytes of one packed row
+    const float *v;            // [batch][d_in]
+    int d_in;
+    const uint32_t *mask_bits; // [batch][mask_words]; rows read = OR over the batch
+    int mask_words;
+    float *out;                // [batch][d_out]
+    int d_out;
+    int batch;                 // tokens in this launch (<= BT)
+    float *partials;
+    unsigned int *tickets;
+    int *status;               // device status word (0 = fine)
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait for the phase with the given parity; false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, unsigned parity)
+{
+    const uint32_t a = smem_u32(bar);
+    unsigned long long t0 = 0;
+    for (unsigned i = 0;; ++i) {
+        unsigned ok;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+                     " selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((i & 255u) == 255u) {
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > GV_WAIT_LIMIT_NS) return false;
+        }
+    }
+}
+// Bulk asynchronous copy global -> this CTA's shared memory, completion counted on `bar`.
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ float silu_f32(float g) { return g / (1.0f + expf(-g)); }
 
 template <int WT> struct WTraits;
-template <> struct WTraits<DIP_W_F32>  { static constexpr int E = 8;  static constexpr int BYTES = 32; };
-template <> struct WTraits<DIP_W_BF16> { static constexpr int E = 16; static constexpr int BYTES = 32; };
+template <> struct WTraits<DIP_W_F32>  { static constexpr int E = 4; static constexpr int EB = 4; };
+template <> struct WTraits<DIP_W_BF16> { static constexpr int E = 8; static constexpr int EB = 2; };
 
-struct Raw32 { uint4 a, b; };
-
-__device__ __forceinline__ uint4 ld_stream16(const void *p)
+template <int WT> __device__ __forceinline__ void decode16(const uint4 &r, float (&w)[WTraits<WT>::E]);
+template <> __device__ __forceinline__ void decode16<DIP_W_F32>(const uint4 &r, float (&w)[4])
 {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+    w[0] = __uint_as_float(r.x); w[1] = __uint_as_float(r.y);
+    w[2] = __uint_as_float(r.z); w[3] = __uint_as_float(r.w);
 }
-
-__device__ __forceinline__ Raw32 ld_row32(const char *p)
-{
-    Raw32 r;
-    r.a = ld_stream16(p);
-    r.b = ld_stream16(p + 16);
-    return r;
-}
-
-template <int WT> __device__ __forceinline__ void decode(const Raw32 &r, float (&w)[WTraits<WT>::E]);
-
-template <> __device__ __forceinline__ void decode<DIP_W_F32>(const Raw32 &r, float (&w)[8])
-{
-    w[0] = __uint_as_float(r.a.x); w[1] = __uint_as_float(r.a.y);
-    w[2] = __uint_as_float(r.a.z); w[3] = __uint_as_float(r.a.w);
-    w[4] = __uint_as_float(r.b.x); w[5] = __uint_as_float(r.b.y);
-    w[6] = __uint_as_float(r.b.z); w[7] = __uint_as_float(r.b.w);
-}
-
 // bfloat16 is the upper half of a binary32: widening is a shift or a mask.
-template <> __device__ __forceinline__ void decode<DIP_W_BF16>(const Raw32 &r, float (&w)[16])
+template <> __device__ __forceinline__ void decode16<DIP_W_BF16>(const uint4 &r, float (&w)[8])
 {
-    const uint32_t u[8] = {r.a.x, r.a.y, r.a.z, r.a.w, r.b.x, r.b.y, r.b.z, r.b.w};
+    const uint32_t u[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < 4; ++i) {
         w[2 * i] = __uint_as_float(u[i] << 16);
         w[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
     }
 }
 
-struct GemvParams {
-    const char *W;            // packed rows
-    size_t row_bytes;         // bytes of one packed row
-    int row_elems;            // elements of one packed row (2*d_ff or d_model)
-    const float *v;           // [batch][d_in]
-    int d_in;
-    const int32_t *kept_idx;
-    int n_kept;
-    const int32_t *n_kept_dev;
-    const uint32_t *mask_bits; // [batch][ceil(d_in/32)] or nullptr
-    int mask_words;
-    float *out;               // [batch][d_out]
-    int d_out;
-    int batch;                // tokens in this launch (<= BT)
-    float *partials;
-    unsigned int *tickets;
+struct __align__(16) GemvSmem {
+    unsigned char ring[GV_STAGES][GV_STAGE_ROWS][GV_SEG_BYTES];
+    uint64_t full[GV_STAGES];
+    uint64_t empty[GV_STAGES];
+    int idx[GV_MAX_ROWS];
+    uint32_t words[DIP_MAX_D / 32];
+    int pre[DIP_MAX_D / 32];
+    int wsum[GV_SCAN_THREADS / 32];
+    int n_total;
+    int last;
+    int issued;          // stages the producer has issued copies for
+    volatile int abort;
 };
 
-__device__ __forceinline__ float silu_f32(float g) { return g / (1.0f + expf(-g)); }
-
 template <int WT, int WHICH, int BT>
-__global__ void __launch_bounds__(GV_THREADS)
+__global__ void __launch_bounds__(GV_THREADS, 1)
 gemv_kernel(const GemvParams p)
 {
     constexpr int E = WTraits<WT>::E;
-    constexpr int SLAB = 32 * E;                              // packed elements per slab
+    constexpr int EB = WTraits<WT>::EB;
+    constexpr int SLAB = GV_SEG_BYTES / EB;                   // packed elements per slab
     constexpr int OUT_PER_SLAB = WHICH == 0 ? SLAB / 2 : SLAB;
-    constexpr int C = E / 2;                                  // gate/up chunk (outputs per lane)
-    __shared__ float s_red[GV_WARPS][SLAB];
-    __shared__ float s_sum[BT][SLAB];
-    __shared__ int s_last;
+    constexpr int C = 16 / EB;                                // gate/up interleave chunk (elements)
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    GemvSmem &s = *reinterpret_cast<GemvSmem *>(smem_raw);
+    float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem));   // [BT][GV_MAX_ROWS]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slab = blockIdx.x, part = blockIdx.y, nparts = gridDim.y;
-    const int n_rows = p.n_kept_dev ? *p.n_kept_dev : p.n_kept;
-    const int r_begin = (int)(((long long)part * n_rows) / nparts);
-    const int r_end = (int)(((long long)(part + 1) * n_rows) / nparts);
+    const size_t seg_off = (size_t)slab * GV_SEG_BYTES;
+    const int seg_bytes = (int)min((size_t)GV_SEG_BYTES, p.row_bytes - seg_off);
 
-    const int elem0 = slab * SLAB + lane * E;                 // first packed element of this lane
-    const bool lane_ok = elem0 < p.row_elems;
-    const char *wbase = p.W + (size_t)(lane_ok ? elem0 : 0) * (WTraits<WT>::BYTES / E);
+    if (tid == 0) {
+        for (int i = 0; i < GV_STAGES; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], GV_CONSUMER_WARPS);
+        }
+        s.abort = 0;
+        s.issued = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
 
-    float acc[BT][E];
+    // ---- 1. kept rows of this part, from the mask bits ----
+    if (tid < GV_SCAN_THREADS) {
+        // thread t owns words 4t .. 4t+3 (ascending), OR-ed over the tokens of the batch
+        uint32_t u[4];
+        int c = 0;
 #pragma unroll
-    for (int b = 0; b < BT; ++b)
+        for (int j = 0; j < 4; ++j) {
+            const int w = 4 * tid + j;
+            u[j] = 0;
+            if (w < p.mask_words)
+                for (int b = 0; b < p.batch; ++b) u[j] |= p.mask_bits[(size_t)b * p.mask_words + w];
+            if (w == p.mask_words - 1 && (p.d_in & 31)) u[j] &= (1u << (p.d_in & 31)) - 1u;   // no column beyond d_in
+            c += __popc(u[j]);
+        }
+        int incl = c;
 #pragma unroll
-        for (int e = 0; e < E; ++e) acc[b][e] = 0.f;
+        for (int o = 1; o < 32; o <<= 1) {
+            int n = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += n;
+        }
+        if (lane == 31) s.wsum[warp] = incl;
+        asm volatile("bar.sync 1, %0;" ::"n"(GV_SCAN_THREADS) : "memory");
+        int before = 0;
+#pragma unroll
+        for (int w = 0; w < GV_SCAN_THREADS / 32; ++w) before += w < warp ? s.wsum[w] : 0;
+        int pre = before + incl - c;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int w = 4 * tid + j;
+            if (w < p.mask_words) {
+                s.words[w] = u[j];
+                s.pre[w] = pre;
+            }
+            pre += __popc(u[j]);
+        }
+        if (tid == GV_SCAN_THREADS - 1) s.n_total = pre;
+    }
+    __syncthreads();
+    const int n_total = s.n_total;
+    const int r_begin = (int)(((long long)part * n_total) / nparts);
+    const int r_end = (int)(((long long)(part + 1) * n_total) / nparts);
+    const int n_rows = min(r_end - r_begin, GV_MAX_ROWS);     // the host sizes nparts so that this never clips
+    // row r of this CTA: the word holding rank r_begin + r (binary search), then the bit in it
+    for (int r = tid; r < n_rows; r += GV_THREADS) {
+        const int rank = r_begin + r;
+        int lo = 0, hi = p.mask_words - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (s.pre[mid] <= rank) lo = mid; else hi = mid - 1;
+        }
+        s.idx[r] = lo * 32 + (int)__fns(s.words[lo], 0, rank - s.pre[lo] + 1);
+    }
+    __syncthreads();
 
-    // this warp's rows: r_begin + warp, + GV_WARPS, ...
-    const int n_mine = (r_end - r_begin - warp + GV_WARPS - 1) / GV_WARPS;
-    for (int c0 = 0; c0 < n_mine; c0 += 32) {
-        // lane l stages row c0 + l of this warp: its column index and the tokens' values
-        int my_idx = 0;
-        float my_v[BT];
-#pragma unroll
-        for (int b = 0; b < BT; ++b) my_v[b] = 0.f;
-        if (c0 + lane < n_mine) {
-            my_idx = p.kept_idx[r_begin + warp + (c0 + lane) * GV_WARPS];
+    const int n_stages = (n_rows + GV_STAGE_ROWS - 1) / GV_STAGE_ROWS;
+    bool failed = false;
+
+    if (warp == GV_CONSUMER_WARPS) {
+        // ---- 2. producer warp: lane l copies row l of each stage ----
+        for (int it = 0; it < n_stages && !failed; ++it) {
+            const int st = it % GV_STAGES;
+            if (it >= GV_STAGES) {
+                if (!mbar_wait(&s.empty[st], ((it / GV_STAGES) - 1) & 1)) failed = true;
+            }
+            failed = __any_sync(0xffffffffu, failed) || s.abort;
+            if (failed) break;
+            const int rows_here = min(GV_STAGE_ROWS, n_rows - it * GV_STAGE_ROWS);
+            if (lane == 0) mbar_expect_tx(&s.full[st], (unsigned)(rows_here * seg_bytes));
+            __syncwarp();
+            if (lane < rows_here) {
+                const int idx = s.idx[it * GV_STAGE_ROWS + lane];
+                bulk_g2s(&s.ring[st][lane][0], p.W + (size_t)idx * p.row_bytes + seg_off, (unsigned)seg_bytes,
+                         &s.full[st]);
+            }
+            if (lane == 0) s.issued = it + 1;
+        }
+        if (failed && lane == 0) {
+            s.abort = 1;
+            atomicExch(p.status, 1);
+        }
+    } else {
+        // ---- 3. consumers ----
+        // the tokens' values for the kept rows (zero where a token's own mask drops the row)
+        for (int r = tid; r < n_rows; r += GV_CONSUMER_WARPS * 32) {
+            const int idx = s.idx[r];
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
-                if (b < p.batch) {
-                    bool on = true;
-                    if (p.mask_bits)
-                        on = (p.mask_bits[(size_t)b * p.mask_words + (my_idx >> 5)] >> (my_idx & 31)) & 1u;
-                    my_v[b] = on ? p.v[(size_t)b * p.d_in + my_idx] : 0.f;
-                }
+                float val = 0.f;
+                if (b < p.batch &&
+                    ((p.mask_bits[(size_t)b * p.mask_words + (idx >> 5)] >> (idx & 31)) & 1u))
+                    val = p.v[(size_t)b * p.d_in + idx];
+                s_v[b * GV_MAX_ROWS + r] = val;
             }
         }
-        const int n_here = min(32, n_mine - c0);
-        for (int j0 = 0; j0 < n_here; j0 += GV_UNROLL) {
-            Raw32 raw[GV_UNROLL];
+        asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
+
+        const int cw = warp & 3, rg = warp >> 2;
+        const int byte_off = cw * 512 + lane * 16;
+        const bool lane_ok = byte_off < seg_bytes;
+        float acc[BT][E];
 #pragma unroll
-            for (int u = 0; u < GV_UNROLL; ++u) {
-                int idx = __shfl_sync(0xffffffffu, my_idx, (j0 + u) & 31);
-                if (j0 + u < n_here && lane_ok)
-                    raw[u] = ld_row32(wbase + (size_t)idx * p.row_bytes);
-                else
-                    raw[u].a = raw[u].b = make_uint4(0, 0, 0, 0);
-            }
+        for (int b = 0; b < BT; ++b)
 #pragma unroll
-            for (int u = 0; u < GV_UNROLL; ++u) {
-                float w[E];
-                decode<WT>(raw[u], w);
+            for (int e = 0; e < E; ++e) acc[b][e] = 0.f;
+
+        for (int it = 0; it < n_stages; ++it) {
+            const int st = it % GV_STAGES;
+            if (!mbar_wait(&s.full[st], (it / GV_STAGES) & 1)) failed = true;
+            if (failed || s.abort) { failed = true; break; }
+            const int rows_here = min(GV_STAGE_ROWS, n_rows - it * GV_STAGE_ROWS);
+            if (lane_ok) {
 #pragma unroll
-                for (int b = 0; b < BT; ++b) {
-                    float xv = __shfl_sync(0xffffffffu, my_v[b], (j0 + u) & 31);
-                    if (j0 + u >= n_here) xv = 0.f;
+                for (int rr = 0; rr < GV_STAGE_ROWS / 2; ++rr) {
+                    const int r = 2 * rr + rg;
+                    if (r < rows_here) {
+                        const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r][byte_off]);
+                        float w[E];
+                        decode16<WT>(raw, w);
 #pragma unroll
-                    for (int e = 0; e < E; ++e) acc[b][e] = fmaf(w[e], xv, acc[b][e]);
+                        for (int b = 0; b < BT; ++b) {
+                            const float xv = s_v[b * GV_MAX_ROWS + it * GV_STAGE_ROWS + r];
+#pragma unroll
+                            for (int e = 0; e < E; ++e) acc[b][e] = fmaf(w[e], xv, acc[b][e]);
+                        }
+                    }
                 }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s.empty[st]);
+        }
+
+        if (failed) {
+            s.abort = 1;
+            if (lane == 0) atomicExch(p.status, 1);
+        }
+        // combine the two row groups: group 1 parks its sums in the (now idle) ring
+        float *red = reinterpret_cast<float *>(&s.ring[0][0][0]);    // [4 cw][32 lanes][BT][E]
+        asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
+        if (rg == 1) {
+#pragma unroll
+            for (int b = 0; b < BT; ++b)
+#pragma unroll
+                for (int e = 0; e < E; ++e) red[((cw * 32 + lane) * BT + b) * E + e] = acc[b][e];
+        }
+        asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
+        if (rg == 0) {
+            float *dst = nparts > 1 ? p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB)
+                                    : reinterpret_cast<float *>(&s.ring[1][0][0]);
+#pragma unroll
+            for (int b = 0; b < BT; ++b) {
+                float sum[E];
+#pragma unroll
+                for (int e = 0; e < E; ++e) sum[e] = acc[b][e] + red[((cw * 32 + lane) * BT + b) * E + e];
+                float *d = dst + b * SLAB + (cw * 512 + lane * 16) / EB;
+#pragma unroll
+                for (int e = 0; e < E; e += 4)
+                    *reinterpret_cast<float4 *>(d + e) = make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
             }
         }
     }
 
-    // combine the warps in warp order, one token at a time
-#pragma unroll
-    for (int b = 0; b < BT; ++b) {
-#pragma unroll
-        for (int e = 0; e < E; ++e) s_red[warp][lane * E + e] = acc[b][e];
-        __syncthreads();
-        for (int t = tid; t < SLAB; t += GV_THREADS) {
-            float sum = 0.f;
-#pragma unroll
-            for (int w = 0; w < GV_WARPS; ++w) sum += s_red[w][t];
-            s_sum[b][t] = sum;
-        }
-        __syncthreads();
-    }
-
+    // ---- 4. combine the parts ----
     if (nparts > 1) {
-        float *my_part = p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB);
-        for (int t = tid; t < BT * SLAB; t += GV_THREADS) my_part[t] = s_sum[t / SLAB][t % SLAB];
         __threadfence();
         __syncthreads();
-        if (tid == 0) {
-            unsigned prev = atomicAdd(&p.tickets[slab], 1u);
-            s_last = prev == (unsigned)(nparts - 1);
-        }
+        if (tid == 0) s.last = atomicAdd(&p.tickets[slab], 1u) == (unsigned)(nparts - 1);
         __syncthreads();
-        if (!s_last) return;
+        if (!s.last) return;
         __threadfence();
+    } else {
+        __syncthreads();
     }
-
-    // epilogue by the CTA that completes the slab
+    if (s.abort) {
+        // a wait ran out: let the copies already issued into this CTA's shared memory land
+        // (bounded again) before leaving, and leave the slab's counter clean
+        if (tid == 0) {
+            for (int it = max(0, s.issued - GV_STAGES); it < s.issued; ++it)
+                (void)mbar_wait(&s.full[it % GV_STAGES], (it / GV_STAGES) & 1);
+            if (nparts > 1) p.tickets[slab] = 0;
+        }
+        return;
+    }
+    const float *own = reinterpret_cast<const float *>(&s.ring[1][0][0]);
     for (int t = tid; t < BT * OUT_PER_SLAB; t += GV_THREADS) {
         const int b = t / OUT_PER_SLAB, o = t % OUT_PER_SLAB;
         const int j = slab * OUT_PER_SLAB + o;
         if (b >= p.batch || j >= p.d_out) continue;
         int e0, e1 = 0;
         if (WHICH == 0) {
-            e0 = (o / C) * E + (o % C);      // gate element of output o
-            e1 = e0 + C;                     // matching up element
+            e0 = (o / C) * 2 * C + (o % C);      // gate element of output o
+            e1 = e0 + C;                         // matching up element
         } else {
             e0 = o;
         }
@@ -206,8 +350,8 @@ gemv_kernel(const GemvParams p)
                 if (WHICH == 0) s1 += __ldcg(pp + e1);
             }
         } else {
-            s0 = s_sum[b][e0];
-            if (WHICH == 0) s1 = s_sum[b][e1];
+            s0 = own[b * SLAB + e0];
+            if (WHICH == 0) s1 = own[b * SLAB + e1];
         }
         p.out[(size_t)b * p.d_out + j] = WHICH == 0 ? silu_f32(s0) * s1 : s0;
     }
@@ -218,22 +362,38 @@ gemv_kernel(const GemvParams p)
 
 namespace {
 
+// Bit set from an ascending index list (the list-based entry points).
+__global__ void idx_to_mask_kernel(const int32_t *__restrict__ idx, int n, int d, uint32_t *__restrict__ mask)
+{
+    for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < n; r += gridDim.x * blockDim.x) {
+        const int i = idx[r];
+        if (i >= 0 && i < d) atomicOr(&mask[i >> 5], 1u << (i & 31));   // out-of-range entries are ignored
+    }
+}
+
 template <int WT, int WHICH, int BT>
 dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t stream)
 {
-    constexpr int SLAB = 32 * WTraits<WT>::E;
-    const int n_slabs = (p.row_elems + SLAB - 1) / SLAB;
+    constexpr int SLAB = GV_SEG_BYTES / WTraits<WT>::EB;
+    const int n_slabs = (int)((p.row_bytes + GV_SEG_BYTES - 1) / GV_SEG_BYTES);
     if (n_slabs > ctx->n_tickets) return DIP_ERR_WORKSPACE;
-    // enough CTAs to fill the device a few times over, but no part thinner than a few rows per warp
-    const int target = ctx->sm_count * 4;
-    int nparts = (target + n_slabs - 1) / n_slabs;
-    const int max_by_rows = n_kept_max / (2 * GV_WARPS);
-    if (nparts > max_by_rows) nparts = max_by_rows;
-    const size_t per_part = (size_t)n_slabs * BT * SLAB;
-    if ((size_t)nparts * per_part > ctx->partials_floats) nparts = (int)(ctx->partials_floats / per_part);
+    // one CTA per SM, all resident at once; parts no longer than the in-kernel row list
+    int nparts = ctx->sm_count / n_slabs;
+    const int min_parts = (n_kept_max + GV_MAX_ROWS - 1) / GV_MAX_ROWS;
+    if (nparts < min_parts) nparts = min_parts;
+    if (nparts > n_kept_max) nparts = n_kept_max;
     if (nparts < 1) nparts = 1;
+    const size_t per_part = (size_t)n_slabs * BT * SLAB;
+    if ((size_t)nparts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
+    const size_t smem = sizeof(GemvSmem) + (size_t)BT * GV_MAX_ROWS * sizeof(float);
+    static bool attr_set = false;   // per (WT, WHICH, BT) instantiation
+    if (!attr_set) {
+        DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(gemv_kernel<WT, WHICH, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)smem));
+        attr_set = true;
+    }
     dim3 grid(n_slabs, nparts);
-    gemv_kernel<WT, WHICH, BT><<<grid, GV_THREADS, 0, stream>>>(p);
+    gemv_kernel<WT, WHICH, BT><<<grid, GV_THREADS, smem, stream>>>(p);
     DIP_CUDA_TRY(ctx, cudaGetLastError());
     return DIP_OK;
 }
@@ -251,29 +411,26 @@ dip_status launch_bt(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t s
 }  // namespace
 
 dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
-                           const float *v, int batch,
-                           const int32_t *kept_idx, int n_kept_max, const int32_t *n_kept_dev,
-                           const uint32_t *mask_bits, float *out, cudaStream_t stream)
+                           const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
+                           float *out, cudaStream_t stream)
 {
     if (w->wtype != DIP_W_F32 && w->wtype != DIP_W_BF16) return DIP_ERR_UNSUPPORTED;
     const int elem_bytes = w->wtype == DIP_W_F32 ? 4 : 2;
     GemvParams p;
     p.W = (const char *)(which == 0 ? w->gate_up : w->down);
-    p.row_elems = which == 0 ? 2 * w->d_ff : w->d_model;
-    p.row_bytes = (size_t)p.row_elems * elem_bytes;
+    p.row_bytes = (size_t)(which == 0 ? 2 * w->d_ff : w->d_model) * elem_bytes;
     p.d_in = which == 0 ? w->d_model : w->d_ff;
     p.d_out = which == 0 ? w->d_ff : w->d_model;
-    p.kept_idx = kept_idx;
-    p.n_kept = n_kept_max;
-    p.n_kept_dev = n_kept_dev;
     p.mask_words = (p.d_in + 31) / 32;
     p.partials = ctx->partials;
     p.tickets = ctx->tickets;
-    // tokens go through in groups of at most four (accumulators live in registers)
+    p.status = ctx->status;
+    // tokens go through in groups of at most four (accumulators live in registers); each group
+    // reads the union of its own tokens' rows
     for (int b0 = 0; b0 < batch; b0 += 4) {
         p.batch = batch - b0 < 4 ? batch - b0 : 4;
         p.v = v + (size_t)b0 * p.d_in;
-        p.mask_bits = mask_bits ? mask_bits + (size_t)b0 * p.mask_words : nullptr;
+        p.mask_bits = mask_bits + (size_t)b0 * p.mask_words;
         p.out = out + (size_t)b0 * p.d_out;
         dip_status st;
         if (w->wtype == DIP_W_F32)
@@ -284,5 +441,13 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                             : launch_bt<DIP_W_BF16, 1>(ctx, p, n_kept_max, stream);
         if (st != DIP_OK) return st;
     }
+    return DIP_OK;
+}
+
+dip_status dip_launch_idx_to_mask(dip_ctx *ctx, const int32_t *idx, int n, int d, uint32_t *mask, cudaStream_t stream)
+{
+    DIP_CUDA_TRY(ctx, cudaMemsetAsync(mask, 0, sizeof(uint32_t) * ((d + 31) / 32), stream));
+    idx_to_mask_kernel<<<(n + 255) / 256, 256, 0, stream>>>(idx, n, d, mask);
+    DIP_CUDA_TRY(ctx, cudaGetLastError());
     return DIP_OK;
 }

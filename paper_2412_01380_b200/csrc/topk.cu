@@ -1,12 +1,14 @@
-// Masking kernels: magnitude top-k (Sec. 3.1, Eq. 7-8), the cache-aware ranking of Eq. 10
-// with the LRU column-cache update of Algorithm 1, the union of per-token masks for batched
-// decode, and the residual + RMS re-normalisation that chains layers.
+// Masking kernels: magnitude top-k (Sec. 3.1, Eq. 7-8), the cache-aware ranking of Eq. 10, the
+// LRU column-cache update of Algorithm 1, index lists / unions from bit masks, and the residual
+// + RMS re-normalisation that chains layers.
 //
-// One CTA of 1024 threads handles one input row.  The row's rank keys live in shared memory;
-// the k-th largest key is found by an 11-bit-per-pass radix select, then one ordered sweep
-// (warp ballots over 32 consecutive columns = one mask word) emits the bit mask and the
-// ascending index list.  Everything here is integer work on bit patterns, so results are
-// exact and unique (ties go to the lower column index).
+// The step's critical path only needs the mask, so the work is split in two kernels:
+//   select_kernel        rank keys -> k-th largest key by radix select -> bit mask.  One CTA of
+//                        1024 threads per row; the keys live in shared memory.
+//   cache_update_kernel  hits, misses, LRU victims and the new stamps from (mask, state).  It
+//                        does not feed the GEMVs and runs beside them on another stream.
+// Everything here is integer work on bit patterns, so results are exact and unique (ties go
+// to the lower column index).
 #include "common.cuh"
 
 namespace {
@@ -59,7 +61,7 @@ __device__ __forceinline__ int warp_array_prefix(const int *arr, int warp, int l
 // are by far the most frequent ones when the keys are ages of cache lines, are counted in
 // registers instead of with contended atomics.
 __device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask, int top_bit, int k,
-                                   TkShared &s, uint32_t &T, int &quota)
+                                   TkShared &s, uint32_t &T, int &quota, int &n_eq)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t prefix = 0, prefmask = 0;
@@ -118,16 +120,19 @@ __device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask
         if (cum < krem && krem <= cum + (int)h1) {
             s.bcast[0] = 2 * tid + 1;
             s.bcast[1] = krem - cum;
+            s.bcast[2] = (int)h1;
         }
         cum += (int)h1;
         if (cum < krem && krem <= cum + (int)h0) {
             s.bcast[0] = 2 * tid;
             s.bcast[1] = krem - cum;
+            s.bcast[2] = (int)h0;
         }
         __syncthreads();
         prefix |= (uint32_t)s.bcast[0] << shift;
         prefmask |= dmask << shift;
         krem = s.bcast[1];
+        n_eq = s.bcast[2];        // after the last pass: the number of keys equal to T
         hi = shift;
     }
     T = prefix;
@@ -135,10 +140,10 @@ __device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask
 }
 
 // ---------------------------------------------------------------------------------------
-// mask_kernel: Algorithm 1 for one row.
+// select_kernel: the mask of one row.
 //   CA == false: key = bits(|x|)                              (DIP, Eq. 7-8)
-//   CA == true : key = bits(|x| * (resident ? 1 : gamma))     (numerator of Eq. 10), then the
-//                LRU cache update c' = cache_update(c, m).
+//   CA == true : key = bits(|x| * (resident ? 1 : gamma))     (numerator of Eq. 10); the cache
+//                state is only read.
 //   NORM == true: the row is first formed as x = (xa + xb) / rms(xa + xb) (the layer chaining
 //                of a stack) and written to x_out; the summation order is that of
 //                residual_rmsnorm_kernel, so both give the same bits.
@@ -146,13 +151,12 @@ __device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask
 // ---------------------------------------------------------------------------------------
 template <bool CA, bool NORM>
 __global__ void __launch_bounds__(TK_THREADS, 1)
-mask_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *__restrict__ x_out,
-            int d, int k, float gamma, int32_t *stamp, int32_t *meta, int capacity,
-            uint32_t *__restrict__ mask_bits, int32_t *__restrict__ kept_idx)
+select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *__restrict__ x_out,
+              int d, int k, float gamma, const int32_t *__restrict__ stamp,
+              uint32_t *__restrict__ mask_bits)
 {
     extern __shared__ uint32_t keys[];
     __shared__ TkShared s;
-    __shared__ unsigned int s_mask[DIP_MAX_D / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x;
     const int n_words = (d + 31) >> 5;
@@ -161,14 +165,7 @@ mask_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *_
         xb += (size_t)row * d;
         x_out += (size_t)row * d;
     }
-    if (mask_bits) mask_bits += (size_t)row * n_words;
-    if (kept_idx) kept_idx += (size_t)row * k;
-
-    int n_res = 0, t_now = 0;
-    if (CA) {
-        n_res = meta[0];
-        t_now = meta[1] + 1;
-    }
+    mask_bits += (size_t)row * n_words;
 
     if (NORM) {
         float ss = 0.f;
@@ -207,76 +204,80 @@ mask_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *_
     __syncthreads();
 
     uint32_t T;
-    int quota;
-    block_radix_select(keys, d, 0x7fffffffu, 31, k, s, T, quota);
+    int quota, n_eq;
+    block_radix_select(keys, d, 0x7fffffffu, 31, k, s, T, quota, n_eq);
 
-    // ordered sweeps: warp w owns columns [w*span, (w+1)*span), span a multiple of 32
+    // warp w owns columns [w*span, (w+1)*span), span a multiple of 32: one ballot = one mask word
+    const int span = ((d + TK_THREADS - 1) / TK_THREADS) * 32;
+    const int base = warp * span;
+    if (quota == n_eq) {
+        // every column tied with the threshold is kept: the mask is key >= T
+        for (int it = 0; it < span && base + it < d; it += 32) {
+            const int e = base + it + lane;
+            const unsigned bk = __ballot_sync(0xffffffffu, e < d && keys[e] >= T);
+            if (lane == 0) mask_bits[(base + it) >> 5] = bk;
+        }
+        return;
+    }
+    // only the first `quota` tied columns (by index) are kept: rank the ties in order
+    const unsigned lt = lanemask_lt();
+    int eq = 0;
+    for (int it = 0; it < span; it += 32) {
+        const int e = base + it + lane;
+        eq += __popc(__ballot_sync(0xffffffffu, e < d && keys[e] == T));
+    }
+    if (lane == 0) s.wb[warp] = eq;
+    __syncthreads();
+    int tot;
+    int eq_before = warp_array_prefix(s.wb, warp, lane, tot);
+    for (int it = 0; it < span && base + it < d; it += 32) {
+        const int e = base + it + lane;
+        const uint32_t key = e < d ? keys[e] : 0u;
+        const bool q = e < d && key == T;
+        const unsigned bq = __ballot_sync(0xffffffffu, q);
+        const bool keep = (e < d && key > T) || (q && (eq_before + __popc(bq & lt)) < quota);
+        const unsigned bk = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) mask_bits[(base + it) >> 5] = bk;
+        eq_before += __popc(bq);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// cache_update_kernel: c' = cache_update(c, m) of Algorithm 1 with the LRU policy of Sec. 5.1,
+// from the mask bits and the state alone.  One CTA; keys[] (dynamic shared memory, d words)
+// holds (resident flag << 31) | eviction key, the eviction key being the age of the column's
+// last use for columns that may be evicted (resident and outside the mask) and 0 otherwise.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(TK_THREADS, 1)
+cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stamp, int32_t *meta, int capacity)
+{
+    extern __shared__ uint32_t keys[];
+    __shared__ TkShared s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_res = meta[0];
+    const int t_now = meta[1] + 1;
     const int span = ((d + TK_THREADS - 1) / TK_THREADS) * 32;
     const int base = warp * span;
     const unsigned lt = lanemask_lt();
 
-    int gt = 0, eq = 0;
-    for (int it = 0; it < span; it += 32) {
-        int e = base + it + lane;
-        uint32_t key = e < d ? keys[e] : 0u;
-        bool valid = e < d;
-        gt += __popc(__ballot_sync(0xffffffffu, valid && key > T));
-        eq += __popc(__ballot_sync(0xffffffffu, valid && key == T));
-    }
-    if (lane == 0) {
-        s.wa[warp] = gt;
-        s.wb[warp] = eq;
-    }
-    __syncthreads();
-    int tot;
-    int gt_before = warp_array_prefix(s.wa, warp, lane, tot);
-    int eq_before = warp_array_prefix(s.wb, warp, lane, tot);
-    __syncthreads();   // wa/wb are reused below
-
-    // second sweep: emit the mask and the index list; for CA also turn keys[] into
-    // (resident flag << 31) | eviction key and count hits and misses
     int hits = 0, misses = 0;
-    for (int it = 0; it < span; it += 32) {
-        int e = base + it + lane;
-        bool valid = e < d;
-        uint32_t key = valid ? keys[e] : 0u;
-        bool g = valid && key > T;
-        bool q = valid && key == T;
-        unsigned bg = __ballot_sync(0xffffffffu, g);
-        unsigned bq = __ballot_sync(0xffffffffu, q);
-        bool keep = g || (q && (eq_before + __popc(bq & lt)) < quota);
-        unsigned bk = __ballot_sync(0xffffffffu, keep);
-        if (base + it < d) {
-            if (lane == 0) {
-                if (CA) s_mask[(base + it) >> 5] = bk;
-                if (mask_bits) mask_bits[(base + it) >> 5] = bk;
-            }
-            if (kept_idx && keep) {
-                int pos = gt_before + min(eq_before, quota) + __popc(bk & lt);
-                kept_idx[pos] = e;
-            }
-        }
-        if (CA) {
-            int st = valid ? stamp[e] : -1;
-            bool res = st >= 0;
-            // eviction key = age of the last use: an older column has a larger key; columns
-            // that cannot be evicted (not resident, or in the current mask) get 0
-            if (valid) keys[e] = (res ? 0x80000000u : 0u) | ((res && !keep) ? (uint32_t)(t_now - st) : 0u);
-            hits += __popc(__ballot_sync(0xffffffffu, keep && res));
-            misses += __popc(__ballot_sync(0xffffffffu, keep && !res));
-        }
-        gt_before += __popc(bg);
-        eq_before += __popc(bq);
+    for (int it = 0; it < span && base + it < d; it += 32) {
+        const int e = base + it + lane;
+        const bool valid = e < d;
+        const unsigned mw = mask_bits[(base + it) >> 5];
+        const bool keep = valid && ((mw >> lane) & 1u);
+        const int st = valid ? stamp[e] : -1;
+        const bool res = st >= 0;
+        if (valid) keys[e] = (res ? 0x80000000u : 0u) | ((res && !keep) ? (uint32_t)(t_now - st) : 0u);
+        hits += __popc(__ballot_sync(0xffffffffu, keep && res));
+        misses += __popc(mw) - __popc(__ballot_sync(0xffffffffu, keep && res));
     }
-    if (!CA) return;
-
-    // ---------------- cache update (LRU, Sec. 5.1; Algorithm 1's cache_update) ----------------
     if (lane == 0) {
         s.wa[warp] = hits;
         s.wc[warp] = misses;
     }
     __syncthreads();
-    int total_hits, total_misses;
+    int total_hits, total_misses, tot;
     (void)warp_array_prefix(s.wa, warp, lane, total_hits);
     int miss_before = warp_array_prefix(s.wc, warp, lane, total_misses);
     const int free_slots = capacity - n_res;
@@ -287,48 +288,51 @@ mask_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *_
 
     // victims: the n_evict largest eviction keys (oldest stamps), lower index first among equals
     uint32_t T2 = 0x7fffffffu;   // no key exceeds it: no victim
-    int quota2 = 0;
+    int quota2 = 0, n_eq2 = 0;
     if (n_evict > 0) {
         if (n_evict == evictable)
             T2 = 0u;             // every evictable column (key > 0) goes
         else
-            block_radix_select(keys, d, 0x7fffffffu, 32 - __clz(t_now), n_evict, s, T2, quota2);
+            block_radix_select(keys, d, 0x7fffffffu, 32 - __clz(t_now), n_evict, s, T2, quota2, n_eq2);
     }
-
-    // ordered rank of the eviction-key ties
+    // ordered rank of the eviction-key ties (needed only if some of them stay)
     int veq_before = 0;
-    if (quota2 > 0) {
+    const bool ranked_ties = quota2 > 0 && quota2 < n_eq2;
+    if (ranked_ties) {
         int veq = 0;
         for (int it = 0; it < span; it += 32) {
-            int e = base + it + lane;
+            const int e = base + it + lane;
             veq += __popc(__ballot_sync(0xffffffffu, e < d && (keys[e] & 0x7fffffffu) == T2));
         }
         if (lane == 0) s.wb[warp] = veq;
         __syncthreads();
         veq_before = warp_array_prefix(s.wb, warp, lane, tot);
     }
+    const bool all_ties = quota2 > 0 && !ranked_ties;
 
-    for (int it = 0; it < span; it += 32) {
-        int e = base + it + lane;
-        bool valid = e < d;
-        uint32_t kv = valid ? keys[e] : 0u;
-        uint32_t vkey = kv & 0x7fffffffu;
-        bool res = (kv >> 31) != 0u;
-        bool keep = valid && ((s_mask[e >> 5] >> lane) & 1u);
-        bool vq = valid && quota2 > 0 && vkey == T2;
-        unsigned bvq = __ballot_sync(0xffffffffu, vq);
-        bool evict = valid && (vkey > T2 || (vq && (veq_before + __popc(bvq & lt)) < quota2));
-        bool miss = keep && !res;
-        unsigned bm = __ballot_sync(0xffffffffu, miss);
-        if (valid) {
-            if (evict) {
-                stamp[e] = -1;
-            } else if (keep) {
-                // a hit, or a miss that still finds room (ascending index order)
-                if (!miss || (miss_before + __popc(bm & lt)) < room) stamp[e] = t_now;
-            }
+    for (int it = 0; it < span && base + it < d; it += 32) {
+        const int e = base + it + lane;
+        const bool valid = e < d;
+        const uint32_t kv = valid ? keys[e] : 0u;
+        const uint32_t vkey = kv & 0x7fffffffu;
+        const bool res = (kv >> 31) != 0u;
+        const bool keep = valid && ((mask_bits[(base + it) >> 5] >> lane) & 1u);
+        const bool vq = valid && vkey == T2 && vkey != 0u;
+        bool evict = valid && vkey > T2;
+        if (all_ties) evict = evict || vq;
+        if (ranked_ties) {
+            const unsigned bvq = __ballot_sync(0xffffffffu, vq);
+            evict = evict || (vq && (veq_before + __popc(bvq & lt)) < quota2);
+            veq_before += __popc(bvq);
         }
-        veq_before += __popc(bvq);
+        const bool miss = keep && !res;
+        const unsigned bm = __ballot_sync(0xffffffffu, miss);
+        if (evict) {
+            stamp[e] = -1;
+        } else if (keep) {
+            // a hit, or a miss that still finds room (ascending index order)
+            if (!miss || (miss_before + __popc(bm & lt)) < room) stamp[e] = t_now;
+        }
         miss_before += __popc(bm);
     }
     if (tid == 0) {
@@ -343,19 +347,21 @@ mask_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *_
 }
 
 // ---------------------------------------------------------------------------------------
-// union_kernel: U = OR_b m_b as an ascending index list plus |U| (batched decode: the set of
-// weight columns a step reads once).  One CTA; thread t owns mask word t.
+// mask_to_idx_kernel: ascending index list of a bit mask, or of the union of `nb` masks
+// (batched decode: the set of weight columns a step reads once).  CTA r handles masks
+// r*nb .. r*nb+nb-1 and writes to idx_out + r*out_stride; thread t owns mask word t.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(TK_THREADS, 1)
-union_kernel(const uint32_t *__restrict__ mask_bits, int batch, int d,
-             int32_t *__restrict__ union_idx, int32_t *__restrict__ union_count)
+mask_to_idx_kernel(const uint32_t *__restrict__ mask_bits, int nb, int d,
+                   int32_t *__restrict__ idx_out, int out_stride, int32_t *__restrict__ count_out)
 {
     __shared__ int wsum[TK_WARPS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_words = (d + 31) >> 5;
+    mask_bits += (size_t)blockIdx.x * nb * n_words;
     uint32_t u = 0;
     if (tid < n_words)
-        for (int b = 0; b < batch; ++b) u |= mask_bits[(size_t)b * n_words + tid];
+        for (int b = 0; b < nb; ++b) u |= mask_bits[(size_t)b * n_words + tid];
     int c = __popc(u);
     int incl = c;
 #pragma unroll
@@ -367,12 +373,15 @@ union_kernel(const uint32_t *__restrict__ mask_bits, int batch, int d,
     __syncthreads();
     int total;
     int before = warp_array_prefix(wsum, warp, lane, total) + incl - c;
-    while (u) {
-        int bit = __ffs(u) - 1;
-        u &= u - 1;
-        union_idx[before++] = tid * 32 + bit;
+    if (idx_out) {
+        int32_t *o = idx_out + (size_t)blockIdx.x * out_stride;
+        while (u) {
+            int bit = __ffs(u) - 1;
+            u &= u - 1;
+            o[before++] = tid * 32 + bit;
+        }
     }
-    if (tid == 0) *union_count = total;
+    if (count_out && tid == 0) count_out[blockIdx.x] = total;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -414,53 +423,50 @@ residual_rmsnorm_kernel(const float *x, const float *__restrict__ y, int d, floa
 // ---------------------------------------------------------------------------------------
 // host launchers
 // ---------------------------------------------------------------------------------------
-dip_status dip_launch_mask(dip_ctx *ctx, const float *x, int batch, int d, int k, float gamma,
-                           int32_t *stamp, int32_t *meta, int capacity,
-                           uint32_t *mask_bits, int32_t *kept_idx, cudaStream_t stream)
+dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d, int k,
+                             float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream)
 {
     const size_t smem = (size_t)d * sizeof(uint32_t);
-    if (stamp)
-        mask_kernel<true, false><<<batch, TK_THREADS, smem, stream>>>(x, nullptr, nullptr, d, k, gamma, stamp, meta,
-                                                                      capacity, mask_bits, kept_idx);
-    else
-        mask_kernel<false, false><<<batch, TK_THREADS, smem, stream>>>(x, nullptr, nullptr, d, k, 1.0f, nullptr,
-                                                                       nullptr, 0, mask_bits, kept_idx);
+    if (xb) {
+        if (stamp)
+            select_kernel<true, true><<<batch, TK_THREADS, smem, stream>>>(xa, xb, x_out, d, k, gamma, stamp, mask_bits);
+        else
+            select_kernel<false, true><<<batch, TK_THREADS, smem, stream>>>(xa, xb, x_out, d, k, 1.0f, nullptr, mask_bits);
+    } else {
+        if (stamp)
+            select_kernel<true, false><<<batch, TK_THREADS, smem, stream>>>(xa, nullptr, nullptr, d, k, gamma, stamp, mask_bits);
+        else
+            select_kernel<false, false><<<batch, TK_THREADS, smem, stream>>>(xa, nullptr, nullptr, d, k, 1.0f, nullptr, mask_bits);
+    }
     DIP_CUDA_TRY(ctx, cudaGetLastError());
     return DIP_OK;
 }
 
-// x_out = (xa + xb) / rms(xa + xb), then the mask of x_out: one launch for the layer chaining
-// and the first mask of the next layer.
-dip_status dip_launch_norm_mask(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d,
-                                int k, float gamma, int32_t *stamp, int32_t *meta, int capacity,
-                                uint32_t *mask_bits, int32_t *kept_idx, cudaStream_t stream)
+dip_status dip_launch_cache_update(dip_ctx *ctx, const uint32_t *mask_bits, int d, int32_t *stamp, int32_t *meta,
+                                   int capacity, cudaStream_t stream)
 {
-    const size_t smem = (size_t)d * sizeof(uint32_t);
-    if (stamp)
-        mask_kernel<true, true><<<batch, TK_THREADS, smem, stream>>>(xa, xb, x_out, d, k, gamma, stamp, meta,
-                                                                     capacity, mask_bits, kept_idx);
-    else
-        mask_kernel<false, true><<<batch, TK_THREADS, smem, stream>>>(xa, xb, x_out, d, k, 1.0f, nullptr, nullptr,
-                                                                      0, mask_bits, kept_idx);
+    cache_update_kernel<<<1, TK_THREADS, (size_t)d * sizeof(uint32_t), stream>>>(mask_bits, d, stamp, meta, capacity);
     DIP_CUDA_TRY(ctx, cudaGetLastError());
     return DIP_OK;
 }
 
-// Per-device set-up: the mask kernels keep up to DIP_MAX_D rank keys in dynamic shared memory.
+// Per-device set-up: the mask kernels keep up to DIP_MAX_D keys in dynamic shared memory.
 dip_status dip_init_mask_kernels(dip_ctx *ctx)
 {
     const int bytes = DIP_MAX_D * (int)sizeof(uint32_t);
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(mask_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(cache_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     return DIP_OK;
 }
 
-dip_status dip_launch_union(dip_ctx *ctx, const uint32_t *mask_bits, int batch, int d,
-                            int32_t *union_idx, int32_t *union_count, cudaStream_t stream)
+// rows x (OR of nb masks) -> ascending index lists (and their lengths)
+dip_status dip_launch_mask_to_idx(dip_ctx *ctx, const uint32_t *mask_bits, int rows, int nb, int d,
+                                  int32_t *idx_out, int out_stride, int32_t *count_out, cudaStream_t stream)
 {
-    union_kernel<<<1, TK_THREADS, 0, stream>>>(mask_bits, batch, d, union_idx, union_count);
+    mask_to_idx_kernel<<<rows, TK_THREADS, 0, stream>>>(mask_bits, nb, d, idx_out, out_stride, count_out);
     DIP_CUDA_TRY(ctx, cudaGetLastError());
     return DIP_OK;
 }
