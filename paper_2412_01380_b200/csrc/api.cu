@@ -2,6 +2,7 @@
 // composition of the kernels into the sparse MLP step of Eq. 3 / 7 / 8.
 #include <math.h>
 #include <new>
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -80,6 +81,10 @@ dip_status dip_create(dip_ctx **out, int device)
     if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
         return fail(DIP_ERR_CUDA);
     ctx->partials_floats = PARTIALS_FLOATS;
+    if (const char *e = getenv("DIP_GEMV_SEG")) {          // tuning aid: force the GEMV segment width
+        const int v = atoi(e);
+        if (v == 512 || v == 1024 || v == 2048) ctx->gemv_seg = v;
+    }
     ctx->n_tickets = N_TICKETS;
     const size_t vec = (size_t)DIP_MAX_BATCH * DIP_MAX_D;
     if ((st = dev_alloc(ctx, &ctx->partials, ctx->partials_floats)) != DIP_OK) return fail(st);

@@ -11,6 +11,7 @@
 struct dip_ctx {
     int device;
     int sm_count;
+    int gemv_seg;        // 0 = choose per launch; else force the GEMV segment width (tuning aid)
     // split-row partial sums of the two GEMVs (binary32)
     float *partials;
     size_t partials_floats;
@@ -50,6 +51,34 @@ constexpr int DIP_RING_LAYERS = 128;
             return DIP_ERR_CUDA;                                                       \
         }                                                                              \
     } while (0)
+
+#ifdef __CUDACC__
+// Programmatic dependent launch: a kernel may be scheduled before its predecessor in the stream
+// has finished; it must not touch the predecessor's results before this wait returns.
+__device__ __forceinline__ void dip_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream be scheduled early (it still waits as above).
+__device__ __forceinline__ void dip_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+
+// Launch on `stream` with programmatic dependent launch enabled: the kernel may start while the
+// previous kernel in the stream drains; it orders itself with dip_grid_dependency_wait().
+template <typename... KArgs, typename... Args>
+static inline cudaError_t dip_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                         cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
 
 static inline bool dip_aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
 

@@ -1,14 +1,14 @@
 // Sparse vector-matrix products over the kept weight columns (Eq. 3 with the masks of Eq. 7-8).
 //
 // A packed matrix stores column i of W as row i (see dip.h), so a kept column is one contiguous
-// row.  The kernel is a gather-GEMV: grid = (output slabs of 2 KB of row) x (row parts), sized to
-// one CTA per SM.  Each CTA
+// row.  The kernel is a gather-GEMV: grid = (output slabs of SEG bytes of row) x (row parts),
+// sized to one CTA per SM.  Each CTA
 //   1. reads the mask bits, prefix-sums their popcounts and extracts the kept rows whose rank
 //      falls in its part (so parts are balanced whatever the mask looks like);
-//   2. streams its rows' 2 KB slab segments from HBM into a ring of shared-memory stages with
+//   2. streams its rows' slab segments from HBM into a ring of shared-memory stages with
 //      bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts), issued by one
 //      producer warp, so that ~160 KB per SM are in flight independent of register pressure;
-//   3. eight consumer warps (4 column groups x 2 row groups) multiply-accumulate from shared
+//   3. eight consumer warps (column groups x row groups) multiply-accumulate from shared
 //      memory, 16 bytes of a row per lane, in binary32;
 //   4. the row groups are combined through shared memory, the parts through a scratch buffer in
 //      part order by the last CTA to arrive at the slab (an arrival counter).
@@ -22,10 +22,8 @@ namespace {
 
 constexpr int GV_CONSUMER_WARPS = 8;
 constexpr int GV_THREADS = (GV_CONSUMER_WARPS + 1) * 32;   // + one producer warp
-constexpr int GV_SEG_BYTES = 2048;                         // bytes of one row handled by a CTA
-constexpr int GV_STAGE_ROWS = 16;
 constexpr int GV_STAGES = 5;
-constexpr int GV_MAX_ROWS = 1536;                          // kept rows per CTA (index list in smem)
+constexpr int GV_MAX_ROWS = 2048;                          // kept rows per round (index list in smem)
 constexpr int GV_SCAN_THREADS = 256;                       // threads that scan the mask words
 constexpr unsigned long long GV_WAIT_LIMIT_NS = 1000000000ull;   // a wait gives up after one second
 
@@ -106,8 +104,10 @@ template <> __device__ __forceinline__ void decode16<DIP_W_BF16>(const uint4 &r,
     }
 }
 
-struct __align__(16) GemvSmem {
-    unsigned char ring[GV_STAGES][GV_STAGE_ROWS][GV_SEG_BYTES];
+constexpr int GV_STAGE_BYTES = 32768;
+
+template <int SEG> struct __align__(16) GemvSmem {
+    unsigned char ring[GV_STAGES][GV_STAGE_BYTES];   // [stage][row][SEG]
     uint64_t full[GV_STAGES];
     uint64_t empty[GV_STAGES];
     int idx[GV_MAX_ROWS];
@@ -120,23 +120,28 @@ struct __align__(16) GemvSmem {
     volatile int abort;
 };
 
-template <int WT, int WHICH, int BT>
+// SEG = bytes of one row handled by a CTA (512, 1024 or 2048): SEG/512 column groups of one warp
+// each (16 bytes per lane), 8/(SEG/512) row groups; a stage holds 32 KB = 32768/SEG rows.
+template <int WT, int WHICH, int BT, int SEG>
 __global__ void __launch_bounds__(GV_THREADS, 1)
 gemv_kernel(const GemvParams p)
 {
     constexpr int E = WTraits<WT>::E;
     constexpr int EB = WTraits<WT>::EB;
-    constexpr int SLAB = GV_SEG_BYTES / EB;                   // packed elements per slab
+    constexpr int SLAB = SEG / EB;                            // packed elements per slab
     constexpr int OUT_PER_SLAB = WHICH == 0 ? SLAB / 2 : SLAB;
     constexpr int C = 16 / EB;                                // gate/up interleave chunk (elements)
+    constexpr int CG = SEG / 512;                             // column groups (warps across the segment)
+    constexpr int RG = GV_CONSUMER_WARPS / CG;                // row groups
+    constexpr int R = GV_STAGE_BYTES / SEG;                   // rows per stage
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    GemvSmem &s = *reinterpret_cast<GemvSmem *>(smem_raw);
-    float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem));   // [BT][GV_MAX_ROWS]
+    GemvSmem<SEG> &s = *reinterpret_cast<GemvSmem<SEG> *>(smem_raw);
+    float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem<SEG>));   // [BT][GV_MAX_ROWS]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slab = blockIdx.x, part = blockIdx.y, nparts = gridDim.y;
-    const size_t seg_off = (size_t)slab * GV_SEG_BYTES;
-    const int seg_bytes = (int)min((size_t)GV_SEG_BYTES, p.row_bytes - seg_off);
+    const size_t seg_off = (size_t)slab * SEG;
+    const int seg_bytes = (int)min((size_t)SEG, p.row_bytes - seg_off);
 
     if (tid == 0) {
         for (int i = 0; i < GV_STAGES; ++i) {
@@ -147,18 +152,30 @@ gemv_kernel(const GemvParams p)
         s.issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    dip_grid_dependency_wait();        // the mask and the vector come from the previous kernels
+    dip_launch_dependents();
 
-    // ---- 1. kept rows of this part, from the mask bits ----
+    // ---- 1. the mask words and their popcount prefix ----
     if (tid < GV_SCAN_THREADS) {
         // thread t owns words 4t .. 4t+3 (ascending), OR-ed over the tokens of the batch
-        uint32_t u[4];
+        uint32_t u[4] = {0u, 0u, 0u, 0u};
         int c = 0;
+        if (4 * tid < p.mask_words) {
+            if ((p.mask_words & 3) == 0) {
+                for (int b = 0; b < p.batch; ++b) {
+                    const uint4 q = *reinterpret_cast<const uint4 *>(p.mask_bits + (size_t)b * p.mask_words + 4 * tid);
+                    u[0] |= q.x; u[1] |= q.y; u[2] |= q.z; u[3] |= q.w;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (4 * tid + j < p.mask_words)
+                        for (int b = 0; b < p.batch; ++b) u[j] |= p.mask_bits[(size_t)b * p.mask_words + 4 * tid + j];
+            }
+        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int w = 4 * tid + j;
-            u[j] = 0;
-            if (w < p.mask_words)
-                for (int b = 0; b < p.batch; ++b) u[j] |= p.mask_bits[(size_t)b * p.mask_words + w];
             if (w == p.mask_words - 1 && (p.d_in & 31)) u[j] &= (1u << (p.d_in & 31)) - 1u;   // no column beyond d_in
             c += __popc(u[j]);
         }
@@ -189,127 +206,150 @@ gemv_kernel(const GemvParams p)
     const int n_total = s.n_total;
     const int r_begin = (int)(((long long)part * n_total) / nparts);
     const int r_end = (int)(((long long)(part + 1) * n_total) / nparts);
-    const int n_rows = min(r_end - r_begin, GV_MAX_ROWS);     // the host sizes nparts so that this never clips
-    // row r of this CTA: the word holding rank r_begin + r (binary search), then the bit in it
-    for (int r = tid; r < n_rows; r += GV_THREADS) {
-        const int rank = r_begin + r;
-        int lo = 0, hi = p.mask_words - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (s.pre[mid] <= rank) lo = mid; else hi = mid - 1;
-        }
-        s.idx[r] = lo * 32 + (int)__fns(s.words[lo], 0, rank - s.pre[lo] + 1);
-    }
-    __syncthreads();
 
-    const int n_stages = (n_rows + GV_STAGE_ROWS - 1) / GV_STAGE_ROWS;
+    const int cw = warp % CG, rg = warp / CG;                 // consumer roles
+    const int byte_off = cw * 512 + lane * 16;
+    const bool lane_ok = byte_off < seg_bytes;
+    float acc[BT][E];
+#pragma unroll
+    for (int b = 0; b < BT; ++b)
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[b][e] = 0.f;
     bool failed = false;
+    int it_base = 0;                                          // stages issued in earlier rounds
 
-    if (warp == GV_CONSUMER_WARPS) {
-        // ---- 2. producer warp: lane l copies row l of each stage ----
-        for (int it = 0; it < n_stages && !failed; ++it) {
-            const int st = it % GV_STAGES;
-            if (it >= GV_STAGES) {
-                if (!mbar_wait(&s.empty[st], ((it / GV_STAGES) - 1) & 1)) failed = true;
-            }
-            failed = __any_sync(0xffffffffu, failed) || s.abort;
-            if (failed) break;
-            const int rows_here = min(GV_STAGE_ROWS, n_rows - it * GV_STAGE_ROWS);
-            if (lane == 0) mbar_expect_tx(&s.full[st], (unsigned)(rows_here * seg_bytes));
-            __syncwarp();
-            if (lane < rows_here) {
-                const int idx = s.idx[it * GV_STAGE_ROWS + lane];
-                bulk_g2s(&s.ring[st][lane][0], p.W + (size_t)idx * p.row_bytes + seg_off, (unsigned)seg_bytes,
-                         &s.full[st]);
-            }
-            if (lane == 0) s.issued = it + 1;
+    // The part's rows go through in rounds of at most GV_MAX_ROWS (the in-kernel row list).
+    for (int round_begin = r_begin; round_begin < r_end; round_begin += GV_MAX_ROWS) {
+        const int n_rows = min(r_end - round_begin, GV_MAX_ROWS);
+        if (round_begin != r_begin) {
+            __syncthreads();                                  // everyone is done with the previous list
+            if (s.abort) break;                               // uniform: read after the barrier
         }
-        if (failed && lane == 0) {
-            s.abort = 1;
-            atomicExch(p.status, 1);
-        }
-    } else {
-        // ---- 3. consumers ----
-        // the tokens' values for the kept rows (zero where a token's own mask drops the row)
-        for (int r = tid; r < n_rows; r += GV_CONSUMER_WARPS * 32) {
-            const int idx = s.idx[r];
-#pragma unroll
-            for (int b = 0; b < BT; ++b) {
-                float val = 0.f;
-                if (b < p.batch &&
-                    ((p.mask_bits[(size_t)b * p.mask_words + (idx >> 5)] >> (idx & 31)) & 1u))
-                    val = p.v[(size_t)b * p.d_in + idx];
-                s_v[b * GV_MAX_ROWS + r] = val;
+        // ---- 2. the round's rows in rank order: each mask word that overlaps the round's rank
+        //         range is expanded by one thread ----
+        {
+            const int lo_rank = round_begin, hi_rank = round_begin + n_rows;
+            for (int w = tid; w < p.mask_words; w += GV_THREADS) {
+                uint32_t u = s.words[w];
+                int rank = s.pre[w];
+                if (rank >= hi_rank || rank + __popc(u) <= lo_rank) continue;
+                while (u) {
+                    const int bit = __ffs(u) - 1;
+                    u &= u - 1;
+                    if (rank >= lo_rank && rank < hi_rank) s.idx[rank - lo_rank] = w * 32 + bit;
+                    ++rank;
+                }
             }
         }
-        asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
+        __syncthreads();
+        const int n_stages = (n_rows + R - 1) / R;
 
-        const int cw = warp & 3, rg = warp >> 2;
-        const int byte_off = cw * 512 + lane * 16;
-        const bool lane_ok = byte_off < seg_bytes;
-        float acc[BT][E];
+        if (warp == GV_CONSUMER_WARPS) {
+            // ---- 3. producer warp: its lanes copy the rows of each stage ----
+            for (int i = 0; i < n_stages && !failed; ++i) {
+                const int it = it_base + i;
+                const int st = it % GV_STAGES;
+                if (it >= GV_STAGES) {
+                    if (!mbar_wait(&s.empty[st], ((it / GV_STAGES) - 1) & 1)) failed = true;
+                }
+                failed = __any_sync(0xffffffffu, failed) || s.abort;
+                if (failed) break;
+                const int rows_here = min(R, n_rows - i * R);
+                if (lane == 0) mbar_expect_tx(&s.full[st], (unsigned)(rows_here * seg_bytes));
+                __syncwarp();
+                for (int r = lane; r < rows_here; r += 32) {
+                    const int idx = s.idx[i * R + r];
+                    bulk_g2s(&s.ring[st][r * SEG], p.W + (size_t)idx * p.row_bytes + seg_off, (unsigned)seg_bytes,
+                             &s.full[st]);
+                }
+                if (lane == 0) s.issued = it + 1;
+            }
+            if (failed && lane == 0) {
+                s.abort = 1;
+                atomicExch(p.status, 1);
+            }
+        } else {
+            // ---- 4. consumers ----
+            // the tokens' values for the kept rows (zero where a token's own mask drops the row)
+            for (int r = tid; r < n_rows; r += GV_CONSUMER_WARPS * 32) {
+                const int idx = s.idx[r];
 #pragma unroll
-        for (int b = 0; b < BT; ++b)
-#pragma unroll
-            for (int e = 0; e < E; ++e) acc[b][e] = 0.f;
+                for (int b = 0; b < BT; ++b) {
+                    float val = 0.f;
+                    // one token: every listed row is its own; several: ask the token's mask
+                    if (b < p.batch && (p.batch == 1 ||
+                        ((p.mask_bits[(size_t)b * p.mask_words + (idx >> 5)] >> (idx & 31)) & 1u)))
+                        val = p.v[(size_t)b * p.d_in + idx];
+                    s_v[b * GV_MAX_ROWS + r] = val;
+                }
+            }
+            asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
 
-        for (int it = 0; it < n_stages; ++it) {
-            const int st = it % GV_STAGES;
-            if (!mbar_wait(&s.full[st], (it / GV_STAGES) & 1)) failed = true;
-            if (failed || s.abort) { failed = true; break; }
-            const int rows_here = min(GV_STAGE_ROWS, n_rows - it * GV_STAGE_ROWS);
-            if (lane_ok) {
+            for (int i = 0; i < n_stages; ++i) {
+                const int it = it_base + i;
+                const int st = it % GV_STAGES;
+                if (!mbar_wait(&s.full[st], (it / GV_STAGES) & 1)) failed = true;
+                if (failed || s.abort) { failed = true; break; }
+                const int rows_here = min(R, n_rows - i * R);
+                if (lane_ok) {
 #pragma unroll
-                for (int rr = 0; rr < GV_STAGE_ROWS / 2; ++rr) {
-                    const int r = 2 * rr + rg;
-                    if (r < rows_here) {
-                        const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r][byte_off]);
-                        float w[E];
-                        decode16<WT>(raw, w);
+                    for (int rr = 0; rr < R / RG; ++rr) {
+                        const int r = rr * RG + rg;
+                        if (r < rows_here) {
+                            const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * SEG + byte_off]);
+                            float w[E];
+                            decode16<WT>(raw, w);
 #pragma unroll
-                        for (int b = 0; b < BT; ++b) {
-                            const float xv = s_v[b * GV_MAX_ROWS + it * GV_STAGE_ROWS + r];
+                            for (int b = 0; b < BT; ++b) {
+                                const float xv = s_v[b * GV_MAX_ROWS + i * R + r];
 #pragma unroll
-                            for (int e = 0; e < E; ++e) acc[b][e] = fmaf(w[e], xv, acc[b][e]);
+                                for (int e = 0; e < E; ++e) acc[b][e] = fmaf(w[e], xv, acc[b][e]);
+                            }
                         }
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s.empty[st]);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s.empty[st]);
+            if (failed) {
+                s.abort = 1;
+                if (lane == 0) atomicExch(p.status, 1);
+            }
         }
+        it_base += n_stages;
+    }
 
-        if (failed) {
-            s.abort = 1;
-            if (lane == 0) atomicExch(p.status, 1);
-        }
-        // combine the two row groups: group 1 parks its sums in the (now idle) ring
-        float *red = reinterpret_cast<float *>(&s.ring[0][0][0]);    // [4 cw][32 lanes][BT][E]
-        asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
-        if (rg == 1) {
+    // ---- 5. combine the row groups through the (now idle) ring, in group order ----
+    __syncthreads();
+    float *red = reinterpret_cast<float *>(&s.ring[0][0]);    // [RG-1][CG*32 lanes][BT][E]
+    float *own = reinterpret_cast<float *>(&s.ring[GV_STAGES - 1][0]);   // [BT][SLAB] sums of this CTA
+    if (warp < GV_CONSUMER_WARPS && rg > 0) {
 #pragma unroll
-            for (int b = 0; b < BT; ++b)
+        for (int b = 0; b < BT; ++b)
 #pragma unroll
-                for (int e = 0; e < E; ++e) red[((cw * 32 + lane) * BT + b) * E + e] = acc[b][e];
-        }
-        asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
-        if (rg == 0) {
-            float *dst = nparts > 1 ? p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB)
-                                    : reinterpret_cast<float *>(&s.ring[1][0][0]);
+            for (int e = 0; e < E; ++e)
+                red[((((rg - 1) * CG + cw) * 32 + lane) * BT + b) * E + e] = acc[b][e];
+    }
+    __syncthreads();
+    if (warp < GV_CONSUMER_WARPS && rg == 0) {
+        float *dst = nparts > 1 ? p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB) : own;
 #pragma unroll
-            for (int b = 0; b < BT; ++b) {
-                float sum[E];
+        for (int b = 0; b < BT; ++b) {
+            float sum[E];
 #pragma unroll
-                for (int e = 0; e < E; ++e) sum[e] = acc[b][e] + red[((cw * 32 + lane) * BT + b) * E + e];
-                float *d = dst + b * SLAB + (cw * 512 + lane * 16) / EB;
+            for (int e = 0; e < E; ++e) sum[e] = acc[b][e];
 #pragma unroll
-                for (int e = 0; e < E; e += 4)
-                    *reinterpret_cast<float4 *>(d + e) = make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
-            }
+            for (int g = 1; g < RG; ++g)
+#pragma unroll
+                for (int e = 0; e < E; ++e) sum[e] += red[((((g - 1) * CG + cw) * 32 + lane) * BT + b) * E + e];
+            float *d = dst + b * SLAB + (cw * 512 + lane * 16) / EB;
+#pragma unroll
+            for (int e = 0; e < E; e += 4)
+                *reinterpret_cast<float4 *>(d + e) = make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
         }
     }
 
-    // ---- 4. combine the parts ----
+    // ---- 6. combine the parts ----
     if (nparts > 1) {
         __threadfence();
         __syncthreads();
@@ -330,7 +370,6 @@ gemv_kernel(const GemvParams p)
         }
         return;
     }
-    const float *own = reinterpret_cast<const float *>(&s.ring[1][0][0]);
     for (int t = tid; t < BT * OUT_PER_SLAB; t += GV_THREADS) {
         const int b = t / OUT_PER_SLAB, o = t % OUT_PER_SLAB;
         const int j = slab * OUT_PER_SLAB + o;
@@ -344,10 +383,21 @@ gemv_kernel(const GemvParams p)
         }
         float s0 = 0.f, s1 = 0.f;
         if (nparts > 1) {
-            for (int q = 0; q < nparts; ++q) {
-                const float *pp = p.partials + ((size_t)q * gridDim.x + slab) * (BT * SLAB) + b * SLAB;
-                s0 += __ldcg(pp + e0);
-                if (WHICH == 0) s1 += __ldcg(pp + e1);
+            // parts in part order; eight loads in flight at a time
+            const size_t stride = (size_t)gridDim.x * (BT * SLAB);
+            const float *pp = p.partials + (size_t)slab * (BT * SLAB) + b * SLAB;
+            for (int q0 = 0; q0 < nparts; q0 += 8) {
+                float a0[8], a1[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    a0[q] = q0 + q < nparts ? __ldcg(pp + (size_t)(q0 + q) * stride + e0) : 0.f;
+                    a1[q] = (WHICH == 0 && q0 + q < nparts) ? __ldcg(pp + (size_t)(q0 + q) * stride + e1) : 0.f;
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    s0 += a0[q];
+                    s1 += a1[q];
+                }
             }
         } else {
             s0 = own[b * SLAB + e0];
@@ -371,31 +421,51 @@ __global__ void idx_to_mask_kernel(const int32_t *__restrict__ idx, int n, int d
     }
 }
 
-template <int WT, int WHICH, int BT>
-dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t stream)
+template <int WT, int WHICH, int BT, int SEG>
+dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cudaStream_t stream)
 {
-    constexpr int SLAB = GV_SEG_BYTES / WTraits<WT>::EB;
-    const int n_slabs = (int)((p.row_bytes + GV_SEG_BYTES - 1) / GV_SEG_BYTES);
-    if (n_slabs > ctx->n_tickets) return DIP_ERR_WORKSPACE;
-    // one CTA per SM, all resident at once; parts no longer than the in-kernel row list
-    int nparts = ctx->sm_count / n_slabs;
-    const int min_parts = (n_kept_max + GV_MAX_ROWS - 1) / GV_MAX_ROWS;
-    if (nparts < min_parts) nparts = min_parts;
-    if (nparts > n_kept_max) nparts = n_kept_max;
-    if (nparts < 1) nparts = 1;
+    constexpr int SLAB = SEG / WTraits<WT>::EB;
     const size_t per_part = (size_t)n_slabs * BT * SLAB;
-    if ((size_t)nparts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
-    const size_t smem = sizeof(GemvSmem) + (size_t)BT * GV_MAX_ROWS * sizeof(float);
-    static bool attr_set = false;   // per (WT, WHICH, BT) instantiation
+    if (nparts > 1 && (size_t)nparts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
+    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * GV_MAX_ROWS * sizeof(float);
+    static bool attr_set = false;   // per instantiation
     if (!attr_set) {
-        DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(gemv_kernel<WT, WHICH, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)smem));
+        DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(gemv_kernel<WT, WHICH, BT, SEG>,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr_set = true;
     }
     dim3 grid(n_slabs, nparts);
-    gemv_kernel<WT, WHICH, BT><<<grid, GV_THREADS, smem, stream>>>(p);
-    DIP_CUDA_TRY(ctx, cudaGetLastError());
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(gemv_kernel<WT, WHICH, BT, SEG>, grid, dim3(GV_THREADS), smem, stream, p));
     return DIP_OK;
+}
+
+// Segment width and number of row parts: one CTA per SM, all resident at once.  A wide
+// segment is kinder to DRAM, but few slabs mean many parts, and the CTA that finishes a slab
+// then has nparts * SEG bytes of partial sums to add up alone; narrow the segment until that
+// tail is short (or until no split is needed at all).
+template <int WT, int WHICH, int BT>
+dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t stream)
+{
+    int seg = ctx->gemv_seg;
+    int n_slabs = 0, nparts = 1;
+    const int cands[3] = {2048, 1024, 512};
+    for (int c = 0; c < 3; ++c) {
+        const int sg = seg ? seg : cands[c];
+        n_slabs = (int)((p.row_bytes + sg - 1) / sg);
+        nparts = ctx->sm_count / n_slabs;
+        if (nparts > n_kept_max) nparts = n_kept_max;
+        if (nparts < 1) nparts = 1;
+        if (seg || (long long)nparts * sg <= 20480 || sg == 512) {
+            seg = sg;
+            break;
+        }
+    }
+    if (n_slabs > ctx->n_tickets) return DIP_ERR_WORKSPACE;
+    switch (seg) {
+    case 2048: return launch_seg<WT, WHICH, BT, 2048>(ctx, p, n_slabs, nparts, stream);
+    case 1024: return launch_seg<WT, WHICH, BT, 1024>(ctx, p, n_slabs, nparts, stream);
+    default: return launch_seg<WT, WHICH, BT, 512>(ctx, p, n_slabs, nparts, stream);
+    }
 }
 
 template <int WT, int WHICH>

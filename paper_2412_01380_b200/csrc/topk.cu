@@ -26,7 +26,11 @@ struct TkShared {
     int wc[TK_WARPS];
     float wf[TK_WARPS];
     float scale;
+    int n_cand, n_cand2;
+    uint32_t last_key[32];
+    int last_idx[32];
 };
+constexpr int TK_CAND_CAP = 2048;   // candidates of the threshold bin kept for the refinement passes
 
 __device__ __forceinline__ unsigned lanemask_lt()
 {
@@ -48,6 +52,46 @@ __device__ __forceinline__ int warp_array_prefix(const int *arr, int warp, int l
     total = __shfl_sync(0xffffffffu, incl, 31);
     int excl = incl - v;
     return __shfl_sync(0xffffffffu, excl, warp);
+}
+
+// Find the histogram bin holding the krem-th largest key: suffix scan over the RADIX_BINS bins,
+// two per thread.  Leaves bcast[0] = bin, bcast[1] = rank of the wanted key inside the bin
+// (1-based, from the top), bcast[2] = keys in the bin.  All threads call it; ends with a barrier.
+__device__ __forceinline__ void find_bin(TkShared &s, int krem)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // suffix scan: thread t owns bins 2t and 2t+1
+    const unsigned h0 = s.hist[2 * tid], h1 = s.hist[2 * tid + 1];
+    const int own = (int)(h0 + h1);
+    int suf = own;   // inclusive suffix within the warp
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += n;
+    }
+    if (lane == 0) s.wa[warp] = suf;
+    __syncthreads();
+    int wv = s.wa[lane];
+    int wsuf = wv;   // inclusive suffix over warps
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_down_sync(0xffffffffu, wsuf, o);
+        if (lane + o < 32) wsuf += n;
+    }
+    const int above_warp = __shfl_sync(0xffffffffu, wsuf - wv, warp);
+    int cum = above_warp + suf - own;         // keys in bins above 2t+1
+    if (cum < krem && krem <= cum + (int)h1) {
+        s.bcast[0] = 2 * tid + 1;
+        s.bcast[1] = krem - cum;
+        s.bcast[2] = (int)h1;
+    }
+    cum += (int)h1;
+    if (cum < krem && krem <= cum + (int)h0) {
+        s.bcast[0] = 2 * tid;
+        s.bcast[1] = krem - cum;
+        s.bcast[2] = (int)h0;
+    }
+    __syncthreads();
 }
 
 // k-th largest of (keys[e] & keymask), e in [0, d).  All threads of the CTA take part and get
@@ -97,38 +141,7 @@ __device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask
             if (c3) atomicAdd(&s.hist[3], (unsigned)c3);
         }
         __syncthreads();
-        // suffix scan: thread t owns bins 2t and 2t+1
-        const unsigned h0 = s.hist[2 * tid], h1 = s.hist[2 * tid + 1];
-        const int own = (int)(h0 + h1);
-        int suf = own;   // inclusive suffix within the warp
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int n = __shfl_down_sync(0xffffffffu, suf, o);
-            if (lane + o < 32) suf += n;
-        }
-        if (lane == 0) s.wa[warp] = suf;
-        __syncthreads();
-        int wv = s.wa[lane];
-        int wsuf = wv;   // inclusive suffix over warps
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int n = __shfl_down_sync(0xffffffffu, wsuf, o);
-            if (lane + o < 32) wsuf += n;
-        }
-        const int above_warp = __shfl_sync(0xffffffffu, wsuf - wv, warp);
-        int cum = above_warp + suf - own;             // keys in bins above 2t+1
-        if (cum < krem && krem <= cum + (int)h1) {
-            s.bcast[0] = 2 * tid + 1;
-            s.bcast[1] = krem - cum;
-            s.bcast[2] = (int)h1;
-        }
-        cum += (int)h1;
-        if (cum < krem && krem <= cum + (int)h0) {
-            s.bcast[0] = 2 * tid;
-            s.bcast[1] = krem - cum;
-            s.bcast[2] = (int)h0;
-        }
-        __syncthreads();
+        find_bin(s, krem);
         prefix |= (uint32_t)s.bcast[0] << shift;
         prefmask |= dmask << shift;
         krem = s.bcast[1];
@@ -157,6 +170,9 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
 {
     extern __shared__ uint32_t keys[];
     __shared__ TkShared s;
+    __shared__ uint32_t cand_key[TK_CAND_CAP];
+    __shared__ int cand_idx[TK_CAND_CAP];
+    __shared__ unsigned int s_maskw[DIP_MAX_D / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x;
     const int n_words = (d + 31) >> 5;
@@ -166,6 +182,15 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
         x_out += (size_t)row * d;
     }
     mask_bits += (size_t)row * n_words;
+
+    s.hist[2 * tid] = 0;
+    s.hist[2 * tid + 1] = 0;
+    if (tid == 0) {
+        s.n_cand = 0;
+        s.n_cand2 = 0;
+    }
+    dip_grid_dependency_wait();        // the inputs come from the previous kernel in the stream
+    dip_launch_dependents();
 
     if (NORM) {
         float ss = 0.f;
@@ -187,8 +212,9 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
                 s.scale = rms > 0.f ? 1.0f / rms : 1.0f;
             }
         }
-        __syncthreads();
     }
+    __syncthreads();
+    // rank keys, and the histogram of their top 11 bits (first radix pass) in the same sweep
     for (int e = tid; e < d; e += TK_THREADS) {
         float v;
         if (NORM) {
@@ -199,17 +225,82 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
         }
         float a = fabsf(v);
         if (CA) a = __fmul_rn(a, stamp[e] >= 0 ? 1.0f : gamma);
-        keys[e] = __float_as_uint(a) & 0x7fffffffu;
+        const uint32_t key = __float_as_uint(a) & 0x7fffffffu;
+        keys[e] = key;
+        atomicAdd(&s.hist[key >> 20], 1u);
     }
     __syncthreads();
-
-    uint32_t T;
-    int quota, n_eq;
-    block_radix_select(keys, d, 0x7fffffffu, 31, k, s, T, quota, n_eq);
+    find_bin(s, k);
+    const uint32_t b1 = (uint32_t)s.bcast[0];
+    const int krem1 = s.bcast[1], cnt1 = s.bcast[2];
 
     // warp w owns columns [w*span, (w+1)*span), span a multiple of 32: one ballot = one mask word
     const int span = ((d + TK_THREADS - 1) / TK_THREADS) * 32;
     const int base = warp * span;
+
+    bool fast = cnt1 <= TK_CAND_CAP;
+    if (fast) {
+        // Every key in a bin above b1 is kept, every key below is dropped; the krem1 largest of the
+        // cnt1 keys in bin b1 (lower index first among equals) complete the mask.  One sweep
+        // writes the certain bits and collects the bin's keys with their columns.
+        s.hist[2 * tid] = 0;          // free again: refilled below with the candidates' next digit
+        s.hist[2 * tid + 1] = 0;
+        for (int it = 0; it < span && base + it < d; it += 32) {
+            const int e = base + it + lane;
+            const uint32_t key = e < d ? keys[e] : 0u;
+            const uint32_t dg = key >> 20;
+            const unsigned bk = __ballot_sync(0xffffffffu, e < d && dg > b1);
+            if (lane == 0) s_maskw[(base + it) >> 5] = bk;
+            if (e < d && dg == b1) {
+                const int pos = atomicAdd(&s.n_cand, 1);
+                cand_key[pos] = key & 0xfffffu;
+                cand_idx[pos] = e;
+            }
+        }
+        __syncthreads();
+        // second digit (bits 19..9) of the candidates
+        for (int c = tid; c < cnt1; c += TK_THREADS) atomicAdd(&s.hist[cand_key[c] >> 9], 1u);
+        __syncthreads();
+        find_bin(s, krem1);
+        const uint32_t b2 = (uint32_t)s.bcast[0];
+        const int krem2 = s.bcast[1], cnt2 = s.bcast[2];
+        fast = cnt2 <= 32;
+        if (fast) {
+            for (int c = tid; c < cnt1; c += TK_THREADS) {
+                const uint32_t dg = cand_key[c] >> 9;
+                if (dg > b2) {
+                    atomicOr(&s_maskw[cand_idx[c] >> 5], 1u << (cand_idx[c] & 31));
+                } else if (dg == b2) {
+                    const int pos = atomicAdd(&s.n_cand2, 1);
+                    s.last_key[pos] = cand_key[c] & 0x1ffu;
+                    s.last_idx[pos] = cand_idx[c];
+                }
+            }
+            __syncthreads();
+            if (warp == 0) {
+                // at most 32 keys share the threshold's top 22 bits: rank them by (key descending,
+                // column ascending) and keep the first krem2
+                const uint32_t kv = lane < cnt2 ? s.last_key[lane] : 0u;
+                const int iv = lane < cnt2 ? s.last_idx[lane] : 0x7fffffff;
+                int rank = 0;
+                for (int j = 0; j < cnt2; ++j) {
+                    const uint32_t kj = __shfl_sync(0xffffffffu, kv, j);
+                    const int ij = __shfl_sync(0xffffffffu, iv, j);
+                    rank += (kj > kv) || (kj == kv && ij < iv);
+                }
+                if (lane < cnt2 && rank < krem2) atomicOr(&s_maskw[iv >> 5], 1u << (iv & 31));
+            }
+            __syncthreads();
+            for (int w = tid; w < n_words; w += TK_THREADS) mask_bits[w] = s_maskw[w];
+            return;
+        }
+    }
+
+    // General path (very many keys tied around the threshold): full radix select on all keys,
+    // then an ordered sweep that ranks the ties by column.
+    uint32_t T;
+    int quota, n_eq;
+    block_radix_select(keys, d, 0x7fffffffu, 31, k, s, T, quota, n_eq);
     if (quota == n_eq) {
         // every column tied with the threshold is kept: the mask is key >= T
         for (int it = 0; it < span && base + it < d; it += 32) {
@@ -427,18 +518,23 @@ dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, flo
                              float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream)
 {
     const size_t smem = (size_t)d * sizeof(uint32_t);
+    const dim3 grid(batch), block(TK_THREADS);
+    cudaError_t e;
     if (xb) {
         if (stamp)
-            select_kernel<true, true><<<batch, TK_THREADS, smem, stream>>>(xa, xb, x_out, d, k, gamma, stamp, mask_bits);
+            e = dip_launch_pdl(select_kernel<true, true>, grid, block, smem, stream, xa, xb, x_out, d, k, gamma, stamp, mask_bits);
         else
-            select_kernel<false, true><<<batch, TK_THREADS, smem, stream>>>(xa, xb, x_out, d, k, 1.0f, nullptr, mask_bits);
+            e = dip_launch_pdl(select_kernel<false, true>, grid, block, smem, stream, xa, xb, x_out, d, k, 1.0f,
+                               (const int32_t *)nullptr, mask_bits);
     } else {
         if (stamp)
-            select_kernel<true, false><<<batch, TK_THREADS, smem, stream>>>(xa, nullptr, nullptr, d, k, gamma, stamp, mask_bits);
+            e = dip_launch_pdl(select_kernel<true, false>, grid, block, smem, stream, xa, (const float *)nullptr,
+                               (float *)nullptr, d, k, gamma, stamp, mask_bits);
         else
-            select_kernel<false, false><<<batch, TK_THREADS, smem, stream>>>(xa, nullptr, nullptr, d, k, 1.0f, nullptr, mask_bits);
+            e = dip_launch_pdl(select_kernel<false, false>, grid, block, smem, stream, xa, (const float *)nullptr,
+                               (float *)nullptr, d, k, 1.0f, (const int32_t *)nullptr, mask_bits);
     }
-    DIP_CUDA_TRY(ctx, cudaGetLastError());
+    DIP_CUDA_TRY(ctx, e);
     return DIP_OK;
 }
 
