@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging; not a valid bench)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--timeline", action="store_true",
+                    help="print the device-side timeline of one graph replay (per kernel: start, ready, end) and exit")
     return ap.parse_args()
 
 
@@ -289,6 +291,45 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
     return res
 
 
+def print_timeline(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget):
+    """One decode token through the stack as a CUDA graph, with the library's device-side
+    timeline on: per kernel, when it started, when its inputs were ready, when it ended."""
+    L, d_model, d_ff = len(layers), w.d_model, w.d_ff
+    k_x, k_h = di.keep_count(keep_ratio, d_model), di.keep_count(keep_ratio, d_ff)
+    ca = budget is not None
+    gamma = w.gamma if ca else 1.0
+    if ca:
+        stack = dip.Stack(layers, [dip.CacheState(d_model, di.cache_capacity(budget, d_model), "cuda") for _ in range(L)],
+                          [dip.CacheState(d_ff, di.cache_capacity(budget, d_ff), "cuda") for _ in range(L)])
+    else:
+        stack = dip.Stack(layers)
+    xs = xs_host.cuda()
+    x_cur, x_out = torch.empty(d_model, device="cuda"), torch.empty(d_model, device="cuda")
+    x_cur.copy_(xs[0])
+    dip.dip_stack_step(ctx, stack, x_cur, k_x, k_h, gamma, x_out)
+    torch.cuda.synchronize()
+    ctx.trace_begin()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        dip.dip_stack_step(ctx, stack, x_cur, k_x, k_h, gamma, x_out)
+    for t in range(6):
+        x_cur.copy_(xs[t % xs.shape[0]])
+        g.replay()
+    torch.cuda.synchronize()
+    ctx.trace_reset()
+    x_cur.copy_(xs[6 % xs.shape[0]])
+    g.replay()
+    recs = ctx.trace_read()
+    ctx.trace_end()
+    print("# %s keep_ratio %g cache_budget %s: one graph replay of %d layers; times in us" % (w.name, keep_ratio, budget, L))
+    print("%-14s %9s %9s %9s %9s %9s" % ("kernel", "start", "ready", "stream", "end", "end-ready"))
+    for r in recs:
+        print("%-14s %9.2f %9.2f %9s %9.2f %9.2f" % (r["kind"], r["start"], r["ready"],
+              "%.2f" % r["aux"] if r["aux"] is not None else "-", r["end"], r["end"] - r["ready"]))
+    main_path = [r for r in recs if r["kind"] != "cache_update"]
+    print("# critical path per layer: %.2f us" % ((main_path[-1]["end"] - main_path[0]["ready"]) / L))
+
+
 def oracle_rate(w, keep_ratio, budget, n_layers_sample, n_steps, warmup=0):
     """The CPU oracle as it stands, timed on this machine's host cores on a bounded sample of the
     workload: `n_steps` MLP-steps cycling over `n_layers_sample` host-generated layers."""
@@ -369,6 +410,9 @@ def main():
     wl_rank = w.scaled(seed=w.seed + 1000 * rank)
     xs_host = torch.from_numpy(di.token_inputs(wl_rank, n_tokens=n_tok, batch=1)[:, 0].copy())
 
+    if args.timeline:
+        print_timeline(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget)
+        return
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
                            else int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])) if rank == 0 else None
     head = run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, args.steps, args.warmup,

@@ -88,6 +88,29 @@ int dip_sm_count(const dip_ctx *ctx);
 dip_status dip_device_status(dip_ctx *ctx, int *status_out, void *stream);
 
 /* ------------------------------------------------------------------------
+ * Timeline of the library's own kernels (diagnostics; off by default).  Between
+ * dip_trace_begin and dip_trace_end every kernel the context launches (up to
+ * 1024 launches) gets a slot in which it stamps, with the device's nanosecond
+ * timer: the first CTA's entry, the first return from the wait on the previous
+ * kernel in the stream, the last CTA's exit and, for the GEMVs, the end of the
+ * weight streaming.  A CUDA graph captured while tracing is on keeps its slots:
+ * dip_trace_reset clears the stamps (not the slots) before a replay, and
+ * dip_trace_read returns the records of the launches that ran since.  These
+ * calls synchronise the device; the stamps cost one atomic per CTA.
+ *   kind: 1 select (DIP), 2 select (cache-aware), 3 cache update, 4 gate/up GEMV,
+ *         5 down GEMV.
+ * ------------------------------------------------------------------------ */
+typedef struct {
+    int32_t kind;
+    int32_t reserved;
+    uint64_t t_start_ns, t_ready_ns, t_end_ns, t_aux_ns;
+} dip_trace_record;
+dip_status dip_trace_begin(dip_ctx *ctx);
+dip_status dip_trace_reset(dip_ctx *ctx);
+dip_status dip_trace_read(dip_ctx *ctx, dip_trace_record *out /* host */, int max_records, int *n_out /* host */);
+dip_status dip_trace_end(dip_ctx *ctx);
+
+/* ------------------------------------------------------------------------
  * Weights.  The paper's unit of selection is a column W[:, i] of a matrix
  * W in R^{d_out x d_in} (Eq. 4, 7, 8), so the library stores each matrix
  * column-contiguous: row i of the packed array holds column i.  Gate and up

@@ -80,10 +80,23 @@ _lib.dip_sparse_gemv_down_noalloc.restype = _i32
 _lib.dip_sparse_gemv_down_noalloc.argtypes = [C.POINTER(MlpWeightsStruct), _vp, _vp, _i32, _vp, _vp]
 
 EXPORTED = ["dip_create", "dip_destroy", "dip_status_string", "dip_last_error", "dip_sm_count",
-            "dip_device_status",
+            "dip_device_status", "dip_trace_begin", "dip_trace_reset", "dip_trace_read", "dip_trace_end",
             "dip_packed_bytes", "dip_pack_weights", "dip_mask_topk", "dip_ca_mask",
             "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_mlp_step",
             "dip_residual_rmsnorm", "dip_stack_step", "dip_sparse_gemv_down_noalloc"]
+
+
+class TraceRecord(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("reserved", C.c_int32), ("t_start_ns", C.c_uint64),
+                ("t_ready_ns", C.c_uint64), ("t_end_ns", C.c_uint64), ("t_aux_ns", C.c_uint64)]
+
+
+TRACE_KINDS = {1: "select", 2: "select_ca", 3: "cache_update", 4: "gemv_gate_up", 5: "gemv_down"}
+for _name in ("dip_trace_begin", "dip_trace_reset", "dip_trace_end"):
+    getattr(_lib, _name).restype = _i32
+    getattr(_lib, _name).argtypes = [_vp]
+_lib.dip_trace_read.restype = _i32
+_lib.dip_trace_read.argtypes = [_vp, C.POINTER(TraceRecord), _i32, C.POINTER(C.c_int)]
 
 
 class DipError(RuntimeError):
@@ -127,6 +140,29 @@ class Context:
         out = C.c_int(-1)
         self.check(_lib.dip_device_status(self.handle, C.byref(out), _stream()))
         return out.value
+
+    def trace_begin(self) -> None:
+        self.check(_lib.dip_trace_begin(self.handle))
+
+    def trace_reset(self) -> None:
+        self.check(_lib.dip_trace_reset(self.handle))
+
+    def trace_end(self) -> None:
+        self.check(_lib.dip_trace_end(self.handle))
+
+    def trace_read(self):
+        """Records of the launches that ran since the last reset: list of dicts with times in
+        microseconds relative to the earliest start."""
+        buf = (TraceRecord * 1024)()
+        n = C.c_int(0)
+        self.check(_lib.dip_trace_read(self.handle, buf, 1024, C.byref(n)))
+        recs = [buf[i] for i in range(n.value)]
+        if not recs:
+            return []
+        t0 = min(r.t_start_ns for r in recs)
+        return [{"kind": TRACE_KINDS.get(r.kind, str(r.kind)), "start": (r.t_start_ns - t0) / 1e3,
+                 "ready": (r.t_ready_ns - t0) / 1e3, "end": (r.t_end_ns - t0) / 1e3,
+                 "aux": (r.t_aux_ns - t0) / 1e3 if r.t_aux_ns else None} for r in recs]
 
     def close(self) -> None:
         if self.handle:

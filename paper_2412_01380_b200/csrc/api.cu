@@ -104,6 +104,7 @@ dip_status dip_create(dip_ctx **out, int device)
     if ((st = dev_alloc(ctx, &ctx->mask_tmp, (size_t)(DIP_MAX_D / 32))) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->status, (size_t)1)) != DIP_OK) return fail(st);
     if (cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
+    if ((st = dev_alloc(ctx, &ctx->trace, (size_t)DIP_TRACE_SLOTS * DIP_TRACE_WORDS)) != DIP_OK) return fail(st);
     for (int i = 0; i < 2; ++i) {
         if (cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking) != cudaSuccess) return fail(DIP_ERR_CUDA);
         if (cudaEventCreateWithFlags(&ctx->ev_fork[i], cudaEventDisableTiming) != cudaSuccess) return fail(DIP_ERR_CUDA);
@@ -135,6 +136,7 @@ dip_status dip_destroy(dip_ctx *ctx)
     cudaFree(ctx->mask_ring);
     cudaFree(ctx->mask_tmp);
     cudaFree(ctx->status);
+    cudaFree(ctx->trace);
     for (int i = 0; i < 2; ++i) {
         if (ctx->side[i]) cudaStreamDestroy(ctx->side[i]);
         if (ctx->ev_fork[i]) cudaEventDestroy(ctx->ev_fork[i]);
@@ -373,6 +375,63 @@ dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *lay
     dip_status st = dip_residual_rmsnorm(ctx, x_prev, y_prev, batch, d, x_out, stream);
     if (st != DIP_OK) return st;
     return join_cache_updates(ctx, (cudaStream_t)stream);
+}
+
+// ---- device-side timeline (diagnostics) ----
+static dip_status trace_clear(dip_ctx *ctx)
+{
+    static unsigned long long init[DIP_TRACE_SLOTS * DIP_TRACE_WORDS];
+    for (int i = 0; i < DIP_TRACE_SLOTS; ++i) {
+        init[DIP_TRACE_WORDS * i + 0] = ~0ull;
+        init[DIP_TRACE_WORDS * i + 1] = ~0ull;
+        init[DIP_TRACE_WORDS * i + 2] = 0;
+        init[DIP_TRACE_WORDS * i + 3] = 0;
+    }
+    DIP_CUDA_TRY(ctx, cudaDeviceSynchronize());
+    DIP_CUDA_TRY(ctx, cudaMemcpy(ctx->trace, init, sizeof(init), cudaMemcpyHostToDevice));
+    return DIP_OK;
+}
+
+dip_status dip_trace_begin(dip_ctx *ctx)
+{
+    if (!ctx) return DIP_ERR_INVALID_ARG;
+    ctx->trace_on = 1;
+    ctx->trace_next = 0;
+    return trace_clear(ctx);
+}
+
+dip_status dip_trace_reset(dip_ctx *ctx)
+{
+    if (!ctx) return DIP_ERR_INVALID_ARG;
+    return trace_clear(ctx);
+}
+
+dip_status dip_trace_read(dip_ctx *ctx, dip_trace_record *out, int max_records, int *n_out)
+{
+    if (!ctx || !out || !n_out || max_records < 0) return DIP_ERR_INVALID_ARG;
+    static unsigned long long host[DIP_TRACE_SLOTS * DIP_TRACE_WORDS];
+    DIP_CUDA_TRY(ctx, cudaDeviceSynchronize());
+    DIP_CUDA_TRY(ctx, cudaMemcpy(host, ctx->trace, sizeof(host), cudaMemcpyDeviceToHost));
+    int n = 0;
+    for (int i = 0; i < ctx->trace_next && n < max_records; ++i) {
+        const unsigned long long *w = host + (size_t)DIP_TRACE_WORDS * i;
+        if (w[0] == ~0ull) continue;               // that launch has not run since the last reset
+        out[n].kind = ctx->trace_kind[i];
+        out[n].t_start_ns = w[0];
+        out[n].t_ready_ns = w[1];
+        out[n].t_end_ns = w[2];
+        out[n].t_aux_ns = w[3];
+        ++n;
+    }
+    *n_out = n;
+    return DIP_OK;
+}
+
+dip_status dip_trace_end(dip_ctx *ctx)
+{
+    if (!ctx) return DIP_ERR_INVALID_ARG;
+    ctx->trace_on = 0;
+    return DIP_OK;
 }
 
 }  // extern "C"

@@ -7,6 +7,10 @@
 
 #include "dip.h"
 
+constexpr int DIP_RING_LAYERS = 128;
+constexpr int DIP_TRACE_SLOTS = 1024;
+constexpr int DIP_TRACE_WORDS = 4;   // first start, dependency ready, last end, auxiliary
+
 // Scratch workspace of a context.  All device memory the library itself owns.
 struct dip_ctx {
     int device;
@@ -37,10 +41,22 @@ struct dip_ctx {
     cudaStream_t side[2];
     cudaEvent_t ev_fork[2], ev_join[2];
     bool side_busy[2];
+    // device-side timeline (diagnostics): one slot of DIP_TRACE_WORDS words per launch
+    unsigned long long *trace;
+    int trace_on;
+    int trace_next;
+    unsigned char trace_kind[DIP_TRACE_SLOTS];
     char err[256];
 };
 
-constexpr int DIP_RING_LAYERS = 128;
+// Slot of the next launch, or nullptr when tracing is off.
+static inline unsigned long long *dip_trace_slot(dip_ctx *ctx, int kind)
+{
+    if (!ctx->trace_on || ctx->trace_next >= DIP_TRACE_SLOTS) return nullptr;
+    ctx->trace_kind[ctx->trace_next] = (unsigned char)kind;
+    return ctx->trace + (size_t)DIP_TRACE_WORDS * ctx->trace_next++;
+}
+
 
 #define DIP_CUDA_TRY(ctx, call)                                                        \
     do {                                                                               \
@@ -53,6 +69,18 @@ constexpr int DIP_RING_LAYERS = 128;
     } while (0)
 
 #ifdef __CUDACC__
+// Timeline stamps (nanoseconds of %globaltimer) taken by thread 0 of each CTA when tr != nullptr:
+// word 0 = earliest kernel entry, 1 = earliest return from the dependency wait, 2 = latest exit,
+// 3 = latest auxiliary mark.
+__device__ __forceinline__ unsigned long long dip_gtime()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define DIP_TRACE_MIN(tr, i) do { if ((tr) && threadIdx.x == 0) atomicMin(&(tr)[i], dip_gtime()); } while (0)
+#define DIP_TRACE_MAX(tr, i) do { if ((tr) && threadIdx.x == 0) atomicMax(&(tr)[i], dip_gtime()); } while (0)
+
 // Programmatic dependent launch: a kernel may be scheduled before its predecessor in the stream
 // has finished; it must not touch the predecessor's results before this wait returns.
 __device__ __forceinline__ void dip_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -40,6 +40,7 @@ struct GemvParams {
     float *partials;
     unsigned int *tickets;
     int *status;               // device status word (0 = fine)
+    unsigned long long *tr;    // timeline slot or nullptr
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -138,6 +139,7 @@ gemv_kernel(const GemvParams p)
     GemvSmem<SEG> &s = *reinterpret_cast<GemvSmem<SEG> *>(smem_raw);
     float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem<SEG>));   // [BT][GV_MAX_ROWS]
 
+    DIP_TRACE_MIN(p.tr, 0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slab = blockIdx.x, part = blockIdx.y, nparts = gridDim.y;
     const size_t seg_off = (size_t)slab * SEG;
@@ -153,6 +155,7 @@ gemv_kernel(const GemvParams p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     dip_grid_dependency_wait();        // the mask and the vector come from the previous kernels
+    DIP_TRACE_MIN(p.tr, 1);
     dip_launch_dependents();
 
     // ---- 1. the mask words and their popcount prefix ----
@@ -319,6 +322,7 @@ gemv_kernel(const GemvParams p)
         it_base += n_stages;
     }
 
+    DIP_TRACE_MAX(p.tr, 3);            // streaming done
     // ---- 5. combine the row groups through the (now idle) ring, in group order ----
     __syncthreads();
     float *red = reinterpret_cast<float *>(&s.ring[0][0]);    // [RG-1][CG*32 lanes][BT][E]
@@ -355,7 +359,10 @@ gemv_kernel(const GemvParams p)
         __syncthreads();
         if (tid == 0) s.last = atomicAdd(&p.tickets[slab], 1u) == (unsigned)(nparts - 1);
         __syncthreads();
-        if (!s.last) return;
+        if (!s.last) {
+            DIP_TRACE_MAX(p.tr, 2);
+            return;
+        }
         __threadfence();
     } else {
         __syncthreads();
@@ -406,6 +413,7 @@ gemv_kernel(const GemvParams p)
         p.out[(size_t)b * p.d_out + j] = WHICH == 0 ? silu_f32(s0) * s1 : s0;
     }
     if (nparts > 1 && tid == 0) p.tickets[slab] = 0;   // ready for the next launch
+    DIP_TRACE_MAX(p.tr, 2);
 }
 
 }  // namespace
@@ -502,6 +510,7 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
         p.v = v + (size_t)b0 * p.d_in;
         p.mask_bits = mask_bits + (size_t)b0 * p.mask_words;
         p.out = out + (size_t)b0 * p.d_out;
+        p.tr = dip_trace_slot(ctx, which == 0 ? 4 : 5);
         dip_status st;
         if (w->wtype == DIP_W_F32)
             st = which == 0 ? launch_bt<DIP_W_F32, 0>(ctx, p, n_kept_max, stream)

@@ -166,8 +166,9 @@ template <bool CA, bool NORM>
 __global__ void __launch_bounds__(TK_THREADS, 1)
 select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *__restrict__ x_out,
               int d, int k, float gamma, const int32_t *__restrict__ stamp,
-              uint32_t *__restrict__ mask_bits)
+              uint32_t *__restrict__ mask_bits, unsigned long long *tr)
 {
+    DIP_TRACE_MIN(tr, 0);
     extern __shared__ uint32_t keys[];
     __shared__ TkShared s;
     __shared__ uint32_t cand_key[TK_CAND_CAP];
@@ -190,6 +191,7 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
         s.n_cand2 = 0;
     }
     dip_grid_dependency_wait();        // the inputs come from the previous kernel in the stream
+    DIP_TRACE_MIN(tr, 1);
     dip_launch_dependents();
 
     if (NORM) {
@@ -292,6 +294,7 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
             }
             __syncthreads();
             for (int w = tid; w < n_words; w += TK_THREADS) mask_bits[w] = s_maskw[w];
+            DIP_TRACE_MAX(tr, 2);
             return;
         }
     }
@@ -308,6 +311,7 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
             const unsigned bk = __ballot_sync(0xffffffffu, e < d && keys[e] >= T);
             if (lane == 0) mask_bits[(base + it) >> 5] = bk;
         }
+        DIP_TRACE_MAX(tr, 2);
         return;
     }
     // only the first `quota` tied columns (by index) are kept: rank the ties in order
@@ -331,6 +335,7 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
         if (lane == 0) mask_bits[(base + it) >> 5] = bk;
         eq_before += __popc(bq);
     }
+    DIP_TRACE_MAX(tr, 2);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -340,8 +345,11 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
 // last use for columns that may be evicted (resident and outside the mask) and 0 otherwise.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(TK_THREADS, 1)
-cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stamp, int32_t *meta, int capacity)
+cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stamp, int32_t *meta, int capacity,
+                    unsigned long long *tr)
 {
+    DIP_TRACE_MIN(tr, 0);
+    DIP_TRACE_MIN(tr, 1);
     extern __shared__ uint32_t keys[];
     __shared__ TkShared s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -435,6 +443,7 @@ cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stam
         meta[4] += n_evict;
         meta[5] += total_misses - inserted;
     }
+    DIP_TRACE_MAX(tr, 2);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -519,20 +528,21 @@ dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, flo
 {
     const size_t smem = (size_t)d * sizeof(uint32_t);
     const dim3 grid(batch), block(TK_THREADS);
+    unsigned long long *tr = dip_trace_slot(ctx, d <= 0 ? 0 : (stamp ? 2 : 1));
     cudaError_t e;
     if (xb) {
         if (stamp)
-            e = dip_launch_pdl(select_kernel<true, true>, grid, block, smem, stream, xa, xb, x_out, d, k, gamma, stamp, mask_bits);
+            e = dip_launch_pdl(select_kernel<true, true>, grid, block, smem, stream, xa, xb, x_out, d, k, gamma, stamp, mask_bits, tr);
         else
             e = dip_launch_pdl(select_kernel<false, true>, grid, block, smem, stream, xa, xb, x_out, d, k, 1.0f,
-                               (const int32_t *)nullptr, mask_bits);
+                               (const int32_t *)nullptr, mask_bits, tr);
     } else {
         if (stamp)
             e = dip_launch_pdl(select_kernel<true, false>, grid, block, smem, stream, xa, (const float *)nullptr,
-                               (float *)nullptr, d, k, gamma, stamp, mask_bits);
+                               (float *)nullptr, d, k, gamma, stamp, mask_bits, tr);
         else
             e = dip_launch_pdl(select_kernel<false, false>, grid, block, smem, stream, xa, (const float *)nullptr,
-                               (float *)nullptr, d, k, 1.0f, (const int32_t *)nullptr, mask_bits);
+                               (float *)nullptr, d, k, 1.0f, (const int32_t *)nullptr, mask_bits, tr);
     }
     DIP_CUDA_TRY(ctx, e);
     return DIP_OK;
@@ -541,7 +551,8 @@ dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, flo
 dip_status dip_launch_cache_update(dip_ctx *ctx, const uint32_t *mask_bits, int d, int32_t *stamp, int32_t *meta,
                                    int capacity, cudaStream_t stream)
 {
-    cache_update_kernel<<<1, TK_THREADS, (size_t)d * sizeof(uint32_t), stream>>>(mask_bits, d, stamp, meta, capacity);
+    cache_update_kernel<<<1, TK_THREADS, (size_t)d * sizeof(uint32_t), stream>>>(mask_bits, d, stamp, meta, capacity,
+                                                                                   dip_trace_slot(ctx, 3));
     DIP_CUDA_TRY(ctx, cudaGetLastError());
     return DIP_OK;
 }
