@@ -377,40 +377,47 @@ gemv_kernel(const GemvParams p)
         }
         return;
     }
-    for (int t = tid; t < BT * OUT_PER_SLAB; t += GV_THREADS) {
-        const int b = t / OUT_PER_SLAB, o = t % OUT_PER_SLAB;
+    // four consecutive outputs per thread (16-byte loads of the partial sums)
+    for (int t = tid; t < BT * (OUT_PER_SLAB / 4); t += GV_THREADS) {
+        const int b = t / (OUT_PER_SLAB / 4), o = (t % (OUT_PER_SLAB / 4)) * 4;
         const int j = slab * OUT_PER_SLAB + o;
         if (b >= p.batch || j >= p.d_out) continue;
         int e0, e1 = 0;
         if (WHICH == 0) {
-            e0 = (o / C) * 2 * C + (o % C);      // gate element of output o
-            e1 = e0 + C;                         // matching up element
+            e0 = (o / C) * 2 * C + (o % C);      // gate elements of outputs o .. o+3
+            e1 = e0 + C;                         // matching up elements
         } else {
             e0 = o;
         }
-        float s0 = 0.f, s1 = 0.f;
+        float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
         if (nparts > 1) {
             // parts in part order; eight loads in flight at a time
             const size_t stride = (size_t)gridDim.x * (BT * SLAB);
             const float *pp = p.partials + (size_t)slab * (BT * SLAB) + b * SLAB;
             for (int q0 = 0; q0 < nparts; q0 += 8) {
-                float a0[8], a1[8];
+                float4 a0[8], a1[8];
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
-                    a0[q] = q0 + q < nparts ? __ldcg(pp + (size_t)(q0 + q) * stride + e0) : 0.f;
-                    a1[q] = (WHICH == 0 && q0 + q < nparts) ? __ldcg(pp + (size_t)(q0 + q) * stride + e1) : 0.f;
+                    a0[q] = a1[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q0 + q < nparts) {
+                        a0[q] = __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(q0 + q) * stride + e0));
+                        if (WHICH == 0)
+                            a1[q] = __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(q0 + q) * stride + e1));
+                    }
                 }
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
-                    s0 += a0[q];
-                    s1 += a1[q];
+                    s0.x += a0[q].x; s0.y += a0[q].y; s0.z += a0[q].z; s0.w += a0[q].w;
+                    s1.x += a1[q].x; s1.y += a1[q].y; s1.z += a1[q].z; s1.w += a1[q].w;
                 }
             }
         } else {
-            s0 = own[b * SLAB + e0];
-            if (WHICH == 0) s1 = own[b * SLAB + e1];
+            s0 = *reinterpret_cast<const float4 *>(own + b * SLAB + e0);
+            if (WHICH == 0) s1 = *reinterpret_cast<const float4 *>(own + b * SLAB + e1);
         }
-        p.out[(size_t)b * p.d_out + j] = WHICH == 0 ? silu_f32(s0) * s1 : s0;
+        float4 r = s0;
+        if (WHICH == 0) r = make_float4(silu_f32(s0.x) * s1.x, silu_f32(s0.y) * s1.y, silu_f32(s0.z) * s1.z, silu_f32(s0.w) * s1.w);
+        *reinterpret_cast<float4 *>(p.out + (size_t)b * p.d_out + j) = r;
     }
     if (nparts > 1 && tid == 0) p.tickets[slab] = 0;   // ready for the next launch
     DIP_TRACE_MAX(p.tr, 2);
@@ -449,8 +456,9 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cuda
 
 // Segment width and number of row parts: one CTA per SM, all resident at once.  A wide
 // segment is kinder to DRAM, but few slabs mean many parts, and the CTA that finishes a slab
-// then has nparts * SEG bytes of partial sums to add up alone; narrow the segment until that
-// tail is short (or until no split is needed at all).
+// then has nparts * SEG bytes of partial sums to add up alone.  Bulk copies shorter than 2 KB
+// run into the copy engine's request rate (measured: 1 KB segments stream a third slower), so
+// the segment is narrowed only when that tail would get very long.
 template <int WT, int WHICH, int BT>
 dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t stream)
 {
@@ -463,7 +471,7 @@ dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t 
         nparts = ctx->sm_count / n_slabs;
         if (nparts > n_kept_max) nparts = n_kept_max;
         if (nparts < 1) nparts = 1;
-        if (seg || (long long)nparts * sg <= 20480 || sg == 512) {
+        if (seg || (long long)nparts * sg <= 65536 || sg == 512) {
             seg = sg;
             break;
         }
