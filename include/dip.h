@@ -115,16 +115,16 @@ dip_status dip_trace_end(dip_ctx *ctx);
  * W in R^{d_out x d_in} (Eq. 4, 7, 8), so the library stores each matrix
  * column-contiguous: row i of the packed array holds column i.  Gate and up
  * always share one mask (Eq. 7), so their columns are bundled: packed row i
- * holds W^g[:, i] and W^u[:, i] interleaved in 16-byte pieces
- * (piece 2c = gate outputs of chunk c, piece 2c+1 = up outputs of chunk c;
- * a chunk is 4 outputs for F32, 8 for BF16, 32 for INT4).
+ * holds W^g[:, i] and W^u[:, i] interleaved in chunks of C outputs (piece 2c =
+ * gate outputs of chunk c, piece 2c+1 = up outputs of chunk c), C = 4 for F32
+ * and 8 for BF16 (16-byte pieces), C = 16 for INT4 (8-byte pieces).
  *
  *   gate_up        [d_model][2 * d_ff] elements, interleaved as above
  *   down           [d_ff][d_model]     elements
- *   INT4 codes     two per byte, output j in bits 4*(j&1).. of byte j>>1 within a row
- *                  (within a 16-byte piece for gate_up); value = (code - 8) * scale
- *   gate_up_scales [d_model/128][2 * d_ff] binary16, interleaved in 16-byte pieces
- *                  (8 gate scales, 8 up scales)
+ *   INT4 codes     two per byte, element e of a row in bits 4*(e&1).. of byte e>>1;
+ *                  value = (code - 8) * scale
+ *   gate_up_scales [d_model/128][2 * d_ff] binary16, element for element like a
+ *                  gate_up row (16 gate scales, 16 up scales, ...)
  *   down_scales    [d_ff/128][d_model] binary16
  *
  * Requirements: d_model % 32 == 0, d_ff % 32 == 0 (all formats); INT4 also

@@ -16,6 +16,8 @@
 //
 // which = 0 (gate/up bundle): the epilogue applies silu(gate) * up (Eq. 2).  which = 1: down.
 // Every wait on an mbarrier is bounded; on expiry the kernel records a status word and leaves.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace {
@@ -30,6 +32,8 @@ constexpr unsigned long long GV_WAIT_LIMIT_NS = 1000000000ull;   // a wait gives
 struct GemvParams {
     const char *W;             // packed rows
     size_t row_bytes;          // bytes of one packed row
+    const uint16_t *scales;    // INT4: binary16 scales [d_in/128][row elements], laid out like a row
+    size_t scale_row_elems;    // INT4: elements of one scale row
     const float *v;            // [batch][d_in]
     int d_in;
     const uint32_t *mask_bits; // [batch][mask_words]; rows read = OR over the batch
@@ -85,8 +89,10 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
 __device__ __forceinline__ float silu_f32(float g) { return g / (1.0f + expf(-g)); }
 
 template <int WT> struct WTraits;
-template <> struct WTraits<DIP_W_F32>  { static constexpr int E = 4; static constexpr int EB = 4; };
-template <> struct WTraits<DIP_W_BF16> { static constexpr int E = 8; static constexpr int EB = 2; };
+// E = weights in a lane's 16 bytes; C = gate/up interleave chunk of the bundled rows (weights)
+template <> struct WTraits<DIP_W_F32>       { static constexpr int E = 4;  static constexpr int C = 4; };
+template <> struct WTraits<DIP_W_BF16>      { static constexpr int E = 8;  static constexpr int C = 8; };
+template <> struct WTraits<DIP_W_INT4_G128> { static constexpr int E = 32; static constexpr int C = 16; };
 
 template <int WT> __device__ __forceinline__ void decode16(const uint4 &r, float (&w)[WTraits<WT>::E]);
 template <> __device__ __forceinline__ void decode16<DIP_W_F32>(const uint4 &r, float (&w)[4])
@@ -103,6 +109,20 @@ template <> __device__ __forceinline__ void decode16<DIP_W_BF16>(const uint4 &r,
         w[2 * i] = __uint_as_float(u[i] << 16);
         w[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
     }
+}
+
+// Eight 4-bit codes of one word as (code - 8) in binary32: OR-ing a code into the mantissa of
+// 2^23 gives 8388608 + code exactly; subtracting 8388616 leaves code - 8.
+__device__ __forceinline__ void decode_int4_word(uint32_t w, float *out)
+{
+#pragma unroll
+    for (int n = 0; n < 8; ++n)
+        out[n] = __uint_as_float(0x4b000000u | ((w >> (4 * n)) & 15u)) - 8388616.0f;
+}
+
+__device__ __forceinline__ float half_bits_to_float(uint16_t h)
+{
+    return __half2float(__ushort_as_half(h));
 }
 
 constexpr int GV_STAGE_BYTES = 32768;
@@ -128,10 +148,9 @@ __global__ void __launch_bounds__(GV_THREADS, 1)
 gemv_kernel(const GemvParams p)
 {
     constexpr int E = WTraits<WT>::E;
-    constexpr int EB = WTraits<WT>::EB;
-    constexpr int SLAB = SEG / EB;                            // packed elements per slab
+    constexpr int SLAB = (SEG / 16) * E;                      // packed elements per slab
     constexpr int OUT_PER_SLAB = WHICH == 0 ? SLAB / 2 : SLAB;
-    constexpr int C = 16 / EB;                                // gate/up interleave chunk (elements)
+    constexpr int C = WTraits<WT>::C;                         // gate/up interleave chunk (elements)
     constexpr int CG = SEG / 512;                             // column groups (warps across the segment)
     constexpr int RG = GV_CONSUMER_WARPS / CG;                // row groups
     constexpr int R = GV_STAGE_BYTES / SEG;                   // rows per stage
@@ -218,6 +237,13 @@ gemv_kernel(const GemvParams p)
     for (int b = 0; b < BT; ++b)
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[b][e] = 0.f;
+    // INT4 only: sums of the current scale group, its scales, and which group that is
+    float accg[WT == DIP_W_INT4_G128 ? E : 1], sc[WT == DIP_W_INT4_G128 ? E : 1];
+    int cur_group = -1;
+    if (WT == DIP_W_INT4_G128) {
+#pragma unroll
+        for (int e = 0; e < (WT == DIP_W_INT4_G128 ? E : 1); ++e) accg[e] = sc[e] = 0.f;
+    }
     bool failed = false;
     int it_base = 0;                                          // stages issued in earlier rounds
 
@@ -295,18 +321,60 @@ gemv_kernel(const GemvParams p)
                 if (failed || s.abort) { failed = true; break; }
                 const int rows_here = min(R, n_rows - i * R);
                 if (lane_ok) {
+                    if constexpr (WT == DIP_W_INT4_G128) {
+                        // W = (code - 8) * scale[group of 128 rows]: sum (code - 8) * v within a
+                        // group, multiply by the group's scales when the group changes
+                        for (int rr = 0; rr < R / RG; ++rr) {
+                            const int r = rr * RG + rg;
+                            if (r >= rows_here) break;
+                            const int g = s.idx[i * R + r] >> 7;
+                            if (g != cur_group) {
+                                if (cur_group >= 0) {
 #pragma unroll
-                    for (int rr = 0; rr < R / RG; ++rr) {
-                        const int r = rr * RG + rg;
-                        if (r < rows_here) {
+                                    for (int e = 0; e < E; ++e) {
+                                        acc[0][e] = fmaf(sc[e], accg[e], acc[0][e]);
+                                        accg[e] = 0.f;
+                                    }
+                                }
+                                const uint4 *sp = reinterpret_cast<const uint4 *>(
+                                    p.scales + (size_t)g * p.scale_row_elems + (size_t)slab * SLAB + (cw * 32 + lane) * E);
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const uint4 sv = __ldg(sp + q);
+                                    const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                                    for (int t = 0; t < 4; ++t) {
+                                        sc[q * 8 + 2 * t] = half_bits_to_float((uint16_t)(sw[t] & 0xffffu));
+                                        sc[q * 8 + 2 * t + 1] = half_bits_to_float((uint16_t)(sw[t] >> 16));
+                                    }
+                                }
+                                cur_group = g;
+                            }
                             const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * SEG + byte_off]);
-                            float w[E];
-                            decode16<WT>(raw, w);
+                            const float xv = s_v[i * R + r];
+                            const uint32_t cwd[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-                            for (int b = 0; b < BT; ++b) {
-                                const float xv = s_v[b * GV_MAX_ROWS + i * R + r];
+                            for (int q = 0; q < 4; ++q) {
+                                float w8[8];
+                                decode_int4_word(cwd[q], w8);
 #pragma unroll
-                                for (int e = 0; e < E; ++e) acc[b][e] = fmaf(w[e], xv, acc[b][e]);
+                                for (int n = 0; n < 8; ++n) accg[q * 8 + n] = fmaf(w8[n], xv, accg[q * 8 + n]);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int rr = 0; rr < R / RG; ++rr) {
+                            const int r = rr * RG + rg;
+                            if (r < rows_here) {
+                                const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * SEG + byte_off]);
+                                float w[E];
+                                decode16<WT>(raw, w);
+#pragma unroll
+                                for (int b = 0; b < BT; ++b) {
+                                    const float xv = s_v[b * GV_MAX_ROWS + i * R + r];
+#pragma unroll
+                                    for (int e = 0; e < E; ++e) acc[b][e] = fmaf(w[e], xv, acc[b][e]);
+                                }
                             }
                         }
                     }
@@ -323,6 +391,12 @@ gemv_kernel(const GemvParams p)
     }
 
     DIP_TRACE_MAX(p.tr, 3);            // streaming done
+    if constexpr (WT == DIP_W_INT4_G128) {
+        if (cur_group >= 0) {
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[0][e] = fmaf(sc[e], accg[e], acc[0][e]);
+        }
+    }
     // ---- 5. combine the row groups through the (now idle) ring, in group order ----
     __syncthreads();
     float *red = reinterpret_cast<float *>(&s.ring[0][0]);    // [RG-1][CG*32 lanes][BT][E]
@@ -346,7 +420,7 @@ gemv_kernel(const GemvParams p)
             for (int g = 1; g < RG; ++g)
 #pragma unroll
                 for (int e = 0; e < E; ++e) sum[e] += red[((((g - 1) * CG + cw) * 32 + lane) * BT + b) * E + e];
-            float *d = dst + b * SLAB + (cw * 512 + lane * 16) / EB;
+            float *d = dst + b * SLAB + (cw * 32 + lane) * E;
 #pragma unroll
             for (int e = 0; e < E; e += 4)
                 *reinterpret_cast<float4 *>(d + e) = make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
@@ -439,7 +513,7 @@ __global__ void idx_to_mask_kernel(const int32_t *__restrict__ idx, int n, int d
 template <int WT, int WHICH, int BT, int SEG>
 dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cudaStream_t stream)
 {
-    constexpr int SLAB = SEG / WTraits<WT>::EB;
+    constexpr int SLAB = (SEG / 16) * WTraits<WT>::E;
     const size_t per_part = (size_t)n_slabs * BT * SLAB;
     if (nparts > 1 && (size_t)nparts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
     const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * GV_MAX_ROWS * sizeof(float);
@@ -500,11 +574,14 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                            const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
                            float *out, cudaStream_t stream)
 {
-    if (w->wtype != DIP_W_F32 && w->wtype != DIP_W_BF16) return DIP_ERR_UNSUPPORTED;
-    const int elem_bytes = w->wtype == DIP_W_F32 ? 4 : 2;
+    const bool int4 = w->wtype == DIP_W_INT4_G128;
+    if (int4 && batch > 1) return DIP_ERR_UNSUPPORTED;      // the 4-bit path is single-token
+    const size_t row_elems = which == 0 ? (size_t)2 * w->d_ff : (size_t)w->d_model;
     GemvParams p;
     p.W = (const char *)(which == 0 ? w->gate_up : w->down);
-    p.row_bytes = (size_t)(which == 0 ? 2 * w->d_ff : w->d_model) * elem_bytes;
+    p.row_bytes = w->wtype == DIP_W_F32 ? row_elems * 4 : w->wtype == DIP_W_BF16 ? row_elems * 2 : row_elems / 2;
+    p.scales = (const uint16_t *)(which == 0 ? w->gate_up_scales : w->down_scales);
+    p.scale_row_elems = row_elems;
     p.d_in = which == 0 ? w->d_model : w->d_ff;
     p.d_out = which == 0 ? w->d_ff : w->d_model;
     p.mask_words = (p.d_in + 31) / 32;
@@ -520,7 +597,10 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
         p.out = out + (size_t)b0 * p.d_out;
         p.tr = dip_trace_slot(ctx, which == 0 ? 4 : 5);
         dip_status st;
-        if (w->wtype == DIP_W_F32)
+        if (int4)
+            st = which == 0 ? launch_one<DIP_W_INT4_G128, 0, 1>(ctx, p, n_kept_max, stream)
+                            : launch_one<DIP_W_INT4_G128, 1, 1>(ctx, p, n_kept_max, stream);
+        else if (w->wtype == DIP_W_F32)
             st = which == 0 ? launch_bt<DIP_W_F32, 0>(ctx, p, n_kept_max, stream)
                             : launch_bt<DIP_W_F32, 1>(ctx, p, n_kept_max, stream);
         else

@@ -145,6 +145,8 @@ GEMV_SHAPES = [
     (di.W_F32, 1024, 2816, 0.5), (di.W_BF16, 3072, 8192, 0.25), (di.W_BF16, 1024, 2816, 0.1),
     (di.W_BF16, 1056, 2848, 0.3),      # ragged: the last output slab is partly empty
     (di.W_F32, 96, 160, 1.0), (di.W_BF16, 512, 1024, 1.0), (di.W_BF16, 256, 512, 0.004),
+    (di.W_INT4_G128, 1024, 2816, 0.25), (di.W_INT4_G128, 384, 640, 0.5), (di.W_INT4_G128, 256, 512, 1.0),
+    (di.W_INT4_G128, 4096, 14336, 0.25), (di.W_INT4_G128, 512, 1024, 0.01),
 ]
 
 
@@ -223,6 +225,9 @@ def _check_step(dip, ctx, lw, w, x, k_x, k_h, gamma, ref_gu, ref_d, g_gu, g_d):
     (di.W_BF16, 1024, 4096, 0.1, 0.25),
     (di.W_BF16, 1024, 2048, 0.5, 0.25),     # k > capacity: bypass
     (di.W_BF16, 512, 1536, 1.0, 0.5),       # keep ratio 1: dense
+    (di.W_INT4_G128, 1024, 2816, 0.25, 0.4),
+    (di.W_INT4_G128, 4096, 14336, 0.25, 0.4),   # a full Llama-3-8B-shaped block
+    (di.W_INT4_G128, 512, 1024, 1.0, None),
 ])
 def test_mlp_step_matches_oracle(dip, ctx, wtype, d_model, d_ff, rho, beta):
     lw = _layer(17 + d_ff, d_model, d_ff, wtype)
