@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging; not a valid bench)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--report", default=None, metavar="FILE",
+                    help="run every workload of the five configurations (fewer steps) and write a markdown table")
     ap.add_argument("--timeline", action="store_true",
                     help="print the device-side timeline of one graph replay (per kernel: start, ready, end) and exit")
     return ap.parse_args()
@@ -164,9 +166,11 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
 
     n_tok = xs_host.shape[0]
     xs_dev = xs_host.cuda()
-    x_cur = torch.empty(d_model, device="cuda")
-    x_out = torch.empty(d_model, device="cuda")
-    out_host = torch.empty(d_model).pin_memory()
+    # xs_host is [tokens, d_model] (one sequence) or [tokens, batch, d_model] (batched decode)
+    batch = 1 if xs_host.dim() == 2 else xs_host.shape[1]
+    x_cur = torch.empty(tuple(xs_host.shape[1:]), device="cuda")
+    x_out = torch.empty_like(x_cur)
+    out_host = torch.empty(tuple(xs_host.shape[1:])).pin_memory()
     stack = fresh_stack()
     stream = torch.cuda.current_stream()
 
@@ -216,6 +220,18 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
            "ms_per_step": ms / steps, "mlp_steps_per_s": L * steps / (ms * 1e-3), "clocks": clocks,
            "bytes": algorithmic_bytes(w, k_x, k_h, ca)}
     res["step_gbs"] = res["bytes"]["step"] * L * steps / (ms * 1e-3) / 1e9
+    res["batch"] = batch
+    if batch > 1:
+        # density of the union of the tokens' masks (measured on layer 0): the share of a layer's
+        # columns that a batched step reads
+        counts = torch.zeros(2, dtype=torch.int32, device="cuda")
+        y_tmp = torch.empty_like(x_cur)
+        dip.dip_mlp_step(ctx, layers[0], xs_dev[0], k_x, k_h, gamma, None, None, y_tmp, union_counts=counts)
+        ux, uh = counts.cpu().tolist()
+        res["union_density"] = {"x": ux / d_model, "h": uh / d_ff}
+        ub = weight_bytes(w.wtype)
+        res["union_bytes"] = ux * 2 * d_ff * ub + uh * d_model * ub
+        res["union_gbs"] = res["union_bytes"] * L * steps / (ms * 1e-3) / 1e9
     if ca:
         meta = torch.stack([c.meta for c in stack.cache_gu + stack.cache_d]).sum(0).cpu().tolist()
         res["hit_rate"] = meta[2] / max(1, meta[2] + meta[3])
@@ -245,11 +261,11 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
             dist.all_reduce(tms, op=dist.ReduceOp.MAX)
             ms_e = float(tms.item())
         res["e2e"] = {"value": L * n_e2e / (ms_e * 1e-3), "unit": UNIT, "steps": n_e2e,
-                      "h2d_bytes_per_step": 4 * d_model, "d2h_bytes_per_step": 4 * d_model,
+                      "h2d_bytes_per_step": 4 * d_model * batch, "d2h_bytes_per_step": 4 * d_model * batch,
                       "wall_ms": (time.perf_counter() - t0) * 1e3}
 
     # ---- per-kernel durations (separate instrumented pass, one event pair per launch) ----
-    if kernel_pass:
+    if kernel_pass and batch == 1:
         st2 = fresh_stack()
         mask_x = torch.zeros((d_model + 31) // 32, dtype=torch.int32, device="cuda")
         idx_x = torch.zeros(k_x, dtype=torch.int32, device="cuda")
@@ -330,6 +346,50 @@ def print_timeline(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget):
     print("# critical path per layer: %.2f us" % ((main_path[-1]["end"] - main_path[0]["ready"]) / L))
 
 
+def write_report(dip, ctx, torch, path, steps):
+    """All five configurations (bench workloads), one row each: MLP-steps/s, effective GB/s on the
+    kept-column bytes, fraction of the measured and nominal HBM peak."""
+    peak, kind = measured_peak()
+    rows = []
+
+    def row(name, r, L, extra=""):
+        gbs = r.get("union_gbs", r["step_gbs"])
+        rows.append("| %s | %g | %s | %d | %.0f | %.1f | %.0f | %.1f %% | %.1f %% | %s |" % (
+            name, r["keep_ratio"], r["cache_budget"], r["batch"], r["mlp_steps_per_s"], r["ms_per_step"] * 1e3 / L,
+            gbs, 100 * gbs / NOMINAL_HBM_GBS, 100 * gbs / peak, extra))
+
+    for name in ("block_f32", "phi3_mini", "phi3_medium", "llama3_8b_int4", "phi3_medium_batched"):
+        w = di.WORKLOADS[name]
+        L = 8 if name == "block_f32" else w.n_layers      # 8 distinct blocks cycled: HBM-cold
+        layers = build_stack(dip, ctx, torch, w, L, 0)
+        n_tok = min(w.n_tokens, steps + 8)
+        if name == "phi3_medium_batched":
+            for B in di.BATCH_SIZES:
+                xs = torch.from_numpy(di.token_inputs(w, n_tokens=n_tok, batch=B).copy())
+                xs = xs[:, 0] if B == 1 else xs
+                r = run_config(dip, ctx, torch, w, layers, xs, w.keep_ratio, None, min(steps, 64), 4,
+                               kernel_pass=False, e2e_pass=False)
+                ud = r.get("union_density")
+                row(name, r, L, "union density x %.2f h %.2f" % (ud["x"], ud["h"]) if ud else "")
+        else:
+            xs = torch.from_numpy(di.token_inputs(w, n_tokens=n_tok, batch=1)[:, 0].copy())
+            combos = [(w.keep_ratio, w.cache_budget)]
+            if name == "phi3_medium":
+                combos = [(r_, b_) for r_ in di.PHI3_MEDIUM_KEEP_RATIOS for b_ in di.PHI3_MEDIUM_CACHE_BUDGETS]
+            for rho, beta in combos:
+                r = run_config(dip, ctx, torch, w, layers, xs, rho, beta, steps, 4, kernel_pass=False, e2e_pass=False)
+                extra = "hit rate %.2f" % r["hit_rate"] if "hit_rate" in r else ""
+                if name == "block_f32":
+                    extra = "8 distinct blocks cycled (one block alone fits L2)"
+                row(name, r, L, extra)
+        del layers
+        torch.cuda.empty_cache()
+    with open(path, "w") as f:
+        f.write("| workload | keep ratio | cache budget | batch | MLP-steps/s | us per MLP-step | GB/s (kept-column bytes) | of 8 TB/s | of %s %.0f GB/s | notes |\n" % (kind, peak))
+        f.write("|---|---|---|---|---|---|---|---|---|---|\n")
+        f.write("\n".join(rows) + "\n")
+
+
 def oracle_rate(w, keep_ratio, budget, n_layers_sample, n_steps, warmup=0):
     """The CPU oracle as it stands, timed on this machine's host cores on a bounded sample of the
     workload: `n_steps` MLP-steps cycling over `n_layers_sample` host-generated layers."""
@@ -404,6 +464,9 @@ def main():
 
     import paper_2412_01380_b200 as dip
     ctx = dip.Context(local)
+    if args.report:
+        write_report(dip, ctx, torch, args.report, min(args.steps, 128))
+        return
     L = args.layers if args.layers else w.n_layers
     layers = build_stack(dip, ctx, torch, w, L, rank)
     n_tok = min(w.n_tokens, args.steps + args.warmup)
