@@ -152,6 +152,72 @@ __device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask
     quota = krem;
 }
 
+
+constexpr int TK_VEC_ITERS = DIP_MAX_D / 4 / TK_THREADS;   // float4 loads per thread at the largest d
+constexpr int TK_VEC_BATCH = 4;                            // of which this many are in flight together
+
+// scale = 1 / rms(xa + xb) over d elements, the same bits on every thread of the CTA.  The sums
+// r = xa + xb are optionally parked in stash[] (as bit patterns).  Summation order: each thread
+// adds its elements in index order (16-byte groups tid, tid + 1024, ... when d % 4 == 0, single
+// elements otherwise), then a shuffle tree per warp, then one over the warps.  Both users of this
+// function (the fused select and the stand-alone chaining kernel) therefore agree bit for bit.
+__device__ float block_residual_scale(const float *__restrict__ xa, const float *__restrict__ xb, int d,
+                                      uint32_t *stash, float *wf, float *scale_slot)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float ss = 0.f;
+    if ((d & 3) == 0) {
+        const float4 *a4 = reinterpret_cast<const float4 *>(xa), *b4 = reinterpret_cast<const float4 *>(xb);
+        const int n4 = d >> 2;
+        for (int j0 = 0; j0 < TK_VEC_ITERS && tid + j0 * TK_THREADS < n4; j0 += TK_VEC_BATCH) {
+        float4 va[TK_VEC_BATCH], vb[TK_VEC_BATCH];
+#pragma unroll
+        for (int j = 0; j < TK_VEC_BATCH; ++j) {
+            const int q = tid + (j0 + j) * TK_THREADS;
+            if (q < n4) {
+                va[j] = a4[q];
+                vb[j] = b4[q];
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < TK_VEC_BATCH; ++j) {
+            const int q = tid + (j0 + j) * TK_THREADS;
+            if (q < n4) {
+                const float r0 = va[j].x + vb[j].x, r1 = va[j].y + vb[j].y, r2 = va[j].z + vb[j].z, r3 = va[j].w + vb[j].w;
+                if (stash)
+                    *reinterpret_cast<uint4 *>(stash + 4 * q) =
+                        make_uint4(__float_as_uint(r0), __float_as_uint(r1), __float_as_uint(r2), __float_as_uint(r3));
+                ss = fmaf(r0, r0, ss);
+                ss = fmaf(r1, r1, ss);
+                ss = fmaf(r2, r2, ss);
+                ss = fmaf(r3, r3, ss);
+            }
+        }
+        }
+    } else {
+        for (int e = tid; e < d; e += TK_THREADS) {
+            const float r = xa[e] + xb[e];
+            if (stash) stash[e] = __float_as_uint(r);
+            ss = fmaf(r, r, ss);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (lane == 0) wf[warp] = ss;
+    __syncthreads();
+    if (warp == 0) {
+        float v = wf[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) {
+            const float rms = sqrtf(v / (float)d);
+            *scale_slot = rms > 0.f ? 1.0f / rms : 1.0f;
+        }
+    }
+    __syncthreads();
+    return *scale_slot;
+}
+
 // ---------------------------------------------------------------------------------------
 // select_kernel: the mask of one row.
 //   CA == false: key = bits(|x|)                              (DIP, Eq. 7-8)
@@ -194,42 +260,65 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
     DIP_TRACE_MIN(tr, 1);
     dip_launch_dependents();
 
-    if (NORM) {
-        float ss = 0.f;
-        for (int e = tid; e < d; e += TK_THREADS) {
-            float r = xa[e] + xb[e];
-            keys[e] = __float_as_uint(r);
-            ss = fmaf(r, r, ss);
-        }
+    float scale = 1.0f;
+    if (NORM)
+        scale = block_residual_scale(xa, xb, d, keys, s.wf, &s.scale);   // ends with a barrier
+    else
+        __syncthreads();                                                  // histogram zeroed
+    // rank keys, and the histogram of their top 11 bits (first radix pass) in the same sweep
+    if ((d & 3) == 0) {
+        const int n4 = d >> 2;
+        for (int j0 = 0; j0 < TK_VEC_ITERS && tid + j0 * TK_THREADS < n4; j0 += TK_VEC_BATCH) {
+        float4 v4[TK_VEC_BATCH];
+        int4 st4[TK_VEC_BATCH];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if (lane == 0) s.wf[warp] = ss;
-        __syncthreads();
-        if (warp == 0) {
-            float v = s.wf[lane];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == 0) {
-                float rms = sqrtf(v / (float)d);
-                s.scale = rms > 0.f ? 1.0f / rms : 1.0f;
+        for (int j = 0; j < TK_VEC_BATCH; ++j) {
+            const int q = tid + (j0 + j) * TK_THREADS;
+            if (q < n4) {
+                if (NORM) {
+                    const uint4 r = *reinterpret_cast<const uint4 *>(keys + 4 * q);
+                    v4[j] = make_float4(__uint_as_float(r.x) * scale, __uint_as_float(r.y) * scale,
+                                        __uint_as_float(r.z) * scale, __uint_as_float(r.w) * scale);
+                } else {
+                    v4[j] = reinterpret_cast<const float4 *>(xa)[q];
+                }
+                if (CA) st4[j] = reinterpret_cast<const int4 *>(stamp)[q];
             }
         }
-    }
-    __syncthreads();
-    // rank keys, and the histogram of their top 11 bits (first radix pass) in the same sweep
-    for (int e = tid; e < d; e += TK_THREADS) {
-        float v;
-        if (NORM) {
-            v = __uint_as_float(keys[e]) * s.scale;
-            x_out[e] = v;
-        } else {
-            v = xa[e];
+#pragma unroll
+        for (int j = 0; j < TK_VEC_BATCH; ++j) {
+            const int q = tid + (j0 + j) * TK_THREADS;
+            if (q < n4) {
+                if (NORM) reinterpret_cast<float4 *>(x_out)[q] = v4[j];
+                const float vv[4] = {v4[j].x, v4[j].y, v4[j].z, v4[j].w};
+                const int sv[4] = {CA ? st4[j].x : 0, CA ? st4[j].y : 0, CA ? st4[j].z : 0, CA ? st4[j].w : 0};
+                uint32_t kk[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    float a = fabsf(vv[t]);
+                    if (CA) a = __fmul_rn(a, sv[t] >= 0 ? 1.0f : gamma);
+                    kk[t] = __float_as_uint(a) & 0x7fffffffu;
+                    atomicAdd(&s.hist[kk[t] >> 20], 1u);
+                }
+                *reinterpret_cast<uint4 *>(keys + 4 * q) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+            }
         }
-        float a = fabsf(v);
-        if (CA) a = __fmul_rn(a, stamp[e] >= 0 ? 1.0f : gamma);
-        const uint32_t key = __float_as_uint(a) & 0x7fffffffu;
-        keys[e] = key;
-        atomicAdd(&s.hist[key >> 20], 1u);
+        }
+    } else {
+        for (int e = tid; e < d; e += TK_THREADS) {
+            float v;
+            if (NORM) {
+                v = __uint_as_float(keys[e]) * scale;
+                x_out[e] = v;
+            } else {
+                v = xa[e];
+            }
+            float a = fabsf(v);
+            if (CA) a = __fmul_rn(a, stamp[e] >= 0 ? 1.0f : gamma);
+            const uint32_t key = __float_as_uint(a) & 0x7fffffffu;
+            keys[e] = key;
+            atomicAdd(&s.hist[key >> 20], 1u);
+        }
     }
     __syncthreads();
     find_bin(s, k);
@@ -489,32 +578,15 @@ mask_to_idx_kernel(const uint32_t *__restrict__ mask_bits, int nb, int d,
 // order (per-thread strided partial sums, then a shuffle tree).
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(TK_THREADS, 1)
-residual_rmsnorm_kernel(const float *x, const float *__restrict__ y, int d, float *x_next)
+residual_rmsnorm_kernel(const float *x, const float *y, int d, float *x_next)
 {
-    __shared__ float wsum[TK_WARPS];
+    __shared__ float wf[TK_WARPS];
     __shared__ float s_scale;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
     const size_t off = (size_t)blockIdx.x * d;
-    float ss = 0.f;
-    for (int e = tid; e < d; e += TK_THREADS) {
-        float r = x[off + e] + y[off + e];
-        ss = fmaf(r, r, ss);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    if (lane == 0) wsum[warp] = ss;
-    __syncthreads();
-    if (warp == 0) {
-        float v = wsum[lane];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) {
-            float rms = sqrtf(v / (float)d);
-            s_scale = rms > 0.f ? 1.0f / rms : 1.0f;
-        }
-    }
-    __syncthreads();
-    const float sc = s_scale;
+    dip_grid_dependency_wait();
+    dip_launch_dependents();
+    const float sc = block_residual_scale(x + off, y + off, d, nullptr, wf, &s_scale);
     for (int e = tid; e < d; e += TK_THREADS) x_next[off + e] = (x[off + e] + y[off + e]) * sc;
 }
 
@@ -581,7 +653,6 @@ dip_status dip_launch_mask_to_idx(dip_ctx *ctx, const uint32_t *mask_bits, int r
 dip_status dip_launch_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y, int batch, int d,
                                        float *x_next, cudaStream_t stream)
 {
-    residual_rmsnorm_kernel<<<batch, TK_THREADS, 0, stream>>>(x, y, d, x_next);
-    DIP_CUDA_TRY(ctx, cudaGetLastError());
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(residual_rmsnorm_kernel, dim3(batch), dim3(TK_THREADS), 0, stream, x, y, d, x_next));
     return DIP_OK;
 }
