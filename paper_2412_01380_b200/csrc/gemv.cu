@@ -26,6 +26,9 @@ constexpr int GV_CONSUMER_WARPS = 8;
 constexpr int GV_THREADS = (GV_CONSUMER_WARPS + 1) * 32;   // + one producer warp
 constexpr int GV_STAGES = 5;
 constexpr int GV_MAX_ROWS = 2048;                          // kept rows per round (index list in smem)
+// Rows per round for BT tokens: the tokens' values of a round's rows stay in shared memory
+// (BT x rows floats, at most 32 KB).
+template <int BT> struct GvRound { static constexpr int ROWS = BT <= 4 ? GV_MAX_ROWS : (BT == 8 ? 1024 : 512); };
 constexpr int GV_SCAN_THREADS = 256;                       // threads that scan the mask words
 constexpr unsigned long long GV_WAIT_LIMIT_NS = 1000000000ull;   // a wait gives up after one second
 
@@ -156,7 +159,8 @@ gemv_kernel(const GemvParams p)
     constexpr int R = GV_STAGE_BYTES / SEG;                   // rows per stage
     extern __shared__ __align__(128) unsigned char smem_raw[];
     GemvSmem<SEG> &s = *reinterpret_cast<GemvSmem<SEG> *>(smem_raw);
-    float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem<SEG>));   // [BT][GV_MAX_ROWS]
+    constexpr int ROWS = GvRound<BT>::ROWS;                   // rows per round
+    float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem<SEG>));   // [ROWS][BT]
 
     DIP_TRACE_MIN(p.tr, 0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -247,9 +251,9 @@ gemv_kernel(const GemvParams p)
     bool failed = false;
     int it_base = 0;                                          // stages issued in earlier rounds
 
-    // The part's rows go through in rounds of at most GV_MAX_ROWS (the in-kernel row list).
-    for (int round_begin = r_begin; round_begin < r_end; round_begin += GV_MAX_ROWS) {
-        const int n_rows = min(r_end - round_begin, GV_MAX_ROWS);
+    // The part's rows go through in rounds of at most ROWS (the in-kernel row list).
+    for (int round_begin = r_begin; round_begin < r_end; round_begin += ROWS) {
+        const int n_rows = min(r_end - round_begin, ROWS);
         if (round_begin != r_begin) {
             __syncthreads();                                  // everyone is done with the previous list
             if (s.abort) break;                               // uniform: read after the barrier
@@ -299,17 +303,28 @@ gemv_kernel(const GemvParams p)
             }
         } else {
             // ---- 4. consumers ----
-            // the tokens' values for the kept rows (zero where a token's own mask drops the row)
+            // the tokens' values for the kept rows (zero where a token's own mask drops the row),
+            // stored [row][token]; all of a row's loads are independent and issued together
             for (int r = tid; r < n_rows; r += GV_CONSUMER_WARPS * 32) {
                 const int idx = s.idx[r];
+                constexpr int GB = BT < 8 ? BT : 8;           // tokens gathered together
 #pragma unroll
-                for (int b = 0; b < BT; ++b) {
-                    float val = 0.f;
-                    // one token: every listed row is its own; several: ask the token's mask
-                    if (b < p.batch && (p.batch == 1 ||
-                        ((p.mask_bits[(size_t)b * p.mask_words + (idx >> 5)] >> (idx & 31)) & 1u)))
-                        val = p.v[(size_t)b * p.d_in + idx];
-                    s_v[b * GV_MAX_ROWS + r] = val;
+                for (int b0 = 0; b0 < BT; b0 += GB) {
+                    float vv[GB];
+                    uint32_t mw[GB];
+#pragma unroll
+                    for (int b = 0; b < GB; ++b) {
+                        vv[b] = 0.f;
+                        mw[b] = 0u;
+                        if (b0 + b < p.batch) {
+                            vv[b] = p.v[(size_t)(b0 + b) * p.d_in + idx];
+                            // one token: every listed row is its own; several: ask the token's mask
+                            mw[b] = p.batch == 1 ? 0xffffffffu
+                                                 : p.mask_bits[(size_t)(b0 + b) * p.mask_words + (idx >> 5)];
+                        }
+                    }
+#pragma unroll
+                    for (int b = 0; b < GB; ++b) s_v[r * BT + b0 + b] = ((mw[b] >> (idx & 31)) & 1u) ? vv[b] : 0.f;
                 }
             }
             asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
@@ -369,12 +384,21 @@ gemv_kernel(const GemvParams p)
                                 const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * SEG + byte_off]);
                                 float w[E];
                                 decode16<WT>(raw, w);
+                                float xv[BT];
+                                if constexpr (BT >= 4) {
 #pragma unroll
-                                for (int b = 0; b < BT; ++b) {
-                                    const float xv = s_v[b * GV_MAX_ROWS + i * R + r];
+                                    for (int b = 0; b < BT; b += 4) {
+                                        const float4 t4 = *reinterpret_cast<const float4 *>(&s_v[(i * R + r) * BT + b]);
+                                        xv[b] = t4.x; xv[b + 1] = t4.y; xv[b + 2] = t4.z; xv[b + 3] = t4.w;
+                                    }
+                                } else {
 #pragma unroll
-                                    for (int e = 0; e < E; ++e) acc[b][e] = fmaf(w[e], xv, acc[b][e]);
+                                    for (int b = 0; b < BT; ++b) xv[b] = s_v[(i * R + r) * BT + b];
                                 }
+#pragma unroll
+                                for (int b = 0; b < BT; ++b)
+#pragma unroll
+                                    for (int e = 0; e < E; ++e) acc[b][e] = fmaf(w[e], xv[b], acc[b][e]);
                             }
                         }
                     }
@@ -400,7 +424,8 @@ gemv_kernel(const GemvParams p)
     // ---- 5. combine the row groups through the (now idle) ring, in group order ----
     __syncthreads();
     float *red = reinterpret_cast<float *>(&s.ring[0][0]);    // [RG-1][CG*32 lanes][BT][E]
-    float *own = reinterpret_cast<float *>(&s.ring[GV_STAGES - 1][0]);   // [BT][SLAB] sums of this CTA
+    float *own = red + (RG - 1) * CG * 32 * BT * E;           // [BT][SLAB] sums of this CTA, after red
+    static_assert(((RG - 1) * CG * 32 * BT * E + BT * SLAB) * sizeof(float) <= sizeof(s.ring), "ring too small");
     if (warp < GV_CONSUMER_WARPS && rg > 0) {
 #pragma unroll
         for (int b = 0; b < BT; ++b)
@@ -516,7 +541,7 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cuda
     constexpr int SLAB = (SEG / 16) * WTraits<WT>::E;
     const size_t per_part = (size_t)n_slabs * BT * SLAB;
     if (nparts > 1 && (size_t)nparts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
-    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * GV_MAX_ROWS * sizeof(float);
+    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * GvRound<BT>::ROWS * sizeof(float);
     static bool attr_set = false;   // per instantiation
     if (!attr_set) {
         DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(gemv_kernel<WT, WHICH, BT, SEG>,
@@ -561,11 +586,11 @@ dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t 
 template <int WT, int WHICH>
 dip_status launch_bt(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t stream)
 {
-    switch (p.batch) {
-    case 1: return launch_one<WT, WHICH, 1>(ctx, p, n_kept_max, stream);
-    case 2: return launch_one<WT, WHICH, 2>(ctx, p, n_kept_max, stream);
-    default: return launch_one<WT, WHICH, 4>(ctx, p, n_kept_max, stream);
-    }
+    if (p.batch == 1) return launch_one<WT, WHICH, 1>(ctx, p, n_kept_max, stream);
+    if (p.batch == 2) return launch_one<WT, WHICH, 2>(ctx, p, n_kept_max, stream);
+    if (p.batch <= 4) return launch_one<WT, WHICH, 4>(ctx, p, n_kept_max, stream);
+    if (p.batch <= 8) return launch_one<WT, WHICH, 8>(ctx, p, n_kept_max, stream);
+    return launch_one<WT, WHICH, 16>(ctx, p, n_kept_max, stream);
 }
 
 }  // namespace
@@ -588,10 +613,10 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
     p.partials = ctx->partials;
     p.tickets = ctx->tickets;
     p.status = ctx->status;
-    // tokens go through in groups of at most four (accumulators live in registers); each group
-    // reads the union of its own tokens' rows
-    for (int b0 = 0; b0 < batch; b0 += 4) {
-        p.batch = batch - b0 < 4 ? batch - b0 : 4;
+    // all tokens of the batch in one launch (up to 16 sets of accumulators in registers): the
+    // union of their rows is read once
+    for (int b0 = 0; b0 < batch; b0 += 16) {
+        p.batch = batch - b0 < 16 ? batch - b0 : 16;
         p.v = v + (size_t)b0 * p.d_in;
         p.mask_bits = mask_bits + (size_t)b0 * p.mask_words;
         p.out = out + (size_t)b0 * p.d_out;
