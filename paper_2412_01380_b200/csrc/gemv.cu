@@ -129,6 +129,7 @@ __device__ __forceinline__ float half_bits_to_float(uint16_t h)
 }
 
 constexpr int GV_STAGE_BYTES = 32768;
+constexpr int GV_SCALE_STAGE_BYTES = 32768;                // INT4: shared memory for staged scale rows
 
 template <int SEG> struct __align__(16) GemvSmem {
     unsigned char ring[GV_STAGES][GV_STAGE_BYTES];   // [stage][row][SEG]
@@ -161,6 +162,10 @@ gemv_kernel(const GemvParams p)
     GemvSmem<SEG> &s = *reinterpret_cast<GemvSmem<SEG> *>(smem_raw);
     constexpr int ROWS = GvRound<BT>::ROWS;                   // rows per round
     float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem<SEG>));   // [ROWS][BT]
+    // INT4: the scale rows of the round's groups for this slab, staged once per round
+    uint16_t *s_sc = reinterpret_cast<uint16_t *>(smem_raw + sizeof(GemvSmem<SEG>) + sizeof(float) * BT * ROWS);
+    constexpr int SC_GROUPS = GV_SCALE_STAGE_BYTES / (SLAB * 2);   // groups that fit
+    int sc_first = 0, sc_count = 0;                                  // staged groups (uniform over the CTA)
 
     DIP_TRACE_MIN(p.tr, 0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -327,6 +332,19 @@ gemv_kernel(const GemvParams p)
                     for (int b = 0; b < GB; ++b) s_v[r * BT + b0 + b] = ((mw[b] >> (idx & 31)) & 1u) ? vv[b] : 0.f;
                 }
             }
+            if constexpr (WT == DIP_W_INT4_G128) {
+                // rows are ascending, so the round touches the groups first .. last; stage their
+                // scale segments if they fit (otherwise the consumers read them from global memory)
+                sc_first = s.idx[0] >> 7;
+                const int ng = (s.idx[n_rows - 1] >> 7) - sc_first + 1;
+                sc_count = ng <= SC_GROUPS ? ng : 0;
+                for (int t = tid; t < sc_count * (SLAB / 8); t += GV_CONSUMER_WARPS * 32) {
+                    const int g = t / (SLAB / 8), o = (t % (SLAB / 8)) * 8;
+                    if ((size_t)slab * SLAB + o < p.scale_row_elems)
+                        *reinterpret_cast<uint4 *>(s_sc + g * SLAB + o) = __ldg(reinterpret_cast<const uint4 *>(
+                            p.scales + (size_t)(sc_first + g) * p.scale_row_elems + (size_t)slab * SLAB + o));
+                }
+            }
             asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
 
             for (int i = 0; i < n_stages; ++i) {
@@ -351,11 +369,14 @@ gemv_kernel(const GemvParams p)
                                         accg[e] = 0.f;
                                     }
                                 }
-                                const uint4 *sp = reinterpret_cast<const uint4 *>(
-                                    p.scales + (size_t)g * p.scale_row_elems + (size_t)slab * SLAB + (cw * 32 + lane) * E);
+                                const bool staged = g - sc_first < sc_count;
+                                const uint4 *sp = staged
+                                    ? reinterpret_cast<const uint4 *>(s_sc + (g - sc_first) * SLAB + (cw * 32 + lane) * E)
+                                    : reinterpret_cast<const uint4 *>(p.scales + (size_t)g * p.scale_row_elems +
+                                                                      (size_t)slab * SLAB + (cw * 32 + lane) * E);
 #pragma unroll
                                 for (int q = 0; q < 4; ++q) {
-                                    const uint4 sv = __ldg(sp + q);
+                                    const uint4 sv = sp[q];
                                     const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
 #pragma unroll
                                     for (int t = 0; t < 4; ++t) {
@@ -541,7 +562,8 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cuda
     constexpr int SLAB = (SEG / 16) * WTraits<WT>::E;
     const size_t per_part = (size_t)n_slabs * BT * SLAB;
     if (nparts > 1 && (size_t)nparts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
-    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * GvRound<BT>::ROWS * sizeof(float);
+    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * GvRound<BT>::ROWS * sizeof(float) +
+                        (WT == DIP_W_INT4_G128 ? GV_SCALE_STAGE_BYTES : 0);
     static bool attr_set = false;   // per instantiation
     if (!attr_set) {
         DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(gemv_kernel<WT, WHICH, BT, SEG>,
@@ -570,7 +592,9 @@ dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t 
         nparts = ctx->sm_count / n_slabs;
         if (nparts > n_kept_max) nparts = n_kept_max;
         if (nparts < 1) nparts = 1;
-        if (seg || (long long)nparts * sg <= 65536 || sg == 512) {
+        // bytes of partial sums the CTA that completes a slab adds up: nparts x slab floats
+        const long long tail = (long long)nparts * (sg / 16) * WTraits<WT>::E * 4;
+        if (seg || tail <= 131072 || sg == 512) {
             seg = sg;
             break;
         }
