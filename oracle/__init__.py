@@ -34,15 +34,19 @@ _lib.orc_topk_mask.restype = _i32
 _lib.orc_topk_mask.argtypes = [_vp, _i32, _i32, _vp, _vp]
 _lib.orc_cache_update.restype = _i32
 _lib.orc_cache_update.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp, _vp]
+_lib.orc_cache_update_lfu.restype = _i32
+_lib.orc_cache_update_lfu.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp]
+_lib.orc_belady_hits.restype = C.c_longlong
+_lib.orc_belady_hits.argtypes = [_vp, _i32, _i32, _i32, _vp]
 _lib.orc_dip_ca_mask.restype = _i32
-_lib.orc_dip_ca_mask.argtypes = [_vp, _i32, _i32, _f32, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
+_lib.orc_dip_ca_mask.argtypes = [_vp, _i32, _i32, _f32, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
 _lib.orc_masked_matvec.restype = None
 _lib.orc_masked_matvec.argtypes = [_i32, _vp, _vp, _i32, _i32, _vp, _vp, _vp]
 _lib.orc_dense_mlp.restype = None
 _lib.orc_dense_mlp.argtypes = [_i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp, _vp]
 _lib.orc_mlp_step.restype = _i32
 _lib.orc_mlp_step.argtypes = ([_i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _i32, _f32]
-                              + [_vp, _vp, _vp, _i32, _vp] * 2 + [_vp] * 6)
+                              + [_vp, _vp, _vp, _vp, _i32, _vp] * 2 + [_vp] * 6)
 _lib.orc_residual_rmsnorm.restype = None
 _lib.orc_residual_rmsnorm.argtypes = [_vp, _vp, _i32, _vp]
 _lib.orc_mask_union.restype = _i32
@@ -107,8 +111,10 @@ class Matrix:
 class Cache:
     """LRU column-cache state of one masked linear-layer input (Alg. 1's c)."""
 
-    def __init__(self, d: int, capacity: int):
-        self.d, self.capacity = int(d), int(capacity)
+    def __init__(self, d: int, capacity: int, policy: str = "lru"):
+        assert policy in ("lru", "lfu")
+        self.d, self.capacity, self.policy = int(d), int(capacity), policy
+        self.count = np.zeros(d, dtype=np.int32)      # LFU use counters
         self.stamp = np.full(d, -1, dtype=np.int32)
         self.n_resident = np.zeros(1, dtype=np.int32)
         self.step = np.zeros(1, dtype=np.int32)
@@ -118,7 +124,8 @@ class Cache:
         return (self.stamp >= 0).astype(np.uint8)
 
     def copy(self) -> "Cache":
-        c = Cache(self.d, self.capacity)
+        c = Cache(self.d, self.capacity, self.policy)
+        c.count[:] = self.count
         c.stamp[:] = self.stamp
         c.n_resident[:] = self.n_resident
         c.step[:] = self.step
@@ -146,9 +153,23 @@ def topk_mask(key: np.ndarray, k: int):
 
 def cache_update(cache: Cache, m: np.ndarray) -> None:
     m = _chk(np.ascontiguousarray(m), np.uint8, cache.d)
-    if _lib.orc_cache_update(_p(cache.stamp), _p(cache.n_resident), _p(cache.step), cache.d,
-                             cache.capacity, _p(m), _p(cache.counters)):
+    if cache.policy == "lfu":
+        rc = _lib.orc_cache_update_lfu(_p(cache.stamp), _p(cache.count), _p(cache.n_resident), _p(cache.step),
+                                       cache.d, cache.capacity, _p(m), _p(cache.counters))
+    else:
+        rc = _lib.orc_cache_update(_p(cache.stamp), _p(cache.n_resident), _p(cache.step), cache.d,
+                                   cache.capacity, _p(m), _p(cache.counters))
+    if rc:
         raise ValueError("capacity outside [0, d]")
+
+
+def belady_hits(masks: np.ndarray, capacity: int):
+    """Offline Belady replay of a trace of masks uint8 [T, d]; returns (hits, misses)."""
+    masks = _chk(np.ascontiguousarray(masks), np.uint8)
+    T, d = masks.shape
+    miss = C.c_longlong(0)
+    hits = _lib.orc_belady_hits(_p(masks), T, d, int(capacity), C.byref(miss))
+    return int(hits), int(miss.value)
 
 
 def dip_ca_mask(x: np.ndarray, k: int, gamma: float = 1.0, cache: Optional[Cache] = None):
@@ -158,11 +179,12 @@ def dip_ca_mask(x: np.ndarray, k: int, gamma: float = 1.0, cache: Optional[Cache
     m = np.empty(d, dtype=np.uint8)
     idx = np.empty(max(k, 0), dtype=np.int32)
     if cache is None:
-        rc = _lib.orc_dip_ca_mask(_p(x), d, int(k), float(gamma), None, None, None, 0, _p(m), _p(idx), None)
+        rc = _lib.orc_dip_ca_mask(_p(x), d, int(k), float(gamma), None, None, None, None, 0, _p(m), _p(idx), None)
     else:
         if cache.d != d:
             raise ValueError("cache size mismatch")
-        rc = _lib.orc_dip_ca_mask(_p(x), d, int(k), float(gamma), _p(cache.stamp), _p(cache.n_resident),
+        rc = _lib.orc_dip_ca_mask(_p(x), d, int(k), float(gamma), _p(cache.stamp),
+                                  _p(cache.count) if cache.policy == "lfu" else None, _p(cache.n_resident),
                                   _p(cache.step), cache.capacity, _p(m), _p(idx), _p(cache.counters))
     if rc:
         raise ValueError("invalid k or capacity")
@@ -208,8 +230,9 @@ def mlp_step(Wg: Matrix, Wu: Matrix, Wd: Matrix, x: np.ndarray, k_x: int, k_h: i
 
     def cargs(c):
         if c is None:
-            return [None, None, None, 0, None]
-        return [_p(c.stamp), _p(c.n_resident), _p(c.step), c.capacity, _p(c.counters)]
+            return [None, None, None, None, 0, None]
+        return [_p(c.stamp), _p(c.count) if c.policy == "lfu" else None, _p(c.n_resident), _p(c.step), c.capacity,
+                _p(c.counters)]
 
     rc = _lib.orc_mlp_step(Wg.type, _p(Wg.w), _p(Wg.scales), _p(Wu.w), _p(Wu.scales), _p(Wd.w), _p(Wd.scales),
                            d_model, d_ff, _p(x), int(k_x), int(k_h), float(gamma),

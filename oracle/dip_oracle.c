@@ -315,13 +315,150 @@ int orc_cache_update(int32_t *stamp, int32_t *n_resident, int32_t *step,
 }
 
 /* ------------------------------------------------------------------ *
+ * The same update with the LFU policy of Sec. 5.1: a counter per column
+ * tracks how often it has been used (count[i] = number of updates whose
+ * mask contained column i since the state was created, kept whether or not
+ * the column is resident), and the most rarely used resident column is
+ * evicted.  Reading taken where the paper is silent: ties in the count go
+ * to the lower column index; the columns of the current mask are pinned and
+ * their counters are incremented by this update.  Everything else (hits,
+ * number of evictions, ascending insertion, bypass) is as in the LRU update.
+ * ------------------------------------------------------------------ */
+static int cmp_count_asc_idx_asc(const void *pa, const void *pb)
+{
+    return cmp_stamp_asc_idx_asc(pa, pb);   /* same ordering on (value, index) pairs */
+}
+
+int orc_cache_update_lfu(int32_t *stamp, int32_t *count, int32_t *n_resident, int32_t *step,
+                         int d, int capacity, const uint8_t *m, int32_t *counters)
+{
+    if (capacity < 0 || capacity > d)
+        return -1;
+    int32_t t = *step + 1;
+    int k = 0, hits = 0;
+    for (int i = 0; i < d; ++i)
+        if (m[i]) {
+            ++k;
+            if (stamp[i] >= 0)
+                ++hits;
+        }
+    int misses = k - hits;
+    int free_slots = capacity - *n_resident;
+    int n_evict = misses - free_slots;
+    if (n_evict < 0)
+        n_evict = 0;
+    int evictable = *n_resident - hits;
+    if (n_evict > evictable)
+        n_evict = evictable;
+
+    /* least frequently used first, among resident columns outside the mask */
+    orc_victim *v = (orc_victim *)malloc(sizeof(orc_victim) * (size_t)(evictable > 0 ? evictable : 1));
+    int nv = 0;
+    for (int i = 0; i < d; ++i)
+        if (!m[i] && stamp[i] >= 0) {
+            v[nv].stamp = count[i];
+            v[nv].idx = i;
+            ++nv;
+        }
+    qsort(v, (size_t)nv, sizeof(orc_victim), cmp_count_asc_idx_asc);
+    for (int e = 0; e < n_evict; ++e)
+        stamp[v[e].idx] = -1;
+    free(v);
+
+    int room = free_slots + n_evict;
+    int inserted = 0, bypassed = 0;
+    for (int i = 0; i < d; ++i) {
+        if (!m[i])
+            continue;
+        count[i] += 1;                    /* used once more */
+        if (stamp[i] >= 0) {
+            stamp[i] = t;
+        } else if (room > 0) {
+            stamp[i] = t;
+            --room;
+            ++inserted;
+        } else {
+            ++bypassed;
+        }
+    }
+    *n_resident = *n_resident - n_evict + inserted;
+    *step = t;
+    if (counters) {
+        counters[0] += hits;
+        counters[1] += misses;
+        counters[2] += n_evict;
+        counters[3] += bypassed;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ *
+ * Belady's offline policy (Sec. 5.1: with the future reads known, evict the
+ * resident column whose next use lies farthest in the future).  Replays a
+ * whole trace of masks m[T][d] through a cache of `capacity` columns with the
+ * same conventions as above (columns of the current mask pinned, ascending
+ * insertion, bypass when nothing can be evicted) and returns the hit count;
+ * misses_out (optional) receives the misses.  Ties in the next use (e.g.
+ * never used again) go to the lower index.
+ * ------------------------------------------------------------------ */
+long long orc_belady_hits(const uint8_t *m, int T, int d, int capacity, long long *misses_out)
+{
+    uint8_t *res = (uint8_t *)calloc((size_t)d, 1);
+    int n_res = 0;
+    long long hits = 0, misses = 0;
+    for (int t = 0; t < T; ++t) {
+        const uint8_t *mt = m + (size_t)t * (size_t)d;
+        for (int i = 0; i < d; ++i) {
+            if (!mt[i])
+                continue;
+            if (res[i]) {
+                ++hits;
+                continue;
+            }
+            ++misses;
+            if (n_res < capacity) {
+                res[i] = 1;
+                ++n_res;
+                continue;
+            }
+            /* victim: resident, not in the current mask, next use farthest away */
+            int victim = -1;
+            long long far = -1;
+            for (int j = 0; j < d; ++j) {
+                if (!res[j] || mt[j])
+                    continue;
+                long long next = (long long)T + 1;          /* never again */
+                for (int u = t + 1; u < T; ++u)
+                    if (m[(size_t)u * (size_t)d + (size_t)j]) {
+                        next = u;
+                        break;
+                    }
+                if (next > far) {
+                    far = next;
+                    victim = j;
+                }
+            }
+            if (victim < 0)
+                continue;                                   /* bypass */
+            res[victim] = 0;
+            res[i] = 1;
+        }
+    }
+    free(res);
+    if (misses_out)
+        *misses_out = misses;
+    return hits;
+}
+
+/* ------------------------------------------------------------------ *
  * Algorithm 1, DIP-CA for one linear layer:
  *     s = score(x, c, gamma);  m = topK(s, k);  c' = cache_update(c, m).
  * The masked weights W~ = W (.) m are not materialised; the mask is returned.
  * stamp == NULL means no cache: plain DIP (Eq. 7-8), key = |x|.
+ * count != NULL selects the LFU update, else LRU.
  * ------------------------------------------------------------------ */
 int orc_dip_ca_mask(const float *x, int d, int k, float gamma,
-                    int32_t *stamp, int32_t *n_resident, int32_t *step, int capacity,
+                    int32_t *stamp, int32_t *count, int32_t *n_resident, int32_t *step, int capacity,
                     uint8_t *m, int32_t *idx, int32_t *counters)
 {
     uint32_t *key = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)(d > 0 ? d : 1));
@@ -333,7 +470,9 @@ int orc_dip_ca_mask(const float *x, int d, int k, float gamma,
     free(key);
     if (rc)
         return rc;
-    if (stamp)
+    if (stamp && count)
+        rc = orc_cache_update_lfu(stamp, count, n_resident, step, d, capacity, m, counters);
+    else if (stamp)
         rc = orc_cache_update(stamp, n_resident, step, d, capacity, m, counters);
     return rc;
 }
@@ -366,7 +505,8 @@ void orc_masked_matvec(int type, const void *w, const uint16_t *scales,
  *   m_h = mask(h32, k_h)          [cache of the down input]
  *   y = W~d h32                                           (fp64)
  * Eq. 8 ranks |GLU~(x)|, the GLU of the already sparsified gate/up.
- * Cache arguments: stamp_* == NULL disables the cache for that input.
+ * Cache arguments: stamp_* == NULL disables the cache for that input;
+ * count_* != NULL selects LFU for it.
  * ------------------------------------------------------------------ */
 int orc_mlp_step(int type,
                  const void *Wg, const uint16_t *Sg,
@@ -374,11 +514,11 @@ int orc_mlp_step(int type,
                  const void *Wd, const uint16_t *Sd,
                  int d_model, int d_ff,
                  const float *x, int k_x, int k_h, float gamma,
-                 int32_t *stamp_gu, int32_t *nres_gu, int32_t *step_gu, int cap_gu, int32_t *ctr_gu,
-                 int32_t *stamp_d, int32_t *nres_d, int32_t *step_d, int cap_d, int32_t *ctr_d,
+                 int32_t *stamp_gu, int32_t *count_gu, int32_t *nres_gu, int32_t *step_gu, int cap_gu, int32_t *ctr_gu,
+                 int32_t *stamp_d, int32_t *count_d, int32_t *nres_d, int32_t *step_d, int cap_d, int32_t *ctr_d,
                  uint8_t *m_x, int32_t *idx_x, float *h32, uint8_t *m_h, int32_t *idx_h, double *y)
 {
-    int rc = orc_dip_ca_mask(x, d_model, k_x, gamma, stamp_gu, nres_gu, step_gu, cap_gu,
+    int rc = orc_dip_ca_mask(x, d_model, k_x, gamma, stamp_gu, count_gu, nres_gu, step_gu, cap_gu,
                              m_x, idx_x, ctr_gu);
     if (rc)
         return rc;
@@ -390,7 +530,7 @@ int orc_mlp_step(int type,
         h32[j] = (float)(u[j] * orc_silu(g[j]));
     free(g);
     free(u);
-    rc = orc_dip_ca_mask(h32, d_ff, k_h, gamma, stamp_d, nres_d, step_d, cap_d,
+    rc = orc_dip_ca_mask(h32, d_ff, k_h, gamma, stamp_d, count_d, nres_d, step_d, cap_d,
                          m_h, idx_h, ctr_d);
     if (rc)
         return rc;
