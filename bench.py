@@ -44,6 +44,7 @@ def parse_args():
     ap.add_argument("--workload", default="phi3_medium", choices=sorted(di.WORKLOADS))
     ap.add_argument("--keep-ratio", type=float, default=None)
     ap.add_argument("--cache-budget", type=float, default=None)
+    ap.add_argument("--policy", default="lru", choices=["lru", "lfu"], help="eviction policy of the column caches")
     ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging; not a valid bench)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -164,7 +165,7 @@ def build_stack(dip, ctx, torch, w, n_layers, rank):
 
 
 def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, warmup, use_graph=True,
-               kernel_pass=True, e2e_pass=True, sampler=None, dist=None):
+               kernel_pass=True, e2e_pass=True, sampler=None, dist=None, policy="lru"):
     """Time `steps` decode tokens through the stack at one (keep ratio, cache budget)."""
     L, d_model, d_ff = len(layers), w.d_model, w.d_ff
     k_x, k_h = di.keep_count(keep_ratio, d_model), di.keep_count(keep_ratio, d_ff)
@@ -174,8 +175,8 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
     def fresh_stack():
         if not ca:
             return dip.Stack(layers)
-        cg = [dip.CacheState(d_model, di.cache_capacity(budget, d_model), "cuda") for _ in range(L)]
-        cd = [dip.CacheState(d_ff, di.cache_capacity(budget, d_ff), "cuda") for _ in range(L)]
+        cg = [dip.CacheState(d_model, di.cache_capacity(budget, d_model), "cuda", policy) for _ in range(L)]
+        cd = [dip.CacheState(d_ff, di.cache_capacity(budget, d_ff), "cuda", policy) for _ in range(L)]
         return dip.Stack(layers, cg, cd)
 
     n_tok = xs_host.shape[0]
@@ -502,7 +503,7 @@ def main():
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
                            else int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])) if rank == 0 else None
     head = run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, args.steps, args.warmup,
-                      sampler=sampler, dist=dist)
+                      sampler=sampler, dist=dist, policy=args.policy)
 
     sweep = []
     if not args.no_sweep and world == 1 and w.name == "phi3_medium":
@@ -530,7 +531,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": w.name, "n_layers": L, "d_model": w.d_model, "d_ff": w.d_ff,
                    "keep_ratio": keep_ratio, "k_x": head["k_x"], "k_h": head["k_h"], "cache_budget": budget,
-                   "gamma": w.gamma if budget is not None else 1.0, "batch": 1,
+                   "gamma": w.gamma if budget is not None else 1.0, "cache_policy": args.policy, "batch": 1,
                    "step": "one decode token through %d layers = %d MLP-steps" % (L, L),
                    "l2": "inputs larger than L2: %.1f GB of distinct layer weights cycled" % (sum(l.nbytes for l in layers) / 1e9),
                    "launch": "CUDA graph of dip_stack_step", "parallelism": "replicas only"},

@@ -178,12 +178,23 @@ dip_status dip_pack_weights(dip_ctx *ctx, int wtype, int d_model, int d_ff,
  * resident in ascending index while room remains, the rest are used without
  * being cached ("bypassed", the case of Sec. 6.3 where the active set exceeds
  * the cache).
+ *
+ * LFU (Sec. 5.1, the policy of the paper's experiments): count[i] is the number
+ * of updates whose mask contained column i since the state was created (kept
+ * whether or not the column is resident); victims are the smallest
+ * (count, index) instead of the smallest (stamp, index); everything else is
+ * the same.
  * ------------------------------------------------------------------------ */
+typedef enum { DIP_CACHE_LRU = 0, DIP_CACHE_LFU = 1 } dip_cache_policy;
+
 typedef struct {
     int32_t d;          /* number of columns (input dimension of the layer) */
     int32_t capacity;   /* cache size in columns, 0 <= capacity <= d        */
     int32_t *stamp;     /* device int32[d]                                  */
     int32_t *meta;      /* device int32[DIP_CACHE_META_INTS]                */
+    int32_t *count;     /* LFU only: device int32[d] use counters, 0 when cold; NULL for LRU */
+    int32_t policy;     /* dip_cache_policy                                 */
+    int32_t reserved;
 } dip_cache_state;
 
 /* ------------------------------------------------------------------------

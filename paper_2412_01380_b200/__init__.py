@@ -34,7 +34,8 @@ class MlpWeightsStruct(C.Structure):
 
 
 class CacheStateStruct(C.Structure):
-    _fields_ = [("d", C.c_int32), ("capacity", C.c_int32), ("stamp", _vp), ("meta", _vp)]
+    _fields_ = [("d", C.c_int32), ("capacity", C.c_int32), ("stamp", _vp), ("meta", _vp), ("count", _vp),
+                ("policy", C.c_int32), ("reserved", C.c_int32)]
 
 
 class StepOutputsStruct(C.Structure):
@@ -200,11 +201,14 @@ class MlpWeights:
 class CacheState:
     """Column-cache state of one masked layer input: stamp int32[d], meta int32[8] on the device."""
 
-    def __init__(self, d: int, capacity: int, device):
-        self.d, self.capacity = int(d), int(capacity)
+    def __init__(self, d: int, capacity: int, device, policy: str = "lru"):
+        assert policy in ("lru", "lfu")
+        self.d, self.capacity, self.policy = int(d), int(capacity), policy
         self.stamp = torch.full((d,), -1, dtype=torch.int32, device=device)
         self.meta = torch.zeros(CACHE_META_INTS, dtype=torch.int32, device=device)
-        self.struct = CacheStateStruct(self.d, self.capacity, _ptr(self.stamp), _ptr(self.meta))
+        self.count = torch.zeros(d, dtype=torch.int32, device=device) if policy == "lfu" else None
+        self.struct = CacheStateStruct(self.d, self.capacity, _ptr(self.stamp), _ptr(self.meta), _ptr(self.count),
+                                       1 if policy == "lfu" else 0, 0)
 
     def load(self, stamp, n_resident: int, step: int, counters=(0, 0, 0, 0)) -> None:
         self.stamp.copy_(torch.as_tensor(stamp, dtype=torch.int32))

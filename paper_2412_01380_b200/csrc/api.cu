@@ -34,8 +34,11 @@ bool weights_ok(const dip_mlp_weights *w)
 
 bool cache_ok(const dip_cache_state *c, int d)
 {
-    return c && c->d == d && c->capacity >= 0 && c->capacity <= d && c->stamp && c->meta &&
-           dip_aligned16(c->stamp) && dip_aligned16(c->meta);
+    if (!(c && c->d == d && c->capacity >= 0 && c->capacity <= d && c->stamp && c->meta &&
+          dip_aligned16(c->stamp) && dip_aligned16(c->meta)))
+        return false;
+    if (c->policy == DIP_CACHE_LFU) return c->count && dip_aligned16(c->count);
+    return c->policy == DIP_CACHE_LRU;
 }
 
 template <typename T> dip_status dev_alloc(dip_ctx *ctx, T **p, size_t n)
@@ -183,7 +186,8 @@ static dip_status fork_cache_update(dip_ctx *ctx, int which, const uint32_t *mas
 {
     DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork[which], main));
     DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side[which], ctx->ev_fork[which], 0));
-    dip_status st = dip_launch_cache_update(ctx, mask_bits, c->d, c->stamp, c->meta, c->capacity, ctx->side[which]);
+    dip_status st = dip_launch_cache_update(ctx, mask_bits, c->d, c->stamp, c->policy == DIP_CACHE_LFU ? c->count : nullptr, c->meta,
+                                            c->capacity, ctx->side[which]);
     ctx->side_busy[which] = true;
     return st;
 }
@@ -223,7 +227,8 @@ dip_status dip_ca_mask(dip_ctx *ctx, const float *x, int d, int k, float gamma,
     cudaStream_t s = (cudaStream_t)stream;
     uint32_t *m = mask_bits ? mask_bits : ctx->mask;
     dip_status rc = dip_launch_select(ctx, x, nullptr, nullptr, 1, d, k, gamma, st->stamp, m, s);
-    if (rc == DIP_OK) rc = dip_launch_cache_update(ctx, m, d, st->stamp, st->meta, st->capacity, s);
+    if (rc == DIP_OK) rc = dip_launch_cache_update(ctx, m, d, st->stamp, st->policy == DIP_CACHE_LFU ? st->count : nullptr, st->meta,
+                                                   st->capacity, s);
     if (rc == DIP_OK && kept_idx) rc = dip_launch_mask_to_idx(ctx, m, 1, 1, d, kept_idx, k, nullptr, s);
     return rc;
 }

@@ -118,8 +118,9 @@ dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, flo
                              float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream);
 
 // topk.cu: LRU cache update from (mask, state).
-dip_status dip_launch_cache_update(dip_ctx *ctx, const uint32_t *mask_bits, int d, int32_t *stamp, int32_t *meta,
-                                   int capacity, cudaStream_t stream);
+// count != nullptr: LFU (use counters), else LRU.
+dip_status dip_launch_cache_update(dip_ctx *ctx, const uint32_t *mask_bits, int d, int32_t *stamp, int32_t *count,
+                                   int32_t *meta, int capacity, cudaStream_t stream);
 
 // topk.cu: per-device set-up of the mask kernels (dynamic shared memory limit).
 dip_status dip_init_mask_kernels(dip_ctx *ctx);

@@ -428,14 +428,14 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
 }
 
 // ---------------------------------------------------------------------------------------
-// cache_update_kernel: c' = cache_update(c, m) of Algorithm 1 with the LRU policy of Sec. 5.1,
-// from the mask bits and the state alone.  One CTA; keys[] (dynamic shared memory, d words)
+// cache_update_kernel: c' = cache_update(c, m) of Algorithm 1 with the LRU policy of Sec. 5.1
+// (or LFU when use counters are given), from the mask bits and the state alone.  One CTA; keys[] (dynamic shared memory, d words)
 // holds (resident flag << 31) | eviction key, the eviction key being the age of the column's
 // last use for columns that may be evicted (resident and outside the mask) and 0 otherwise.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(TK_THREADS, 1)
-cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stamp, int32_t *meta, int capacity,
-                    unsigned long long *tr)
+cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stamp, int32_t *count, int32_t *meta,
+                    int capacity, unsigned long long *tr)
 {
     DIP_TRACE_MIN(tr, 0);
     DIP_TRACE_MIN(tr, 1);
@@ -456,7 +456,11 @@ cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stam
         const bool keep = valid && ((mw >> lane) & 1u);
         const int st = valid ? stamp[e] : -1;
         const bool res = st >= 0;
-        if (valid) keys[e] = (res ? 0x80000000u : 0u) | ((res && !keep) ? (uint32_t)(t_now - st) : 0u);
+        // LRU: age of the last use.  LFU (count given): t + 1 - uses, so that the most rarely
+        // used column has the largest key (a column is used at most once per update: uses <= t)
+        uint32_t ek = 0u;
+        if (res && !keep) ek = count ? (uint32_t)(t_now - count[e]) : (uint32_t)(t_now - st);
+        if (valid) keys[e] = (res ? 0x80000000u : 0u) | ek;
         hits += __popc(__ballot_sync(0xffffffffu, keep && res));
         misses += __popc(mw) - __popc(__ballot_sync(0xffffffffu, keep && res));
     }
@@ -521,6 +525,7 @@ cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stam
             // a hit, or a miss that still finds room (ascending index order)
             if (!miss || (miss_before + __popc(bm & lt)) < room) stamp[e] = t_now;
         }
+        if (count && keep) count[e] += 1;       // used once more (resident or not)
         miss_before += __popc(bm);
     }
     if (tid == 0) {
@@ -620,10 +625,10 @@ dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, flo
     return DIP_OK;
 }
 
-dip_status dip_launch_cache_update(dip_ctx *ctx, const uint32_t *mask_bits, int d, int32_t *stamp, int32_t *meta,
-                                   int capacity, cudaStream_t stream)
+dip_status dip_launch_cache_update(dip_ctx *ctx, const uint32_t *mask_bits, int d, int32_t *stamp, int32_t *count,
+                                   int32_t *meta, int capacity, cudaStream_t stream)
 {
-    cache_update_kernel<<<1, TK_THREADS, (size_t)d * sizeof(uint32_t), stream>>>(mask_bits, d, stamp, meta, capacity,
+    cache_update_kernel<<<1, TK_THREADS, (size_t)d * sizeof(uint32_t), stream>>>(mask_bits, d, stamp, count, meta, capacity,
                                                                                    dip_trace_slot(ctx, 3));
     DIP_CUDA_TRY(ctx, cudaGetLastError());
     return DIP_OK;

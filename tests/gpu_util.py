@@ -59,12 +59,16 @@ def bits_to_mask(bits: torch.Tensor, d: int) -> np.ndarray:
 
 
 def gpu_cache_from_oracle(dip, c: "oracle.Cache"):
-    g = dip.CacheState(c.d, c.capacity, "cuda")
+    g = dip.CacheState(c.d, c.capacity, "cuda", c.policy)
     g.load(c.stamp, int(c.n_resident[0]), int(c.step[0]), tuple(int(v) for v in c.counters))
+    if c.policy == "lfu":
+        g.count.copy_(torch.from_numpy(c.count))
     return g
 
 
 def cache_equal(g, c: "oracle.Cache") -> bool:
     meta = g.meta.cpu().numpy()
+    if c.policy == "lfu" and not np.array_equal(g.count.cpu().numpy(), c.count):
+        return False
     return (np.array_equal(g.stamp.cpu().numpy(), c.stamp) and meta[0] == c.n_resident[0]
             and meta[1] == c.step[0] and np.array_equal(meta[2:6], c.counters))

@@ -117,6 +117,44 @@ def test_ca_mask_and_cache_state_bit_exact(dip, ctx, d, k, cap, gamma):
         assert c[3] > 0                       # and the bypass rule
 
 
+@pytest.mark.parametrize("d,k,cap,gamma", [
+    (64, 16, 32, 0.2), (3072, 768, 1536, 0.2), (5120, 1280, 2560, 0.2), (17920, 4480, 8960, 0.2),
+    (5120, 2560, 1280, 0.2), (2048, 512, 0, 0.2), (2048, 512, 2048, 0.2), (777, 100, 150, 1.0),
+])
+def test_ca_mask_lfu_policy_bit_exact(dip, ctx, d, k, cap, gamma):
+    """The LFU eviction policy (Sec. 5.1): masks, use counters and residency against the oracle."""
+    w = di.WORKLOADS["phi3_mini"].scaled(seed=2 * d + k + cap)
+    n_tok = 24
+    xs = di.token_inputs(w, n_tokens=n_tok, batch=1, d=d)[:, 0]
+    for t in range(1, n_tok):
+        xs[t] = (0.6 * xs[t - 1] + 0.8 * xs[t]).astype(np.float32)
+    ref = oracle.Cache(d, cap, "lfu")
+    g = dip.CacheState(d, cap, "cuda", "lfu")
+    bits = torch.zeros((d + 31) // 32, dtype=torch.int32, device="cuda")
+    idx = torch.zeros(k, dtype=torch.int32, device="cuda")
+    for t in range(n_tok):
+        dip.dip_ca_mask(ctx, torch.from_numpy(xs[t]).cuda(), k, gamma, g, bits, idx)
+        torch.cuda.synchronize()
+        m_ref, idx_ref = oracle.dip_ca_mask(xs[t], k, gamma, ref)
+        assert np.array_equal(bits_to_mask(bits, d), m_ref), t
+        assert np.array_equal(idx.cpu().numpy(), idx_ref), t
+        assert cache_equal(g, ref), t
+    assert ref.count.sum() == n_tok * k
+
+
+def test_stack_with_lfu_caches(dip, ctx):
+    """A small stack with LFU caches, teacher-forced per step against the oracle."""
+    d_model, d_ff = 1024, 2816
+    lw = _layer(55, d_model, d_ff, di.W_BF16)
+    w = upload_layer(dip, ctx, lw)
+    wl = di.WORKLOADS["phi3_mini"].scaled(seed=56, d_model=d_model, d_ff=d_ff)
+    xs = di.token_inputs(wl, n_tokens=6, batch=1)[:, 0]
+    ref_gu, ref_d = oracle.Cache(d_model, wl.cap_gu, "lfu"), oracle.Cache(d_ff, wl.cap_d, "lfu")
+    g_gu, g_d = dip.CacheState(d_model, wl.cap_gu, "cuda", "lfu"), dip.CacheState(d_ff, wl.cap_d, "cuda", "lfu")
+    for x in xs:
+        _check_step(dip, ctx, lw, w, x, wl.k_x, wl.k_h, wl.gamma, ref_gu, ref_d, g_gu, g_d)
+
+
 def test_ca_mask_from_saved_state_and_equal_stamps(dip, ctx):
     """Restore a state in which many resident columns share a stamp (ties in the eviction order)."""
     d, k, cap = 4096, 1024, 2048
