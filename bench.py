@@ -149,6 +149,25 @@ def whole_job_rate(units_per_rank, world, ms):
     return units_per_rank * world / (ms * 1e-3)
 
 
+def simulator_view(w, n_layers, meta_gu, meta_d, dram_gbs=60.0, flash_gbs=1.0, bytes_per_weight=0.5):
+    """The run's hit/miss counters pushed through the paper's memory model (Sec. 6, App. A: a phone
+    with DRAM 60 GB/s and Flash 1 GB/s, INT4 weights, compute ignored; MLP weights only): every
+    kept column is read from DRAM, every missed column is first loaded from Flash.  Context for
+    the paper's simulated tok/s, not a measurement of this machine."""
+    used_gu, used_d = meta_gu[2] + meta_gu[3], meta_d[2] + meta_d[3]
+    tokens = max(1, meta_gu[1] // max(1, n_layers))
+    col_gu, col_d = 2 * w.d_ff * bytes_per_weight, w.d_model * bytes_per_weight
+    dram = (used_gu * col_gu + used_d * col_d) / tokens
+    flash = (meta_gu[3] * col_gu + meta_d[3] * col_d) / tokens
+    dense = n_layers * 3 * w.d_model * w.d_ff * bytes_per_weight
+    t_sparse = dram / (dram_gbs * 1e9) + flash / (flash_gbs * 1e9)
+    # dense model with the same cache budget: the cached share from DRAM, the rest from Flash each token
+    return {"dram_gbs": dram_gbs, "flash_gbs": flash_gbs, "bytes_per_weight": bytes_per_weight,
+            "dram_bytes_per_token": dram, "flash_bytes_per_token": flash,
+            "mlp_tokens_per_s": 1.0 / t_sparse if t_sparse > 0 else None,
+            "dense_mlp_bytes_per_token": dense}
+
+
 def build_stack(dip, ctx, torch, w, n_layers, rank):
     """Draw and pack the stack's weights on the device (one canonical layer at a time)."""
     from dip_inputs import device as dd
@@ -245,8 +264,10 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
         res["union_bytes"] = ux * 2 * d_ff * ub + uh * d_model * ub
         res["union_gbs"] = res["union_bytes"] * L * steps / (ms * 1e-3) / 1e9
     if ca:
-        meta = torch.stack([c.meta for c in stack.cache_gu + stack.cache_d]).sum(0).cpu().tolist()
-        res["hit_rate"] = meta[2] / max(1, meta[2] + meta[3])
+        mg = torch.stack([c.meta for c in stack.cache_gu]).sum(0).cpu().tolist()
+        md = torch.stack([c.meta for c in stack.cache_d]).sum(0).cpu().tolist()
+        res["hit_rate"] = (mg[2] + md[2]) / max(1, mg[2] + mg[3] + md[2] + md[3])
+        res["paper_simulator_view"] = simulator_view(w, L, mg, md)
 
     # ---- end to end: host buffers in, host result out, every step ----
     if e2e_pass:
@@ -540,6 +561,7 @@ def main():
         "step_frac_of_measured_hbm": head["step_gbs"] / peak,
         "step_frac_of_nominal_8tbs": head["step_gbs"] / NOMINAL_HBM_GBS,
         "hit_rate": head.get("hit_rate"),
+        "paper_simulator_view": head.get("paper_simulator_view"),
         "clocks": head["clocks"],
         "e2e": {k: head["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
         "gpu_launches": launches_per_step * args.steps,
