@@ -44,6 +44,7 @@ def parse_args():
     ap.add_argument("--workload", default="phi3_medium", choices=sorted(di.WORKLOADS))
     ap.add_argument("--keep-ratio", type=float, default=None)
     ap.add_argument("--cache-budget", type=float, default=None)
+    ap.add_argument("--batch", type=int, default=1, help="tokens per step (batched decode; cache-aware masking off)")
     ap.add_argument("--policy", default="lru", choices=["lru", "lfu"], help="eviction policy of the column caches")
     ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging; not a valid bench)")
     ap.add_argument("--no-sweep", action="store_true")
@@ -365,7 +366,8 @@ def print_timeline(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget):
     else:
         stack = dip.Stack(layers)
     xs = xs_host.cuda()
-    x_cur, x_out = torch.empty(d_model, device="cuda"), torch.empty(d_model, device="cuda")
+    x_cur = torch.empty(tuple(xs.shape[1:]), device="cuda")
+    x_out = torch.empty_like(x_cur)
     x_cur.copy_(xs[0])
     dip.dip_stack_step(ctx, stack, x_cur, k_x, k_h, gamma, x_out)
     torch.cuda.synchronize()
@@ -516,7 +518,11 @@ def main():
     layers = build_stack(dip, ctx, torch, w, L, rank)
     n_tok = min(w.n_tokens, args.steps + args.warmup)
     wl_rank = w.scaled(seed=w.seed + 1000 * rank)
-    xs_host = torch.from_numpy(di.token_inputs(wl_rank, n_tokens=n_tok, batch=1)[:, 0].copy())
+    if args.batch > 1:
+        budget = None                                   # Algorithm 1 is per token
+        xs_host = torch.from_numpy(di.token_inputs(wl_rank, n_tokens=n_tok, batch=args.batch).copy())
+    else:
+        xs_host = torch.from_numpy(di.token_inputs(wl_rank, n_tokens=n_tok, batch=1)[:, 0].copy())
 
     if args.timeline:
         print_timeline(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget)
