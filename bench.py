@@ -547,8 +547,13 @@ def main():
 
     peak, peak_kind = measured_peak()
     gu_bytes = head["bytes"]["gate_up"]
-    gu_us = head["kernels"]["gate_up_train_us"]
-    achieved = gu_bytes / (gu_us * 1e-6) / 1e9
+    if "kernels" in head:
+        gu_us = head["kernels"]["gate_up_train_us"]
+        achieved = gu_bytes / (gu_us * 1e-6) / 1e9
+    else:
+        # batched decode: no per-kernel pass; the whole step on the bytes of the union of the masks
+        gu_us = None
+        achieved = head.get("union_gbs", head["step_gbs"])
     launches_per_step = L * (4 + (2 if budget is not None else 0)) + 1
     line = {
         "metric": METRIC, "value": whole_job_rate(L * args.steps, world, head["ms_total"]), "unit": UNIT, "n_gpus": world,
@@ -558,7 +563,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": w.name, "n_layers": L, "d_model": w.d_model, "d_ff": w.d_ff,
                    "keep_ratio": keep_ratio, "k_x": head["k_x"], "k_h": head["k_h"], "cache_budget": budget,
-                   "gamma": w.gamma if budget is not None else 1.0, "cache_policy": args.policy, "batch": 1,
+                   "gamma": w.gamma if budget is not None else 1.0, "cache_policy": args.policy, "batch": args.batch,
                    "step": "one decode token through %d layers = %d MLP-steps" % (L, L),
                    "l2": "inputs larger than L2: %.1f GB of distinct layer weights cycled" % (sum(l.nbytes for l in layers) / 1e9),
                    "launch": "CUDA graph of dip_stack_step", "parallelism": "replicas only"},
@@ -575,7 +580,8 @@ def main():
                      "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS, "bytes_per_launch": gu_bytes,
                      "us_per_launch": gu_us, "traffic": None},
-        "kernels_us": head["kernels"],
+        "kernels_us": head.get("kernels"),
+        "union_density": head.get("union_density"),
     }
     line["e2e"]["value"] *= world
     if sweep:

@@ -16,6 +16,7 @@
 //
 // which = 0 (gate/up bundle): the epilogue applies silu(gate) * up (Eq. 2).  which = 1: down.
 // Every wait on an mbarrier is bounded; on expiry the kernel records a status word and leaves.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -132,7 +133,9 @@ constexpr int GV_STAGE_BYTES = 32768;
 constexpr int GV_SCALE_STAGE_BYTES = 32768;                // INT4: shared memory for staged scale rows
 
 template <int SEG> struct __align__(16) GemvSmem {
-    unsigned char ring[GV_STAGES][GV_STAGE_BYTES];   // [stage][row][SEG]
+    // [stage][row][SEG + 16]: rows are 16 bytes apart from a multiple of 2 KB, so that the 8 row
+    // addresses of a transposing matrix load fall into different banks
+    unsigned char ring[GV_STAGES][GV_STAGE_BYTES + (GV_STAGE_BYTES / SEG) * 16];
     uint64_t full[GV_STAGES];
     uint64_t empty[GV_STAGES];
     int idx[GV_MAX_ROWS];
@@ -158,12 +161,18 @@ gemv_kernel(const GemvParams p)
     constexpr int CG = SEG / 512;                             // column groups (warps across the segment)
     constexpr int RG = GV_CONSUMER_WARPS / CG;                // row groups
     constexpr int R = GV_STAGE_BYTES / SEG;                   // rows per stage
+    constexpr int RS = SEG + 16;                              // row stride inside a stage
+    constexpr bool MMA = WT == DIP_W_BF16 && BT >= 8;         // many tokens: tensor-core path
+    constexpr int XS = GvRound<BT>::ROWS + 8;                 // MMA: stride of a token's row of values
     extern __shared__ __align__(128) unsigned char smem_raw[];
     GemvSmem<SEG> &s = *reinterpret_cast<GemvSmem<SEG> *>(smem_raw);
     constexpr int ROWS = GvRound<BT>::ROWS;                   // rows per round
     float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem<SEG>));   // [ROWS][BT]
+    // tensor-core path: the same bytes hold the values as bfloat16 pairs, [BT][XS] each
+    __nv_bfloat16 *s_xh = reinterpret_cast<__nv_bfloat16 *>(s_v);
+    __nv_bfloat16 *s_xl = s_xh + BT * XS;
     // INT4: the scale rows of the round's groups for this slab, staged once per round
-    uint16_t *s_sc = reinterpret_cast<uint16_t *>(smem_raw + sizeof(GemvSmem<SEG>) + sizeof(float) * BT * ROWS);
+    uint16_t *s_sc = reinterpret_cast<uint16_t *>(smem_raw + sizeof(GemvSmem<SEG>) + sizeof(float) * BT * (ROWS + 8));
     constexpr int SC_GROUPS = GV_SCALE_STAGE_BYTES / (SLAB * 2);   // groups that fit
     int sc_first = 0, sc_count = 0;                                  // staged groups (uniform over the CTA)
 
@@ -297,7 +306,7 @@ gemv_kernel(const GemvParams p)
                 __syncwarp();
                 for (int r = lane; r < rows_here; r += 32) {
                     const int idx = s.idx[i * R + r];
-                    bulk_g2s(&s.ring[st][r * SEG], p.W + (size_t)idx * p.row_bytes + seg_off, (unsigned)seg_bytes,
+                    bulk_g2s(&s.ring[st][r * RS], p.W + (size_t)idx * p.row_bytes + seg_off, (unsigned)seg_bytes,
                              &s.full[st]);
                 }
                 if (lane == 0) s.issued = it + 1;
@@ -329,7 +338,28 @@ gemv_kernel(const GemvParams p)
                         }
                     }
 #pragma unroll
-                    for (int b = 0; b < GB; ++b) s_v[r * BT + b0 + b] = ((mw[b] >> (idx & 31)) & 1u) ? vv[b] : 0.f;
+                    for (int b = 0; b < GB; ++b) {
+                        const float val = ((mw[b] >> (idx & 31)) & 1u) ? vv[b] : 0.f;
+                        if constexpr (MMA) {
+                            // binary32 value as two bfloat16 (value = hi + lo up to 2^-17 relative),
+                            // stored [token][row] for the B operand of the tensor-core product
+                            const __nv_bfloat16 hi = __float2bfloat16_rn(val);
+                            const __nv_bfloat16 lo = __float2bfloat16_rn(val - __bfloat162float(hi));
+                            s_xh[(b0 + b) * XS + r] = hi;
+                            s_xl[(b0 + b) * XS + r] = lo;
+                        } else {
+                            s_v[r * BT + b0 + b] = val;
+                        }
+                    }
+                }
+            }
+            if constexpr (MMA) {
+                // zero the values up to the next multiple of 16 rows (the last K step is partial)
+                const int n_pad = (n_rows + 15) & ~15;
+                for (int t = tid; t < (n_pad - n_rows) * BT; t += GV_CONSUMER_WARPS * 32) {
+                    const int b = t / (n_pad - n_rows), r = n_rows + t % (n_pad - n_rows);
+                    s_xh[b * XS + r] = __float2bfloat16_rn(0.f);
+                    s_xl[b * XS + r] = __float2bfloat16_rn(0.f);
                 }
             }
             if constexpr (WT == DIP_W_INT4_G128) {
@@ -353,7 +383,57 @@ gemv_kernel(const GemvParams p)
                 if (!mbar_wait(&s.full[st], (it / GV_STAGES) & 1)) failed = true;
                 if (failed || s.abort) { failed = true; break; }
                 const int rows_here = min(R, n_rows - i * R);
-                if (lane_ok) {
+                if constexpr (MMA) {
+                    // Tensor cores: per 16 rows, D[16 outputs][8 tokens] += A[16 outputs][16 rows] * B[16 rows][8 tokens]
+                    // with A = the stage's weights (read transposed out of shared memory) and
+                    // B = the tokens' values, once for their high and once for their low halves.
+                    constexpr int MT = SEG / 256;             // 16-output tiles per warp
+                    constexpr int NT = BT / 8;                // 8-token tiles
+                    float *macc = &acc[0][0];                 // [MT][NT][4]
+                    const int g = lane >> 2, t4 = lane & 3;
+                    for (int kb = 0; kb < rows_here; kb += 16) {
+                        uint32_t bh[NT][2], bl[NT][2];
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const int o = (nt * 8 + g) * XS + i * R + kb + 2 * t4;
+                            bh[nt][0] = *reinterpret_cast<const uint32_t *>(s_xh + o);
+                            bh[nt][1] = *reinterpret_cast<const uint32_t *>(s_xh + o + 8);
+                            bl[nt][0] = *reinterpret_cast<const uint32_t *>(s_xl + o);
+                            bl[nt][1] = *reinterpret_cast<const uint32_t *>(s_xl + o + 8);
+                        }
+                        const int left = rows_here - kb;      // valid rows of this K step
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const int m0 = (warp * MT + mt) * 16;
+                            // lane L addresses row (L & 7) of matrix L >> 3: rows kb..kb+7 / kb+8..kb+15,
+                            // outputs m0..m0+7 / m0+8..m0+15
+                            const int mrow = kb + ((lane >> 4) << 3) + (lane & 7);
+                            const int mcol = m0 + (((lane >> 3) & 1) << 3);
+                            uint32_t a0, a1, a2, a3;
+                            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3)
+                                         : "r"(smem_u32(&s.ring[st][mrow * RS + mcol * 2])));
+                            if (left < 16) {
+                                // rows past the end of the list hold stale bytes: clear them
+                                const int k0 = 2 * t4;
+                                if (k0 >= left) a0 = a1 = 0u; else if (k0 + 1 >= left) { a0 &= 0xffffu; a1 &= 0xffffu; }
+                                if (k0 + 8 >= left) a2 = a3 = 0u; else if (k0 + 9 >= left) { a2 &= 0xffffu; a3 &= 0xffffu; }
+                            }
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                float *c = macc + (mt * NT + nt) * 4;
+                                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
+                                             "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                             : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                                             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bh[nt][0]), "r"(bh[nt][1]));
+                                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
+                                             "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                             : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                                             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bl[nt][0]), "r"(bl[nt][1]));
+                            }
+                        }
+                    }
+                } else if (lane_ok) {
                     if constexpr (WT == DIP_W_INT4_G128) {
                         // W = (code - 8) * scale[group of 128 rows]: sum (code - 8) * v within a
                         // group, multiply by the group's scales when the group changes
@@ -386,7 +466,7 @@ gemv_kernel(const GemvParams p)
                                 }
                                 cur_group = g;
                             }
-                            const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * SEG + byte_off]);
+                            const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * RS + byte_off]);
                             const float xv = s_v[i * R + r];
                             const uint32_t cwd[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
@@ -402,7 +482,7 @@ gemv_kernel(const GemvParams p)
                         for (int rr = 0; rr < R / RG; ++rr) {
                             const int r = rr * RG + rg;
                             if (r < rows_here) {
-                                const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * SEG + byte_off]);
+                                const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * RS + byte_off]);
                                 float w[E];
                                 decode16<WT>(raw, w);
                                 float xv[BT];
@@ -447,29 +527,50 @@ gemv_kernel(const GemvParams p)
     float *red = reinterpret_cast<float *>(&s.ring[0][0]);    // [RG-1][CG*32 lanes][BT][E]
     float *own = red + (RG - 1) * CG * 32 * BT * E;           // [BT][SLAB] sums of this CTA, after red
     static_assert(((RG - 1) * CG * 32 * BT * E + BT * SLAB) * sizeof(float) <= sizeof(s.ring), "ring too small");
+    if constexpr (MMA) {
+        // the accumulator fragments hold whole sums already (the warps split the outputs, not the rows)
+        if (warp < GV_CONSUMER_WARPS) {
+            constexpr int MT = SEG / 256, NT = BT / 8;
+            float *dst = nparts > 1 ? p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB) : own;
+            const float *macc = &acc[0][0];
+            const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const float *c = macc + (mt * NT + nt) * 4;
+                    const int m = (warp * MT + mt) * 16 + g, n = nt * 8 + 2 * t4;
+                    dst[n * SLAB + m] = c[0];
+                    dst[(n + 1) * SLAB + m] = c[1];
+                    dst[n * SLAB + m + 8] = c[2];
+                    dst[(n + 1) * SLAB + m + 8] = c[3];
+                }
+        }
+    } else {
     if (warp < GV_CONSUMER_WARPS && rg > 0) {
 #pragma unroll
-        for (int b = 0; b < BT; ++b)
+            for (int b = 0; b < BT; ++b)
 #pragma unroll
-            for (int e = 0; e < E; ++e)
-                red[((((rg - 1) * CG + cw) * 32 + lane) * BT + b) * E + e] = acc[b][e];
-    }
-    __syncthreads();
-    if (warp < GV_CONSUMER_WARPS && rg == 0) {
-        float *dst = nparts > 1 ? p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB) : own;
+                for (int e = 0; e < E; ++e)
+                    red[((((rg - 1) * CG + cw) * 32 + lane) * BT + b) * E + e] = acc[b][e];
+        }
+        __syncthreads();
+        if (warp < GV_CONSUMER_WARPS && rg == 0) {
+            float *dst = nparts > 1 ? p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB) : own;
 #pragma unroll
-        for (int b = 0; b < BT; ++b) {
-            float sum[E];
+            for (int b = 0; b < BT; ++b) {
+                float sum[E];
 #pragma unroll
-            for (int e = 0; e < E; ++e) sum[e] = acc[b][e];
+                for (int e = 0; e < E; ++e) sum[e] = acc[b][e];
 #pragma unroll
-            for (int g = 1; g < RG; ++g)
+                for (int g = 1; g < RG; ++g)
 #pragma unroll
-                for (int e = 0; e < E; ++e) sum[e] += red[((((g - 1) * CG + cw) * 32 + lane) * BT + b) * E + e];
-            float *d = dst + b * SLAB + (cw * 32 + lane) * E;
+                    for (int e = 0; e < E; ++e) sum[e] += red[((((g - 1) * CG + cw) * 32 + lane) * BT + b) * E + e];
+                float *d = dst + b * SLAB + (cw * 32 + lane) * E;
 #pragma unroll
-            for (int e = 0; e < E; e += 4)
-                *reinterpret_cast<float4 *>(d + e) = make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
+                for (int e = 0; e < E; e += 4)
+                    *reinterpret_cast<float4 *>(d + e) = make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
+            }
         }
     }
 
@@ -562,7 +663,7 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cuda
     constexpr int SLAB = (SEG / 16) * WTraits<WT>::E;
     const size_t per_part = (size_t)n_slabs * BT * SLAB;
     if (nparts > 1 && (size_t)nparts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
-    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * GvRound<BT>::ROWS * sizeof(float) +
+    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * (GvRound<BT>::ROWS + 8) * sizeof(float) +
                         (WT == DIP_W_INT4_G128 ? GV_SCALE_STAGE_BYTES : 0);
     static bool attr_set = false;   // per instantiation
     if (!attr_set) {
