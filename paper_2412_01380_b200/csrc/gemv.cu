@@ -575,6 +575,12 @@ gemv_kernel(const GemvParams p)
     }
 
     // ---- 6. combine the parts ----
+    if (BT >= 8 && nparts > 1) {
+        // many tokens: the partial sums of a slab are too much for one CTA to add up alone;
+        // combine_parts_kernel does it right after this kernel, spread over the whole device
+        DIP_TRACE_MAX(p.tr, 2);
+        return;
+    }
     if (nparts > 1) {
         __threadfence();
         __syncthreads();
@@ -657,6 +663,52 @@ __global__ void idx_to_mask_kernel(const int32_t *__restrict__ idx, int n, int d
     }
 }
 
+// Sum of the row parts in part order and the epilogue, one thread per four outputs: the same
+// arithmetic as the last-CTA path of gemv_kernel, as a kernel of its own (used when the batch is
+// large).  partials: [nparts][n_slabs][bt][slab]; gate/up rows are interleaved in chunks of c.
+template <int WHICH>
+__global__ void __launch_bounds__(256)
+combine_parts_kernel(const float *__restrict__ partials, int nparts, int n_slabs, int bt, int slab_elems, int c,
+                     int batch, int d_out, float *__restrict__ out)
+{
+    dip_grid_dependency_wait();
+    dip_launch_dependents();
+    const int out_per_slab = WHICH == 0 ? slab_elems / 2 : slab_elems;
+    const int groups = out_per_slab / 4;
+    const long long total = (long long)n_slabs * batch * groups;
+    const size_t stride = (size_t)n_slabs * bt * slab_elems;
+    for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
+        const int o = (int)(t % groups) * 4;
+        const int b = (int)((t / groups) % batch);
+        const int slab = (int)(t / ((long long)groups * batch));
+        const int j = slab * out_per_slab + o;
+        if (j >= d_out) continue;
+        const int e0 = WHICH == 0 ? (o / c) * 2 * c + (o % c) : o;
+        const int e1 = e0 + c;
+        const float *pp = partials + ((size_t)slab * bt + b) * slab_elems;
+        float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+        for (int q0 = 0; q0 < nparts; q0 += 8) {
+            float4 a0[8], a1[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                a0[q] = a1[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (q0 + q < nparts) {
+                    a0[q] = __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(q0 + q) * stride + e0));
+                    if (WHICH == 0) a1[q] = __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(q0 + q) * stride + e1));
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                s0.x += a0[q].x; s0.y += a0[q].y; s0.z += a0[q].z; s0.w += a0[q].w;
+                s1.x += a1[q].x; s1.y += a1[q].y; s1.z += a1[q].z; s1.w += a1[q].w;
+            }
+        }
+        float4 r = s0;
+        if (WHICH == 0) r = make_float4(silu_f32(s0.x) * s1.x, silu_f32(s0.y) * s1.y, silu_f32(s0.z) * s1.z, silu_f32(s0.w) * s1.w);
+        *reinterpret_cast<float4 *>(out + (size_t)b * d_out + j) = r;
+    }
+}
+
 template <int WT, int WHICH, int BT, int SEG>
 dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cudaStream_t stream)
 {
@@ -673,6 +725,13 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cuda
     }
     dim3 grid(n_slabs, nparts);
     DIP_CUDA_TRY(ctx, dip_launch_pdl(gemv_kernel<WT, WHICH, BT, SEG>, grid, dim3(GV_THREADS), smem, stream, p));
+    if (BT >= 8 && nparts > 1) {
+        const long long groups = (long long)n_slabs * p.batch * ((WHICH == 0 ? SLAB / 2 : SLAB) / 4);
+        const int blocks = (int)((groups + 255) / 256);
+        DIP_CUDA_TRY(ctx, dip_launch_pdl(combine_parts_kernel<WHICH>, dim3(blocks), dim3(256), 0, stream,
+                                         (const float *)p.partials, nparts, n_slabs, BT, SLAB, WTraits<WT>::C, p.batch,
+                                         p.d_out, p.out));
+    }
     return DIP_OK;
 }
 
@@ -713,7 +772,7 @@ dip_status launch_bt(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t s
 {
     if (p.batch == 1) return launch_one<WT, WHICH, 1>(ctx, p, n_kept_max, stream);
     if (p.batch == 2) return launch_one<WT, WHICH, 2>(ctx, p, n_kept_max, stream);
-    if (p.batch <= 4) return launch_one<WT, WHICH, 4>(ctx, p, n_kept_max, stream);
+    if (p.batch <= 4 && WT != DIP_W_BF16) return launch_one<WT, WHICH, 4>(ctx, p, n_kept_max, stream);
     if (p.batch <= 8) return launch_one<WT, WHICH, 8>(ctx, p, n_kept_max, stream);
     return launch_one<WT, WHICH, 16>(ctx, p, n_kept_max, stream);
 }
