@@ -17,7 +17,10 @@ from . import build as _build
 W_F32, W_BF16, W_INT4_G128 = 0, 1, 2
 GROUP = 128
 
-_lib = C.CDLL(_build.build())
+import os as _os
+
+# DIP_ORACLE_LIB: load another build of the oracle (the mutation tests plant mistakes in a copy)
+_lib = C.CDLL(_os.environ.get("DIP_ORACLE_LIB") or _build.build())
 
 _vp, _i32, _f32, _f64 = C.c_void_p, C.c_int, C.c_float, C.c_double
 
