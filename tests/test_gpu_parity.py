@@ -427,6 +427,39 @@ def test_batched_step_matches_per_token_oracle(dip, ctx, batch):
     assert counts.cpu().tolist() == [n_ux, n_uh]
 
 
+def test_full_size_batched_layer(dip, ctx):
+    """Batched decode at the benchmark's shapes (Phi-3-Medium, 16 tokens, keep ratio 0.25): every
+    token's masks bit-exact, outputs of sampled tokens against the oracle, union sizes."""
+    wl = di.WORKLOADS["phi3_medium_batched"]
+    lw = di.layer_weights(wl, 0)
+    w = upload_layer(dip, ctx, lw)
+    Wg, Wu, Wd = oracle_mats(lw)
+    B, d_model, d_ff, k_x, k_h = 16, wl.d_model, wl.d_ff, wl.k_x, wl.k_h
+    x = di.token_inputs(wl, n_tokens=1, batch=B)[0]
+    dev = "cuda"
+    y = torch.empty((B, d_model), device=dev)
+    mask_x = torch.zeros((B, d_model // 32), dtype=torch.int32, device=dev)
+    mask_h = torch.zeros((B, d_ff // 32), dtype=torch.int32, device=dev)
+    h = torch.empty((B, d_ff), device=dev)
+    counts = torch.zeros(2, dtype=torch.int32, device=dev)
+    dip.dip_mlp_step(ctx, w, torch.from_numpy(x).cuda(), k_x, k_h, 1.0, None, None, y,
+                     mask_x=mask_x, h=h, mask_h=mask_h, union_counts=counts)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    mx, mh, hg, yg = bits_to_mask(mask_x, d_model), bits_to_mask(mask_h, d_ff), h.cpu().numpy(), y.cpu().numpy()
+    for b in range(B):
+        m_x, _ = oracle.dip_ca_mask(x[b], k_x)
+        assert np.array_equal(mx[b], m_x)
+        m_h, _ = oracle.dip_ca_mask(hg[b], k_h)
+        assert np.array_equal(mh[b], m_h)
+    for b in (0, 7, 15):
+        gg = oracle.masked_matvec(Wg, x[b], mx[b])
+        uu = oracle.masked_matvec(Wu, x[b], mx[b])
+        assert rel_err(hg[b], uu * gg / (1 + np.exp(-gg))) <= REL_TOL
+        assert rel_err(yg[b], oracle.masked_matvec(Wd, hg[b], mh[b])) <= REL_TOL
+    assert counts.cpu().tolist() == [oracle.mask_union(mx)[1], oracle.mask_union(mh)[1]]
+
+
 # --------------------------------------------------------------------------------------
 # argument validation: errors come back as codes, nothing is launched
 # --------------------------------------------------------------------------------------
