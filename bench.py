@@ -136,6 +136,17 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def ncu_traffic(w, keep_ratio, batch, algorithmic):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMV launch, from the ncu capture
+    summarised in profiles/kernels_phi3_medium_4layers_rho025.md (91.82 MB read + 2.51 MB written at
+    Phi-3-Medium shapes, keep ratio 0.25, one token).  Other keep ratios of the same workload scale
+    with the kept bytes (the traffic is the kept rows plus the split-row partial sums); anything
+    else has no capture."""
+    if w.name != "phi3_medium" or batch != 1:
+        return None
+    return 94.33e6 if abs(keep_ratio - 0.25) < 1e-9 else algorithmic * (94.33e6 / 91.85e6)
+
+
 def max_over_ranks(ms, dist, torch, device):
     """Slowest rank's time (the job is as fast as its slowest replica)."""
     if dist is None:
@@ -579,7 +590,7 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "gemv_kernel (gate/up bundle)", "achieved": achieved, "peak": peak,
                      "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS, "bytes_per_launch": gu_bytes,
-                     "us_per_launch": gu_us, "traffic": None},
+                     "us_per_launch": gu_us, "traffic": ncu_traffic(w, keep_ratio, args.batch, gu_bytes)},
         "kernels_us": head.get("kernels"),
         "union_density": head.get("union_density"),
     }
