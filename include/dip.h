@@ -301,6 +301,71 @@ dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *lay
                           float *x_out, float *y_last, void *stream);
 
 /* ------------------------------------------------------------------------
+ * Two-tier execution (Sec. 5 and its diagram of a single linear layer; the
+ * memory model of the evaluation in Sec. 6): the weights of a masked input
+ * live in a large slow tier, the columns the cache holds live in a small fast
+ * tier, a step reads the missing columns of its mask from the slow tier,
+ * evicts what the policy names when the fast tier is full, and multiplies with
+ * the fast tier's copy.  Here the fast tier is an arena in device memory and
+ * the slow tier is any memory the device can read: pinned, mapped host memory
+ * (reads cross the host link) or another device allocation.
+ *
+ * A dip_tier belongs to one dip_cache_state (same d, same capacity): the cache
+ * state says WHICH columns are resident, the tier says WHERE.  All buffers are
+ * the caller's.
+ *   backing  slow tier: the d packed rows of the matrix ([d][row_bytes], the
+ *            layout of dip_pack_weights: gate_up or down), device-accessible
+ *   arena    fast tier, device: (capacity + staging) rows of row_bytes; rows
+ *            0 .. capacity-1 are cache slots, the rest hold, for one step,
+ *            columns that are used without being kept (more misses than room)
+ *   slot     device int32[d]: cache slot of column i, -1 = not resident.  Must
+ *            agree with the cache state: slot[i] >= 0 exactly where
+ *            stamp[i] >= 0; start both cold (all -1)
+ *   loc      device int32[d]: scratch; arena row of each column of the current mask
+ *   fetch    device int32[4 + 2 * staging]: scratch; [0] = rows fetched this
+ *            step, then their columns, then their arena rows
+ *   split    device uint32[2][ceil(d/32)]: scratch; the mask's hits and its misses
+ *   counters device uint64[2], accumulated: rows fetched, bytes fetched
+ * Which slot a new column gets is the library's choice (the lowest free slots,
+ * in ascending column order); every choice gives the same products.
+ * INT4: the scales stay whole in device memory (dip_mlp_weights.*_scales);
+ * only the codes are tiered.
+ * ------------------------------------------------------------------------ */
+typedef struct {
+    int32_t d;
+    int32_t capacity;       /* cache slots = capacity of the matching dip_cache_state */
+    int32_t staging;        /* rows after the slots; >= the largest k used with this tier */
+    int32_t reserved;
+    uint64_t row_bytes;     /* bytes of one packed row; a multiple of 16 */
+    const void *backing;
+    void *arena;
+    int32_t *slot;
+    int32_t *loc;
+    int32_t *fetch;
+    uint32_t *split;
+    unsigned long long *counters;
+} dip_tier;
+
+/* ------------------------------------------------------------------------
+ * dip_mlp_step_tiered — dip_mlp_step for one token with both masked inputs
+ * cache-aware and their weights two-tiered.  Per input: mask (Algorithm 1's
+ * ranking), cache update, slot assignment, then the mask's hits are multiplied
+ * out of the arena while a second stream copies its misses from the slow tier
+ * into their slots; the misses' product follows and the two partial results
+ * are added in row order groups (hits first).  w gives the format and shapes
+ * (and the INT4 scales); w->gate_up and w->down are not read and may be NULL.
+ * Results equal dip_mlp_step's on the same cache states up to the order of
+ * the binary32 sums.  k_x <= tier_gu->staging and k_h <= tier_d->staging.
+ * A slot table that disagrees with the cache state (fewer free slots than
+ * columns to insert) sets the sticky device status to 2 and fetches nothing.
+ * ------------------------------------------------------------------------ */
+dip_status dip_mlp_step_tiered(dip_ctx *ctx, const dip_mlp_weights *w,
+                               const dip_tier *tier_gu, const dip_tier *tier_d,
+                               const float *x, int k_x, int k_h, float gamma,
+                               const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                               float *y, const dip_step_outputs *out, void *stream);
+
+/* ------------------------------------------------------------------------
  * dip_sparse_gemv_down_noalloc — the down product y = W~d h of
  * dip_sparse_gemv_down (batch 1, F32 or BF16 weights) for callers that are not
  * allowed to allocate device memory.  The paper has no counterpart of this

@@ -77,6 +77,18 @@ _lib.dip_stack_step.restype = _i32
 _lib.dip_stack_step.argtypes = [_vp, _i32, C.POINTER(MlpWeightsStruct), _vp, _i32, _i32, _i32, _f32,
                                 C.POINTER(CacheStateStruct), C.POINTER(CacheStateStruct), _vp, _vp, _vp]
 
+
+
+class TierStruct(C.Structure):
+    _fields_ = [("d", C.c_int32), ("capacity", C.c_int32), ("staging", C.c_int32), ("reserved", C.c_int32),
+                ("row_bytes", C.c_uint64), ("backing", _vp), ("arena", _vp), ("slot", _vp), ("loc", _vp),
+                ("fetch", _vp), ("split", _vp), ("counters", _vp)]
+
+
+_lib.dip_mlp_step_tiered.restype = _i32
+_lib.dip_mlp_step_tiered.argtypes = [_vp, C.POINTER(MlpWeightsStruct), C.POINTER(TierStruct), C.POINTER(TierStruct),
+                                     _vp, _i32, _i32, _f32, C.POINTER(CacheStateStruct),
+                                     C.POINTER(CacheStateStruct), _vp, C.POINTER(StepOutputsStruct), _vp]
 _lib.dip_sparse_gemv_down_noalloc.restype = _i32
 _lib.dip_sparse_gemv_down_noalloc.argtypes = [C.POINTER(MlpWeightsStruct), _vp, _vp, _i32, _vp, _vp]
 
@@ -84,7 +96,7 @@ EXPORTED = ["dip_create", "dip_destroy", "dip_status_string", "dip_last_error", 
             "dip_device_status", "dip_trace_begin", "dip_trace_reset", "dip_trace_read", "dip_trace_end",
             "dip_packed_bytes", "dip_pack_weights", "dip_mask_topk", "dip_ca_mask",
             "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_mlp_step",
-            "dip_residual_rmsnorm", "dip_stack_step", "dip_sparse_gemv_down_noalloc"]
+            "dip_residual_rmsnorm", "dip_stack_step", "dip_mlp_step_tiered", "dip_sparse_gemv_down_noalloc"]
 
 
 class TraceRecord(C.Structure):
@@ -92,7 +104,8 @@ class TraceRecord(C.Structure):
                 ("t_ready_ns", C.c_uint64), ("t_end_ns", C.c_uint64), ("t_aux_ns", C.c_uint64)]
 
 
-TRACE_KINDS = {1: "select", 2: "select_ca", 3: "cache_update", 4: "gemv_gate_up", 5: "gemv_down"}
+TRACE_KINDS = {1: "select", 2: "select_ca", 3: "cache_update", 4: "gemv_gate_up", 5: "gemv_down",
+               6: "tier_assign", 7: "tier_fetch"}
 for _name in ("dip_trace_begin", "dip_trace_reset", "dip_trace_end"):
     getattr(_lib, _name).restype = _i32
     getattr(_lib, _name).argtypes = [_vp]
@@ -269,6 +282,40 @@ def dip_mlp_step(ctx: Context, w: MlpWeights, x: torch.Tensor, k_x: int, k_h: in
                                 C.byref(cache_gu.struct) if cache_gu else None,
                                 C.byref(cache_d.struct) if cache_d else None,
                                 _ptr(y), C.byref(outs), _stream()))
+
+
+class Tier:
+    """Where the columns of one masked input live: `backing` holds all d packed rows (pinned host
+    memory, or a device tensor), the arena on the device holds the cache's columns.  Belongs to
+    one CacheState; both start cold."""
+
+    def __init__(self, cache: CacheState, backing: torch.Tensor, row_bytes: int, staging: int, device):
+        assert backing.dtype == torch.uint8 and backing.is_contiguous()
+        assert backing.numel() == cache.d * row_bytes
+        assert backing.is_cuda or backing.is_pinned(), "the slow tier must be readable by the device"
+        self.cache, self.backing = cache, backing
+        self.d, self.capacity, self.staging, self.row_bytes = cache.d, cache.capacity, int(staging), int(row_bytes)
+        words = (self.d + 31) // 32
+        self.arena = torch.empty((self.capacity + self.staging) * self.row_bytes, dtype=torch.uint8, device=device)
+        self.slot = torch.full((self.d,), -1, dtype=torch.int32, device=device)
+        self.loc = torch.zeros(self.d, dtype=torch.int32, device=device)
+        self.fetch = torch.zeros(4 + 2 * self.staging, dtype=torch.int32, device=device)
+        self.split = torch.zeros(2 * words, dtype=torch.int32, device=device)
+        self.counters = torch.zeros(2, dtype=torch.int64, device=device)
+        self.struct = TierStruct(self.d, self.capacity, self.staging, 0, self.row_bytes, _ptr(backing),
+                                 _ptr(self.arena), _ptr(self.slot), _ptr(self.loc), _ptr(self.fetch),
+                                 _ptr(self.split), _ptr(self.counters))
+
+
+def dip_mlp_step_tiered(ctx: Context, w: MlpWeights, tier_gu: Tier, tier_d: Tier, x: torch.Tensor,
+                        k_x: int, k_h: int, gamma: float, y: torch.Tensor,
+                        mask_x=None, idx_x=None, h=None, mask_h=None, idx_h=None) -> None:
+    """One token through one block with both inputs' weights two-tiered; the caches are the tiers'."""
+    outs = StepOutputsStruct(_ptr(mask_x), _ptr(idx_x), _ptr(h), _ptr(mask_h), _ptr(idx_h), None)
+    ctx.check(_lib.dip_mlp_step_tiered(ctx.handle, C.byref(w.struct), C.byref(tier_gu.struct),
+                                       C.byref(tier_d.struct), _ptr(x), int(k_x), int(k_h), float(gamma),
+                                       C.byref(tier_gu.cache.struct), C.byref(tier_d.cache.struct),
+                                       _ptr(y), C.byref(outs), _stream()))
 
 
 def dip_residual_rmsnorm(ctx: Context, x: torch.Tensor, y: torch.Tensor, x_next: torch.Tensor) -> None:

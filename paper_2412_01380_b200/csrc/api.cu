@@ -41,6 +41,19 @@ bool cache_ok(const dip_cache_state *c, int d)
     return c->policy == DIP_CACHE_LRU;
 }
 
+size_t packed_row_bytes(int wtype, size_t row_elems)
+{
+    return wtype == DIP_W_F32 ? row_elems * 4 : wtype == DIP_W_BF16 ? row_elems * 2 : row_elems / 2;
+}
+
+bool tier_ok(const dip_tier *t, const dip_cache_state *c, size_t row_bytes, int k)
+{
+    if (!t || !c || t->d != c->d || t->capacity != c->capacity) return false;
+    if (t->staging < k || t->row_bytes != row_bytes || (row_bytes & 15)) return false;
+    if (!t->backing || !t->arena || !t->slot || !t->loc || !t->fetch || !t->split || !t->counters) return false;
+    return dip_aligned16(t->backing) && dip_aligned16(t->arena) && dip_aligned16(t->split);
+}
+
 template <typename T> dip_status dev_alloc(dip_ctx *ctx, T **p, size_t n)
 {
     DIP_CUDA_TRY(ctx, cudaMalloc((void **)p, n * sizeof(T)));
@@ -334,6 +347,67 @@ dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
     if (!ctx) return DIP_ERR_INVALID_ARG;
     return step_impl(ctx, w, x, nullptr, nullptr, batch, k_x, k_h, gamma, cache_gu, cache_d, y, out,
                      ctx->mask, ctx->mask_h, false, stream);
+}
+
+// One masked input of the two-tier step: cache update, slot assignment, then the hits' product
+// on the main stream beside the misses' fetch on a side stream, the misses' product, the sum.
+static dip_status tiered_half(dip_ctx *ctx, const dip_mlp_weights *w, int which, const dip_tier *t,
+                              const dip_cache_state *c, const float *v, const uint32_t *mask_bits, int k,
+                              float *out, cudaStream_t s)
+{
+    dip_status st = dip_launch_cache_update(ctx, mask_bits, c->d, c->stamp, c->policy == DIP_CACHE_LFU ? c->count : nullptr,
+                                            c->meta, c->capacity, s);
+    if (st != DIP_OK) return st;
+    if ((st = dip_launch_tier_assign(ctx, t, mask_bits, c->stamp, s)) != DIP_OK) return st;
+    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork[which], s));
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side[which], ctx->ev_fork[which], 0));
+    if ((st = dip_launch_tier_fetch(ctx, t, ctx->side[which])) != DIP_OK) return st;
+    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join[which], ctx->side[which]));
+    const int words = (t->d + 31) / 32;
+    dip_gemv_rows rows = {t->arena, t->loc, 1};
+    if ((st = dip_launch_gemv(ctx, w, which, v, 1, t->split, k, out, s, &rows)) != DIP_OK) return st;
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->ev_join[which], 0));
+    rows.mode = 2;
+    return dip_launch_gemv(ctx, w, which, v, 1, t->split + words, k, out, s, &rows);
+}
+
+dip_status dip_mlp_step_tiered(dip_ctx *ctx, const dip_mlp_weights *w,
+                               const dip_tier *tier_gu, const dip_tier *tier_d,
+                               const float *x, int k_x, int k_h, float gamma,
+                               const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                               float *y, const dip_step_outputs *out, void *stream)
+{
+    if (!ctx || !w || !dims_ok(w->wtype, w->d_model, w->d_ff) || !x || !y || !dip_aligned16(x) || !dip_aligned16(y))
+        return DIP_ERR_INVALID_ARG;
+    if (w->wtype == DIP_W_INT4_G128 &&
+        (!w->gate_up_scales || !w->down_scales || !dip_aligned16(w->gate_up_scales) || !dip_aligned16(w->down_scales)))
+        return DIP_ERR_INVALID_ARG;
+    if (k_x < 1 || k_x > w->d_model || k_h < 1 || k_h > w->d_ff) return DIP_ERR_INVALID_ARG;
+    if (!(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
+    if (!cache_ok(cache_gu, w->d_model) || !cache_ok(cache_d, w->d_ff)) return DIP_ERR_INVALID_ARG;
+    if (!tier_ok(tier_gu, cache_gu, packed_row_bytes(w->wtype, (size_t)2 * w->d_ff), k_x) ||
+        !tier_ok(tier_d, cache_d, packed_row_bytes(w->wtype, (size_t)w->d_model), k_h))
+        return DIP_ERR_INVALID_ARG;
+    if (ctx->side_busy[0] || ctx->side_busy[1]) return DIP_ERR_INVALID_ARG;   // side streams are in use
+
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t *mask_x = out && out->mask_x ? out->mask_x : ctx->mask;
+    float *h = out && out->h ? out->h : ctx->h;
+    uint32_t *mask_h = out && out->mask_h ? out->mask_h : ctx->mask_h;
+    dip_status st;
+    // m_x from the cache-aware ranking (Algorithm 1), then the gate/up half out of the two tiers
+    st = dip_launch_select(ctx, x, nullptr, nullptr, 1, w->d_model, k_x, gamma, cache_gu->stamp, mask_x, s);
+    if (st != DIP_OK) return st;
+    if ((st = tiered_half(ctx, w, 0, tier_gu, cache_gu, x, mask_x, k_x, h, s)) != DIP_OK) return st;
+    // m_h likewise (Eq. 8), then the down half
+    st = dip_launch_select(ctx, h, nullptr, nullptr, 1, w->d_ff, k_h, gamma, cache_d->stamp, mask_h, s);
+    if (st != DIP_OK) return st;
+    if ((st = tiered_half(ctx, w, 1, tier_d, cache_d, h, mask_h, k_h, y, s)) != DIP_OK) return st;
+    if (out && out->idx_x && (st = dip_launch_mask_to_idx(ctx, mask_x, 1, 1, w->d_model, out->idx_x, k_x, nullptr, s)) != DIP_OK)
+        return st;
+    if (out && out->idx_h && (st = dip_launch_mask_to_idx(ctx, mask_h, 1, 1, w->d_ff, out->idx_h, k_h, nullptr, s)) != DIP_OK)
+        return st;
+    return DIP_OK;
 }
 
 dip_status dip_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y,

@@ -138,12 +138,28 @@ dip_status dip_launch_residual_rmsnorm(dip_ctx *ctx, const float *x, const float
 //   which = 0: gate/up bundle with the silu*up epilogue, out = h[batch][d_ff]
 //   which = 1: down, out = y[batch][d_model]
 // n_kept_max bounds the number of rows (sizes the row parts).
+// rows != nullptr (two-tier execution, one token): the packed row of column i is
+// base + loc[i] * row_bytes instead of row i of the weights; mode 1 leaves this launch's row parts
+// in the workspace, mode 2 adds its own behind them and then sums both launches' parts into out
+// (so that the first launch can run while the second one's rows are still being fetched).
+struct dip_gemv_rows {
+    const void *base;
+    const int32_t *loc;
+    int mode;            // 0 = a launch of its own
+};
 dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                            const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
-                           float *out, cudaStream_t stream);
+                           float *out, cudaStream_t stream, const dip_gemv_rows *rows = nullptr);
 
 // gemv.cu: bit set from an ascending index list.
 dip_status dip_launch_idx_to_mask(dip_ctx *ctx, const int32_t *idx, int n, int d, uint32_t *mask, cudaStream_t stream);
+
+// tier.cu: after the cache update of a mask: slots for the inserted columns, the step's row of
+// every kept column, the fetch list and the hit / miss split of the mask.
+dip_status dip_launch_tier_assign(dip_ctx *ctx, const dip_tier *t, const uint32_t *mask_bits, const int32_t *stamp,
+                                  cudaStream_t stream);
+// tier.cu: copy the rows of the fetch list from the slow tier into the arena.
+dip_status dip_launch_tier_fetch(dip_ctx *ctx, const dip_tier *t, cudaStream_t stream);
 
 // pack.cu
 dip_status dip_launch_pack(dip_ctx *ctx, int wtype, int d_model, int d_ff,

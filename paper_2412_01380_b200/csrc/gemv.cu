@@ -49,6 +49,9 @@ struct GemvParams {
     unsigned int *tickets;
     int *status;               // device status word (0 = fine)
     unsigned long long *tr;    // timeline slot or nullptr
+    const int32_t *loc;        // two-tier: packed row of column i is W + loc[i] * row_bytes (nullptr: row i)
+    int defer;                 // 1: leave the row parts in `partials` for combine_parts_kernel
+    int part_base;             // first part index of this launch inside `partials`
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -306,7 +309,8 @@ gemv_kernel(const GemvParams p)
                 __syncwarp();
                 for (int r = lane; r < rows_here; r += 32) {
                     const int idx = s.idx[i * R + r];
-                    bulk_g2s(&s.ring[st][r * RS], p.W + (size_t)idx * p.row_bytes + seg_off, (unsigned)seg_bytes,
+                    const int row = p.loc ? p.loc[idx] : idx;
+                    bulk_g2s(&s.ring[st][r * RS], p.W + (size_t)row * p.row_bytes + seg_off, (unsigned)seg_bytes,
                              &s.full[st]);
                 }
                 if (lane == 0) s.issued = it + 1;
@@ -524,6 +528,15 @@ gemv_kernel(const GemvParams p)
     }
     // ---- 5. combine the row groups through the (now idle) ring, in group order ----
     __syncthreads();
+    if (s.abort) {
+        // a wait ran out: let the copies already issued into this CTA's shared memory land
+        // (bounded again) before the ring is reused or the CTA leaves
+        if (tid == 0) {
+            for (int it = max(0, s.issued - GV_STAGES); it < s.issued; ++it)
+                (void)mbar_wait(&s.full[it % GV_STAGES], (it / GV_STAGES) & 1);
+        }
+        __syncthreads();
+    }
     float *red = reinterpret_cast<float *>(&s.ring[0][0]);    // [RG-1][CG*32 lanes][BT][E]
     float *own = red + (RG - 1) * CG * 32 * BT * E;           // [BT][SLAB] sums of this CTA, after red
     static_assert(((RG - 1) * CG * 32 * BT * E + BT * SLAB) * sizeof(float) <= sizeof(s.ring), "ring too small");
@@ -531,7 +544,7 @@ gemv_kernel(const GemvParams p)
         // the accumulator fragments hold whole sums already (the warps split the outputs, not the rows)
         if (warp < GV_CONSUMER_WARPS) {
             constexpr int MT = SEG / 256, NT = BT / 8;
-            float *dst = nparts > 1 ? p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB) : own;
+            float *dst = (nparts > 1 || p.defer) ? p.partials + ((size_t)(p.part_base + part) * gridDim.x + slab) * (BT * SLAB) : own;
             const float *macc = &acc[0][0];
             const int g = lane >> 2, t4 = lane & 3;
 #pragma unroll
@@ -556,7 +569,7 @@ gemv_kernel(const GemvParams p)
         }
         __syncthreads();
         if (warp < GV_CONSUMER_WARPS && rg == 0) {
-            float *dst = nparts > 1 ? p.partials + ((size_t)part * gridDim.x + slab) * (BT * SLAB) : own;
+            float *dst = (nparts > 1 || p.defer) ? p.partials + ((size_t)(p.part_base + part) * gridDim.x + slab) * (BT * SLAB) : own;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
                 float sum[E];
@@ -575,9 +588,10 @@ gemv_kernel(const GemvParams p)
     }
 
     // ---- 6. combine the parts ----
-    if (BT >= 8 && nparts > 1) {
+    if ((BT >= 8 && nparts > 1) || p.defer) {
         // many tokens: the partial sums of a slab are too much for one CTA to add up alone;
-        // combine_parts_kernel does it right after this kernel, spread over the whole device
+        // combine_parts_kernel does it right after this kernel, spread over the whole device.
+        // (Also when the caller adds the parts of two launches.)
         DIP_TRACE_MAX(p.tr, 2);
         return;
     }
@@ -595,13 +609,8 @@ gemv_kernel(const GemvParams p)
         __syncthreads();
     }
     if (s.abort) {
-        // a wait ran out: let the copies already issued into this CTA's shared memory land
-        // (bounded again) before leaving, and leave the slab's counter clean
-        if (tid == 0) {
-            for (int it = max(0, s.issued - GV_STAGES); it < s.issued; ++it)
-                (void)mbar_wait(&s.full[it % GV_STAGES], (it / GV_STAGES) & 1);
-            if (nparts > 1) p.tickets[slab] = 0;
-        }
+        // a wait ran out somewhere in this CTA: no result; leave the slab's counter clean
+        if (tid == 0 && nparts > 1) p.tickets[slab] = 0;
         return;
     }
     // four consecutive outputs per thread (16-byte loads of the partial sums)
@@ -710,11 +719,15 @@ combine_parts_kernel(const float *__restrict__ partials, int nparts, int n_slabs
 }
 
 template <int WT, int WHICH, int BT, int SEG>
-dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cudaStream_t stream)
+dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, int mode, cudaStream_t stream)
 {
     constexpr int SLAB = (SEG / 16) * WTraits<WT>::E;
     const size_t per_part = (size_t)n_slabs * BT * SLAB;
-    if (nparts > 1 && (size_t)nparts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
+    // mode 1 / 2: first / second of two launches whose row parts one combine kernel adds up
+    const int total_parts = mode ? 2 * nparts : nparts;
+    if ((nparts > 1 || mode) && (size_t)total_parts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
+    p.defer = mode != 0;
+    p.part_base = mode == 2 ? nparts : 0;
     const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * (GvRound<BT>::ROWS + 8) * sizeof(float) +
                         (WT == DIP_W_INT4_G128 ? GV_SCALE_STAGE_BYTES : 0);
     static bool attr_set = false;   // per instantiation
@@ -725,11 +738,11 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cuda
     }
     dim3 grid(n_slabs, nparts);
     DIP_CUDA_TRY(ctx, dip_launch_pdl(gemv_kernel<WT, WHICH, BT, SEG>, grid, dim3(GV_THREADS), smem, stream, p));
-    if (BT >= 8 && nparts > 1) {
+    if ((BT >= 8 && nparts > 1 && !mode) || mode == 2) {
         const long long groups = (long long)n_slabs * p.batch * ((WHICH == 0 ? SLAB / 2 : SLAB) / 4);
         const int blocks = (int)((groups + 255) / 256);
         DIP_CUDA_TRY(ctx, dip_launch_pdl(combine_parts_kernel<WHICH>, dim3(blocks), dim3(256), 0, stream,
-                                         (const float *)p.partials, nparts, n_slabs, BT, SLAB, WTraits<WT>::C, p.batch,
+                                         (const float *)p.partials, total_parts, n_slabs, BT, SLAB, WTraits<WT>::C, p.batch,
                                          p.d_out, p.out));
     }
     return DIP_OK;
@@ -741,7 +754,7 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, cuda
 // run into the copy engine's request rate (measured: 1 KB segments stream a third slower), so
 // the segment is narrowed only when that tail would get very long.
 template <int WT, int WHICH, int BT>
-dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t stream)
+dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, int mode, cudaStream_t stream)
 {
     int seg = ctx->gemv_seg;
     int n_slabs = 0, nparts = 1;
@@ -761,33 +774,36 @@ dip_status launch_one(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t 
     }
     if (n_slabs > ctx->n_tickets) return DIP_ERR_WORKSPACE;
     switch (seg) {
-    case 2048: return launch_seg<WT, WHICH, BT, 2048>(ctx, p, n_slabs, nparts, stream);
-    case 1024: return launch_seg<WT, WHICH, BT, 1024>(ctx, p, n_slabs, nparts, stream);
-    default: return launch_seg<WT, WHICH, BT, 512>(ctx, p, n_slabs, nparts, stream);
+    case 2048: return launch_seg<WT, WHICH, BT, 2048>(ctx, p, n_slabs, nparts, mode, stream);
+    case 1024: return launch_seg<WT, WHICH, BT, 1024>(ctx, p, n_slabs, nparts, mode, stream);
+    default: return launch_seg<WT, WHICH, BT, 512>(ctx, p, n_slabs, nparts, mode, stream);
     }
 }
 
 template <int WT, int WHICH>
-dip_status launch_bt(dip_ctx *ctx, GemvParams &p, int n_kept_max, cudaStream_t stream)
+dip_status launch_bt(dip_ctx *ctx, GemvParams &p, int n_kept_max, int mode, cudaStream_t stream)
 {
-    if (p.batch == 1) return launch_one<WT, WHICH, 1>(ctx, p, n_kept_max, stream);
-    if (p.batch == 2) return launch_one<WT, WHICH, 2>(ctx, p, n_kept_max, stream);
-    if (p.batch <= 4 && WT != DIP_W_BF16) return launch_one<WT, WHICH, 4>(ctx, p, n_kept_max, stream);
-    if (p.batch <= 8) return launch_one<WT, WHICH, 8>(ctx, p, n_kept_max, stream);
-    return launch_one<WT, WHICH, 16>(ctx, p, n_kept_max, stream);
+    if (p.batch == 1) return launch_one<WT, WHICH, 1>(ctx, p, n_kept_max, mode, stream);
+    if (p.batch == 2) return launch_one<WT, WHICH, 2>(ctx, p, n_kept_max, mode, stream);
+    if (p.batch <= 4 && WT != DIP_W_BF16) return launch_one<WT, WHICH, 4>(ctx, p, n_kept_max, mode, stream);
+    if (p.batch <= 8) return launch_one<WT, WHICH, 8>(ctx, p, n_kept_max, mode, stream);
+    return launch_one<WT, WHICH, 16>(ctx, p, n_kept_max, mode, stream);
 }
 
 }  // namespace
 
 dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                            const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
-                           float *out, cudaStream_t stream)
+                           float *out, cudaStream_t stream, const dip_gemv_rows *rows)
 {
+    const int mode = rows ? rows->mode : 0;
+    if (mode && batch != 1) return DIP_ERR_UNSUPPORTED;
     const bool int4 = w->wtype == DIP_W_INT4_G128;
     if (int4 && batch > 1) return DIP_ERR_UNSUPPORTED;      // the 4-bit path is single-token
     const size_t row_elems = which == 0 ? (size_t)2 * w->d_ff : (size_t)w->d_model;
     GemvParams p;
-    p.W = (const char *)(which == 0 ? w->gate_up : w->down);
+    p.W = rows ? (const char *)rows->base : (const char *)(which == 0 ? w->gate_up : w->down);
+    p.loc = rows ? rows->loc : nullptr;
     p.row_bytes = w->wtype == DIP_W_F32 ? row_elems * 4 : w->wtype == DIP_W_BF16 ? row_elems * 2 : row_elems / 2;
     p.scales = (const uint16_t *)(which == 0 ? w->gate_up_scales : w->down_scales);
     p.scale_row_elems = row_elems;
@@ -807,14 +823,14 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
         p.tr = dip_trace_slot(ctx, which == 0 ? 4 : 5);
         dip_status st;
         if (int4)
-            st = which == 0 ? launch_one<DIP_W_INT4_G128, 0, 1>(ctx, p, n_kept_max, stream)
-                            : launch_one<DIP_W_INT4_G128, 1, 1>(ctx, p, n_kept_max, stream);
+            st = which == 0 ? launch_one<DIP_W_INT4_G128, 0, 1>(ctx, p, n_kept_max, mode, stream)
+                            : launch_one<DIP_W_INT4_G128, 1, 1>(ctx, p, n_kept_max, mode, stream);
         else if (w->wtype == DIP_W_F32)
-            st = which == 0 ? launch_bt<DIP_W_F32, 0>(ctx, p, n_kept_max, stream)
-                            : launch_bt<DIP_W_F32, 1>(ctx, p, n_kept_max, stream);
+            st = which == 0 ? launch_bt<DIP_W_F32, 0>(ctx, p, n_kept_max, mode, stream)
+                            : launch_bt<DIP_W_F32, 1>(ctx, p, n_kept_max, mode, stream);
         else
-            st = which == 0 ? launch_bt<DIP_W_BF16, 0>(ctx, p, n_kept_max, stream)
-                            : launch_bt<DIP_W_BF16, 1>(ctx, p, n_kept_max, stream);
+            st = which == 0 ? launch_bt<DIP_W_BF16, 0>(ctx, p, n_kept_max, mode, stream)
+                            : launch_bt<DIP_W_BF16, 1>(ctx, p, n_kept_max, mode, stream);
         if (st != DIP_OK) return st;
     }
     return DIP_OK;

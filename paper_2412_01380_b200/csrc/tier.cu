@@ -1,0 +1,234 @@
+// Two-tier execution (Sec. 5: cached columns in a small fast memory, the rest read from a large
+// slow one on a miss).  The cache state says which columns are resident; the kernels here keep
+// the table of where they are (slots of an arena in device memory) and bring the missing ones in.
+#include "common.cuh"
+
+namespace {
+
+constexpr int TA_THREADS = 1024;
+constexpr int TA_WORDS = DIP_MAX_D / 32;
+
+struct TierParams {
+    int d, capacity, staging;
+    unsigned long long row_bytes;
+    const uint32_t *mask;      // [words] the step's mask
+    const int32_t *stamp;      // [d] cache state AFTER the step's update (>= 0: resident)
+    int32_t *slot;             // [d] in: slots before the update; out: after it
+    int32_t *loc;              // [d] out: arena row of each kept column
+    int32_t *fetch;            // out: [0] = n, [4 ..) columns, [4 + staging ..) arena rows
+    uint32_t *split;           // out: [0][words] hits, [1][words] misses
+    unsigned long long *counters;
+    int *status;
+    unsigned long long *tr;
+};
+
+// Exclusive prefix sums of three per-thread counts over the block; totals to tot[0..2].
+__device__ __forceinline__ void block_scan3(int (&v)[3], int (&pre)[3], int (*s_ws)[32], int *tot)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl[3];
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        incl[c] = v[c];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(0xffffffffu, incl[c], o);
+            if (lane >= o) incl[c] += n;
+        }
+        if (lane == 31) s_ws[c][warp] = incl[c];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        int before = 0, all = 0;
+#pragma unroll
+        for (int w = 0; w < TA_THREADS / 32; ++w) {
+            const int x = s_ws[c][w];
+            before += w < warp ? x : 0;
+            all += x;
+        }
+        pre[c] = before + incl[c] - v[c];
+        if (threadIdx.x == 0) tot[c] = all;
+    }
+    __syncthreads();
+}
+
+// One CTA.  Compares the slot table (residency before the update) with the stamps (residency
+// after it): evicted columns give up their slots, inserted columns take the lowest free slots in
+// ascending column order, kept columns that did not become resident get a staging row for this
+// step.  Writes the list of rows to fetch and splits the mask into hits and misses.
+__global__ void __launch_bounds__(TA_THREADS, 1)
+tier_assign_kernel(const TierParams t)
+{
+    __shared__ uint32_t s_before[TA_WORDS], s_after[TA_WORDS], s_occ[TA_WORDS];
+    __shared__ int s_ws[3][32];
+    __shared__ int s_tot[3];
+    __shared__ int s_bad;
+    DIP_TRACE_MIN(t.tr, 0);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int words = (t.d + 31) / 32;
+    s_occ[tid] = 0u;
+    if (tid == 0) s_bad = 0;
+    dip_grid_dependency_wait();
+    DIP_TRACE_MIN(t.tr, 1);
+    dip_launch_dependents();
+    __syncthreads();
+
+    for (int base = warp * 32; base < t.d; base += TA_THREADS) {
+        const int i = base + lane;
+        int sl = -1, st = -1;
+        if (i < t.d) {
+            sl = t.slot[i];
+            st = t.stamp[i];
+        }
+        const bool before = sl >= 0, after = st >= 0;
+        const uint32_t bw = __ballot_sync(0xffffffffu, before), aw = __ballot_sync(0xffffffffu, after);
+        if (lane == 0) {
+            s_before[base >> 5] = bw;
+            s_after[base >> 5] = aw;
+        }
+        if (before && after) {
+            if (sl < t.capacity) atomicOr(&s_occ[sl >> 5], 1u << (sl & 31));
+            else s_bad = 1;                                    // a slot outside the arena
+        }
+        if (before && !after) t.slot[i] = -1;                  // evicted
+    }
+    __syncthreads();
+
+    const int w = tid;
+    uint32_t m = 0u, B = 0u, A = 0u, fr = 0u;
+    if (w < words) {
+        m = t.mask[w];
+        B = s_before[w];
+        A = s_after[w];
+    }
+    if (w * 32 < t.capacity) {
+        fr = ~s_occ[w];
+        if (t.capacity - w * 32 < 32) fr &= (1u << (t.capacity - w * 32)) - 1u;
+    }
+    const uint32_t ins = ~B & A;           // became resident in this step
+    const uint32_t hit = m & B & A;        // kept and already there
+    const uint32_t byp = m & ~A;           // kept, not resident afterwards: one-step staging row
+    if (ins & ~m) s_bad = 1;               // only columns of the mask are ever inserted
+    int v[3] = {__popc(ins), __popc(byp), __popc(fr)}, pre[3];
+    block_scan3(v, pre, s_ws, s_tot);
+    const int n_ins = s_tot[0], n_byp = s_tot[1], n_free = s_tot[2];
+    const bool bad = s_bad || n_ins > n_free || n_ins + n_byp > t.staging;
+    int32_t *cols = t.fetch + 4, *dsts = t.fetch + 4 + t.staging;
+    if (bad) {
+        // the table and the cache state disagree: fetch nothing, multiply nothing, say so
+        if (w < words) t.split[w] = t.split[words + w] = 0u;
+        if (tid == 0) {
+            t.fetch[0] = 0;
+            atomicExch(t.status, 2);
+        }
+        DIP_TRACE_MAX(t.tr, 2);
+        return;
+    }
+    {
+        int r = pre[0];
+        for (uint32_t u = ins; u; u &= u - 1) cols[r++] = w * 32 + __ffs(u) - 1;
+        int q = pre[1];
+        for (uint32_t u = byp; u; u &= u - 1, ++q) {
+            const int i = w * 32 + __ffs(u) - 1;
+            cols[n_ins + q] = i;
+            dsts[n_ins + q] = t.capacity + q;
+            t.loc[i] = t.capacity + q;
+        }
+        for (uint32_t u = hit; u; u &= u - 1) {
+            const int i = w * 32 + __ffs(u) - 1;
+            t.loc[i] = t.slot[i];
+        }
+        int f = pre[2];
+        for (uint32_t u = fr; u && f < n_ins; u &= u - 1) dsts[f++] = w * 32 + __ffs(u) - 1;
+        if (w < words) {
+            t.split[w] = hit;
+            t.split[words + w] = m & ~hit;
+        }
+    }
+    __syncthreads();
+    for (int r = tid; r < n_ins; r += TA_THREADS) {
+        const int c = cols[r], s = dsts[r];
+        t.slot[c] = s;
+        t.loc[c] = s;
+    }
+    if (tid == 0) {
+        const int n = n_ins + n_byp;
+        t.fetch[0] = n;
+        t.counters[0] += (unsigned long long)n;
+        t.counters[1] += (unsigned long long)n * t.row_bytes;
+    }
+    DIP_TRACE_MAX(t.tr, 2);
+}
+
+constexpr int TF_THREADS = 256;
+constexpr int TF_UNROLL = 4;
+constexpr int TF_CHUNK = TF_THREADS * 16 * TF_UNROLL;     // bytes one CTA moves per turn
+
+// Copies the listed rows from the slow tier into their arena rows: a grid-stride loop over
+// (row, 16 KB chunk) units, 16 bytes per thread and four loads in flight per thread.  Plain loads:
+// the source may be host memory mapped into the device's address space.
+__global__ void __launch_bounds__(TF_THREADS)
+tier_fetch_kernel(const char *__restrict__ backing, char *__restrict__ arena, const int32_t *__restrict__ fetch,
+                  int staging, unsigned long long row_bytes, unsigned long long *tr)
+{
+    DIP_TRACE_MIN(tr, 0);
+    dip_grid_dependency_wait();
+    DIP_TRACE_MIN(tr, 1);
+    dip_launch_dependents();
+    const int n = fetch[0];
+    const int32_t *cols = fetch + 4, *dsts = fetch + 4 + staging;
+    const int cpr = (int)((row_bytes + TF_CHUNK - 1) / TF_CHUNK);
+    const long long total = (long long)n * cpr;
+    for (long long u = blockIdx.x; u < total; u += gridDim.x) {
+        const int e = (int)(u / cpr), c = (int)(u % cpr);
+        const size_t off = (size_t)c * TF_CHUNK;
+        const int vecs = (int)(min((unsigned long long)TF_CHUNK, row_bytes - off) / 16);
+        const uint4 *src = reinterpret_cast<const uint4 *>(backing + (size_t)cols[e] * row_bytes + off);
+        uint4 *dst = reinterpret_cast<uint4 *>(arena + (size_t)dsts[e] * row_bytes + off);
+        uint4 q[TF_UNROLL];
+#pragma unroll
+        for (int j = 0; j < TF_UNROLL; ++j) {
+            const int i = threadIdx.x + j * TF_THREADS;
+            if (i < vecs) q[j] = __ldcs(src + i);
+        }
+#pragma unroll
+        for (int j = 0; j < TF_UNROLL; ++j) {
+            const int i = threadIdx.x + j * TF_THREADS;
+            if (i < vecs) dst[i] = q[j];
+        }
+    }
+    DIP_TRACE_MAX(tr, 2);
+}
+
+}  // namespace
+
+dip_status dip_launch_tier_assign(dip_ctx *ctx, const dip_tier *t, const uint32_t *mask_bits, const int32_t *stamp,
+                                  cudaStream_t stream)
+{
+    TierParams p;
+    p.d = t->d;
+    p.capacity = t->capacity;
+    p.staging = t->staging;
+    p.row_bytes = t->row_bytes;
+    p.mask = mask_bits;
+    p.stamp = stamp;
+    p.slot = t->slot;
+    p.loc = t->loc;
+    p.fetch = t->fetch;
+    p.split = t->split;
+    p.counters = t->counters;
+    p.status = ctx->status;
+    p.tr = dip_trace_slot(ctx, 6);
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_assign_kernel, dim3(1), dim3(TA_THREADS), 0, stream, p));
+    return DIP_OK;
+}
+
+dip_status dip_launch_tier_fetch(dip_ctx *ctx, const dip_tier *t, cudaStream_t stream)
+{
+    unsigned long long *tr = dip_trace_slot(ctx, 7);
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_fetch_kernel, dim3(2 * ctx->sm_count), dim3(TF_THREADS), 0, stream,
+                                     (const char *)t->backing, (char *)t->arena, (const int32_t *)t->fetch, t->staging,
+                                     (unsigned long long)t->row_bytes, tr));
+    return DIP_OK;
+}

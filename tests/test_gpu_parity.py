@@ -8,8 +8,8 @@ import torch
 
 import dip_inputs as di
 import oracle
-from gpu_util import (REL_TOL, bits_to_mask, cache_equal, gpu_cache_from_oracle, oracle_mats, rel_err,
-                      upload_layer)
+from gpu_util import (REL_TOL, bits_to_mask, cache_equal, check_step, gpu_cache_from_oracle, oracle_mats,
+                      rel_err, upload_layer)
 
 pytestmark = pytest.mark.gpu
 
@@ -221,40 +221,7 @@ def test_sparse_gemvs_match_oracle(dip, ctx, wtype, d_model, d_ff, rho):
 # --------------------------------------------------------------------------------------
 # the whole step
 # --------------------------------------------------------------------------------------
-def _check_step(dip, ctx, lw, w, x, k_x, k_h, gamma, ref_gu, ref_d, g_gu, g_d):
-    """One dip_mlp_step against the oracle.  The first mask sees identical input and must be
-    bit-exact; the second mask is checked bit-exactly against the oracle's top-k of the GPU's
-    own h; outputs are compared on identical masks."""
-    d_model, d_ff = lw.d_model, lw.d_ff
-    Wg, Wu, Wd = oracle_mats(lw)
-    dev = "cuda"
-    y = torch.empty(d_model, device=dev)
-    mask_x = torch.zeros((d_model + 31) // 32, dtype=torch.int32, device=dev)
-    idx_x = torch.zeros(k_x, dtype=torch.int32, device=dev)
-    h = torch.empty(d_ff, device=dev)
-    mask_h = torch.zeros((d_ff + 31) // 32, dtype=torch.int32, device=dev)
-    idx_h = torch.zeros(k_h, dtype=torch.int32, device=dev)
-    dip.dip_mlp_step(ctx, w, torch.from_numpy(x).cuda(), k_x, k_h, gamma, g_gu, g_d, y,
-                     mask_x=mask_x, idx_x=idx_x, h=h, mask_h=mask_h, idx_h=idx_h)
-    torch.cuda.synchronize()
-    # first half
-    m_x, idx_x_ref = oracle.dip_ca_mask(x, k_x, gamma, ref_gu)
-    assert np.array_equal(bits_to_mask(mask_x, d_model), m_x)
-    assert np.array_equal(idx_x.cpu().numpy(), idx_x_ref)
-    gg = oracle.masked_matvec(Wg, x, m_x)
-    uu = oracle.masked_matvec(Wu, x, m_x)
-    h_ref = uu * gg / (1.0 + np.exp(-gg))
-    h_gpu = h.cpu().numpy()
-    assert rel_err(h_gpu, h_ref) <= REL_TOL
-    # second half, teacher-forced on the GPU's h
-    m_h, idx_h_ref = oracle.dip_ca_mask(h_gpu, k_h, gamma, ref_d)
-    assert np.array_equal(bits_to_mask(mask_h, d_ff), m_h)
-    assert np.array_equal(idx_h.cpu().numpy(), idx_h_ref)
-    y_ref = oracle.masked_matvec(Wd, h_gpu, m_h)
-    assert rel_err(y.cpu().numpy(), y_ref) <= REL_TOL
-    if ref_gu is not None:
-        assert cache_equal(g_gu, ref_gu) and cache_equal(g_d, ref_d)
-    return y.cpu().numpy()
+_check_step = check_step
 
 
 @pytest.mark.parametrize("wtype,d_model,d_ff,rho,beta", [

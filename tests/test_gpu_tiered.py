@@ -1,0 +1,158 @@
+"""GPU parity of the two-tier step (Sec. 5: cached columns in a small fast memory, misses read
+from a large slow one).  The masks, the products and the cache state must equal the oracle's
+exactly as for the single-tier step: where a column is kept is not part of the method.  What
+is particular to the tiers is checked as properties: the slot table mirrors the cache state,
+every resident column's arena row holds that column's bytes, and the rows fetched from the slow
+tier are exactly the oracle's misses."""
+import numpy as np
+import pytest
+import torch
+
+import dip_inputs as di
+import oracle
+from gpu_util import check_step, upload_layer
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dip():
+    import paper_2412_01380_b200 as m
+    return m
+
+
+@pytest.fixture(scope="module")
+def ctx(dip):
+    c = dip.Context(0)
+    yield c
+    torch.cuda.synchronize()
+    c.close()
+
+
+def _layer(seed, d_model, d_ff, wtype):
+    w = di.WORKLOADS["phi3_mini"].scaled(seed=seed, d_model=d_model, d_ff=d_ff, wtype=wtype)
+    return di.layer_weights(w, 0)
+
+
+def _tiers(dip, w, k_x, k_h, beta, policy, pinned):
+    """Caches and tiers of one block; the slow tier is a copy of the packed weights in pinned
+    host memory (or, pinned=False, a second device tensor)."""
+    d_model, d_ff = w.d_model, w.d_ff
+    g_gu = dip.CacheState(d_model, di.cache_capacity(beta, d_model), "cuda", policy)
+    g_d = dip.CacheState(d_ff, di.cache_capacity(beta, d_ff), "cuda", policy)
+    if pinned:
+        back_gu, back_d = w.gate_up.cpu().pin_memory(), w.down.cpu().pin_memory()
+    else:
+        back_gu, back_d = w.gate_up.clone(), w.down.clone()
+    t_gu = dip.Tier(g_gu, back_gu, w.gate_up.numel() // d_model, k_x, "cuda")
+    t_d = dip.Tier(g_d, back_d, w.down.numel() // d_ff, k_h, "cuda")
+    return g_gu, g_d, t_gu, t_d
+
+
+def _check_tier(t, packed, ref_cache, fetched_rows):
+    """Slot table against the cache state, arena rows against the matrix, counters against the misses."""
+    slot = t.slot.cpu().numpy()
+    resident = ref_cache.stamp >= 0
+    assert np.array_equal(slot >= 0, resident)
+    used = slot[resident]
+    assert used.size == len(set(used.tolist())) and (used < t.capacity).all()
+    rows = packed.view(t.d, t.row_bytes)
+    arena = t.arena.view(t.capacity + t.staging, t.row_bytes)
+    cols = torch.from_numpy(np.nonzero(resident)[0]).cuda()
+    assert torch.equal(arena[torch.from_numpy(used.astype(np.int64)).cuda()], rows[cols])
+    c = t.counters.cpu().numpy()
+    assert c[0] == fetched_rows and c[1] == fetched_rows * t.row_bytes
+
+
+@pytest.mark.parametrize("wtype,d_model,d_ff,rho,beta,policy,pinned", [
+    (di.W_BF16, 1024, 4096, 0.25, 0.5, "lru", True),
+    (di.W_BF16, 1024, 2048, 0.5, 0.25, "lru", True),       # k > capacity: staging rows in use
+    (di.W_BF16, 3072, 8192, 0.25, 0.5, "lfu", True),
+    (di.W_F32, 1024, 2816, 0.1, 0.25, "lru", False),
+    (di.W_INT4_G128, 1024, 2816, 0.25, 0.4, "lru", True),
+    (di.W_BF16, 512, 1536, 1.0, 0.5, "lru", False),         # every column kept every step
+])
+def test_tiered_step_matches_oracle(dip, ctx, wtype, d_model, d_ff, rho, beta, policy, pinned):
+    lw = _layer(23 + d_ff, d_model, d_ff, wtype)
+    w = upload_layer(dip, ctx, lw)
+    k_x, k_h = di.keep_count(rho, d_model), di.keep_count(rho, d_ff)
+    g_gu, g_d, t_gu, t_d = _tiers(dip, w, k_x, k_h, beta, policy, pinned)
+    ref_gu = oracle.Cache(d_model, g_gu.capacity, policy)
+    ref_d = oracle.Cache(d_ff, g_d.capacity, policy)
+    wl = di.WORKLOADS["phi3_mini"].scaled(seed=d_ff + 1)
+    xs = di.token_inputs(wl, n_tokens=8, batch=1, d=d_model)[:, 0]
+    # the two-tier step reads nothing from the single-tier weights
+    w.struct.gate_up = None
+    w.struct.down = None
+    for x in xs:
+        check_step(dip, ctx, lw, w, x, k_x, k_h, 0.2, ref_gu, ref_d, g_gu, g_d, tiers=(t_gu, t_d))
+        assert ctx.device_status() == 0
+        # counters: hits, misses, evictions, bypassed; every miss is one row read from the slow tier
+        _check_tier(t_gu, t_gu.backing.cuda(), ref_gu, int(ref_gu.counters[1]))
+        _check_tier(t_d, t_d.backing.cuda(), ref_d, int(ref_d.counters[1]))
+    assert ref_gu.counters[0] > 0 and ref_gu.counters[1] > 0      # both paths were taken
+
+
+def test_tiered_step_equals_single_tier_step(dip, ctx):
+    """Same tokens through dip_mlp_step and dip_mlp_step_tiered: identical masks and cache
+    states, outputs equal up to the order of the binary32 sums."""
+    d_model, d_ff, rho, beta = 2048, 5632, 0.25, 0.5
+    lw = _layer(5, d_model, d_ff, di.W_BF16)
+    w = upload_layer(dip, ctx, lw)
+    k_x, k_h = di.keep_count(rho, d_model), di.keep_count(rho, d_ff)
+    g_gu, g_d, t_gu, t_d = _tiers(dip, w, k_x, k_h, beta, "lru", True)
+    s_gu = dip.CacheState(d_model, g_gu.capacity, "cuda")
+    s_d = dip.CacheState(d_ff, g_d.capacity, "cuda")
+    wl = di.WORKLOADS["phi3_mini"].scaled(seed=77)
+    xs = di.token_inputs(wl, n_tokens=12, batch=1, d=d_model)[:, 0]
+    for x in xs:
+        xd = torch.from_numpy(x).cuda()
+        y1, y2 = torch.empty(d_model, device="cuda"), torch.empty(d_model, device="cuda")
+        m1 = torch.zeros((d_ff + 31) // 32, dtype=torch.int32, device="cuda")
+        m2 = torch.zeros_like(m1)
+        dip.dip_mlp_step(ctx, w, xd, k_x, k_h, 0.2, s_gu, s_d, y1, mask_h=m1)
+        dip.dip_mlp_step_tiered(ctx, w, t_gu, t_d, xd, k_x, k_h, 0.2, y2, mask_h=m2)
+        torch.cuda.synchronize()
+        if not torch.equal(m1, m2):
+            pytest.skip("a near-tie of h flipped between the two summation orders")
+        assert torch.equal(s_gu.stamp, g_gu.stamp) and torch.equal(s_d.stamp, g_d.stamp)
+        assert torch.allclose(y1, y2, rtol=1e-4, atol=1e-5 * float(y1.abs().max()))
+    assert ctx.device_status() == 0
+
+
+def test_tiered_step_flags_an_inconsistent_slot_table(dip, ctx):
+    """A slot table that disagrees with the cache state is reported through the device status
+    (2), not acted upon."""
+    d_model, d_ff = 512, 1024
+    lw = _layer(9, d_model, d_ff, di.W_BF16)
+    w = upload_layer(dip, ctx, lw)
+    k_x, k_h = 128, 256
+    c2 = dip.Context(0)
+    try:
+        g_gu, g_d, t_gu, t_d = _tiers(dip, w, k_x, k_h, 0.5, "lru", False)
+        # the cache state says its first `capacity` columns are resident, the slot table is cold
+        stamp = np.full(d_model, -1, dtype=np.int32)
+        stamp[:g_gu.capacity] = 0
+        g_gu.load(stamp, g_gu.capacity, 1)
+        x = torch.from_numpy(di.token_inputs(di.WORKLOADS["phi3_mini"].scaled(seed=3), 1, 1, d_model)[0, 0]).cuda()
+        y = torch.empty(d_model, device="cuda")
+        dip.dip_mlp_step_tiered(c2, w, t_gu, t_d, x, k_x, k_h, 0.2, y)
+        assert c2.device_status() == 2
+        assert int(t_gu.fetch[0]) == 0
+    finally:
+        torch.cuda.synchronize()
+        c2.close()
+
+
+def test_tiered_step_rejects_bad_arguments(dip, ctx):
+    d_model, d_ff = 512, 1024
+    lw = _layer(9, d_model, d_ff, di.W_BF16)
+    w = upload_layer(dip, ctx, lw)
+    g_gu, g_d, t_gu, t_d = _tiers(dip, w, 128, 256, 0.5, "lru", False)
+    x = torch.zeros(d_model, device="cuda")
+    y = torch.empty(d_model, device="cuda")
+    with pytest.raises(dip.DipError):
+        dip.dip_mlp_step_tiered(ctx, w, t_gu, t_d, x, 129, 256, 0.2, y)     # k_x beyond the staging rows
+    with pytest.raises(dip.DipError):
+        dip.dip_mlp_step_tiered(ctx, w, t_d, t_gu, x, 128, 256, 0.2, y)     # tiers swapped
+    torch.cuda.synchronize()
