@@ -51,6 +51,10 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--report", default=None, metavar="FILE",
                     help="run every workload of the five configurations (fewer steps) and write a markdown table")
+    ap.add_argument("--two-tier", action="store_true",
+                    help="time the two-tier step instead: cache arena in HBM, all weights in pinned host memory")
+    ap.add_argument("--token-correlation", type=float, default=0.0,
+                    help="mix consecutive tokens (x_t = c x_{t-1} + sqrt(1-c^2) draw); 0 = independent tokens")
     ap.add_argument("--timeline", action="store_true",
                     help="print the device-side timeline of one graph replay (per kernel: start, ready, end) and exit")
     return ap.parse_args()
@@ -364,6 +368,220 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
     return res
 
 
+def host_link_peak(torch):
+    """Bandwidth of large copies from pinned host memory to the device, measured here (GB/s)."""
+    n = 256 << 20
+    src = torch.empty(n, dtype=torch.uint8).pin_memory()
+    dst = torch.empty(n, dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        dst.copy_(src, non_blocking=True)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(4):
+        dst.copy_(src, non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    return 4 * n / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
+def print_records(recs):
+    print("%-14s %9s %9s %9s %9s %9s" % ("kernel", "start", "ready", "stream", "end", "end-ready"))
+    for r in recs:
+        print("%-14s %9.2f %9.2f %9s %9.2f %9.2f" % (r["kind"], r["start"], r["ready"],
+              "%.2f" % r["aux"] if r["aux"] is not None else "-", r["end"], r["end"] - r["ready"]))
+
+
+def run_two_tier(dip, ctx, torch, w, L, rank, xs_host, keep_ratio, budget, steps, warmup, policy, sampler=None,
+                 timeline=False):
+    """Decode tokens through a stack whose weights live in pinned host memory; each layer keeps
+    the columns its cache holds in an arena in device memory and fetches the misses of every
+    mask over the host link."""
+    from dip_inputs import device as dd
+    d_model, d_ff = w.d_model, w.d_ff
+    k_x, k_h = di.keep_count(keep_ratio, d_model), di.keep_count(keep_ratio, d_ff)
+    ws, backs = [], []
+    for l in range(L):
+        g, gs = dd.matrix(w, l, "gate", d_ff, d_model, "cuda", rank)
+        u, us = dd.matrix(w, l, "up", d_ff, d_model, "cuda", rank)
+        d_, ds = dd.matrix(w, l, "down", d_model, d_ff, "cuda", rank)
+        pw = dip.dip_pack_weights(ctx, w.wtype, d_model, d_ff, g, u, d_, gs, us, ds)
+        torch.cuda.synchronize()
+        backs.append((pw.gate_up.cpu().pin_memory(), pw.down.cpu().pin_memory()))
+        # only the shapes and the INT4 scales stay on the device
+        pw.gate_up = pw.down = None
+        pw.struct.gate_up = None
+        pw.struct.down = None
+        ws.append(pw)
+        del g, u, d_, gs, us, ds
+    torch.cuda.empty_cache()
+
+    def fresh():
+        tg, td = [], []
+        for l in range(L):
+            cg = dip.CacheState(d_model, di.cache_capacity(budget, d_model), "cuda", policy)
+            cd = dip.CacheState(d_ff, di.cache_capacity(budget, d_ff), "cuda", policy)
+            tg.append(dip.Tier(cg, backs[l][0], backs[l][0].numel() // d_model, k_x, "cuda"))
+            td.append(dip.Tier(cd, backs[l][1], backs[l][1].numel() // d_ff, k_h, "cuda"))
+        return tg, td
+
+    n_tok = xs_host.shape[0]
+    xs_dev = xs_host.cuda()
+    xa, xb = torch.empty(d_model, device="cuda"), torch.empty(d_model, device="cuda")
+    y = torch.empty(d_model, device="cuda")
+    out_host = torch.empty(d_model).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def token(tg, td):
+        cur, nxt = xa, xb
+        for l in range(L):
+            dip.dip_mlp_step_tiered(ctx, ws[l], tg[l], td[l], cur, k_x, k_h, w.gamma, y)
+            dip.dip_residual_rmsnorm(ctx, cur, y, nxt)
+            cur, nxt = nxt, cur
+        return cur
+
+    tg, td = fresh()
+    xa.copy_(xs_dev[0])
+    token(tg, td)                                    # prime outside capture
+    torch.cuda.synchronize()
+    del tg, td
+    tg, td = fresh()
+    if timeline:
+        ctx.trace_begin()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        x_last = token(tg, td)
+
+    def fetched():
+        return sum(int(t.counters[1]) for t in tg + td)
+
+    for t in range(warmup):
+        xa.copy_(xs_dev[t % n_tok], non_blocking=True)
+        graph.replay()
+    torch.cuda.synchronize()
+    if timeline:
+        ctx.trace_reset()
+        xa.copy_(xs_dev[warmup % n_tok])
+        graph.replay()
+        recs = ctx.trace_read()
+        ctx.trace_end()
+        print("# %s two-tier, keep_ratio %g cache_budget %s: one graph replay of %d layers; times in us"
+              % (w.name, keep_ratio, budget, L))
+        print_records(recs)
+        print("# per layer: %.2f us" % ((max(r["end"] for r in recs) - recs[0]["ready"]) / L))
+        return None
+    b0 = fetched()
+    m0 = [torch.stack([t.cache.meta for t in ts]).sum(0).cpu().tolist() for ts in (tg, td)]
+    if sampler:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for t in range(steps):
+        xa.copy_(xs_dev[(warmup + t) % n_tok], non_blocking=True)
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    ms = e0.elapsed_time(e1)
+    b1 = fetched()
+    m1 = [torch.stack([t.cache.meta for t in ts]).sum(0).cpu().tolist() for ts in (tg, td)]
+    hits = sum(a[2] - b[2] for a, b in zip(m1, m0))
+    misses = sum(a[3] - b[3] for a, b in zip(m1, m0))
+    # end to end: the token comes from the host and the result goes back, every step
+    xs_pin = xs_host.pin_memory()
+    n_e2e = min(steps, 64)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for t in range(n_e2e):
+        xa.copy_(xs_pin[(warmup + steps + t) % n_tok], non_blocking=True)
+        graph.replay()
+        out_host.copy_(x_last, non_blocking=True)
+        stream.synchronize()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_e = e0.elapsed_time(e1)
+    # the fetch kernel by itself: a second capture with the device-side timeline on, a few replays
+    ctx.trace_begin()
+    graph_t = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph_t):
+        token(tg, td)
+    fetch_us, fetch_bytes = 0.0, 0
+    for t in range(8):
+        xa.copy_(xs_dev[(warmup + steps + n_e2e + t) % n_tok])
+        torch.cuda.synchronize()
+        c0 = fetched()
+        ctx.trace_reset()
+        graph_t.replay()
+        recs = ctx.trace_read()
+        fetch_us += sum(r["end"] - r["ready"] for r in recs if r["kind"] == "tier_fetch")
+        fetch_bytes += fetched() - c0
+    ctx.trace_end()
+    status = ctx.device_status()
+    if status != 0:
+        raise SystemExit("device status %d after the two-tier run" % status)
+    arena = sum(t.arena.numel() for t in tg + td)
+    return {"ms_total": ms, "ms_per_step": ms / steps, "k_x": k_x, "k_h": k_h, "clocks": clocks,
+            "fetched_bytes": b1 - b0, "fetch_gbs": (b1 - b0) / (ms * 1e-3) / 1e9,
+            "fetch_kernel_gbs": fetch_bytes / max(fetch_us, 1e-9) / 1e3, "fetch_kernel_us": fetch_us / (8 * 2 * L),
+            "fetch_kernel_bytes": fetch_bytes / (8 * 2 * L),
+            "hit_rate": hits / max(1, hits + misses), "arena_bytes": arena,
+            "backing_bytes": sum(a.numel() + b.numel() for a, b in backs),
+            "e2e": {"value": L * n_e2e / (ms_e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * d_model,
+                    "d2h_bytes_per_step": 4 * d_model}}
+
+
+def main_two_tier(args, dip, ctx, torch, w, keep_ratio, budget, rank, world, local):
+    if world > 1 or args.batch > 1 or budget is None:
+        raise SystemExit("--two-tier is a single-GPU, single-token, cache-aware measurement")
+    L = args.layers if args.layers else 4
+    n_tok = min(w.n_tokens, args.steps + args.warmup + 64)
+    xs_host = torch.from_numpy(di.token_inputs(w, n_tokens=n_tok, batch=1,
+                                               correlation=args.token_correlation)[:, 0].copy())
+    link = host_link_peak(torch)
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
+                           else int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local]))
+    if args.timeline:
+        run_two_tier(dip, ctx, torch, w, L, rank, xs_host, keep_ratio, budget, args.steps, args.warmup, args.policy,
+                     timeline=True)
+        return
+    r = run_two_tier(dip, ctx, torch, w, L, rank, xs_host, keep_ratio, budget, args.steps, args.warmup, args.policy,
+                     sampler=sampler)
+    line = {
+        "metric": METRIC, "value": L * args.steps / (r["ms_total"] * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": {di.W_F32: "f32", di.W_BF16: "bf16 weights, f32 accumulate",
+                  di.W_INT4_G128: "int4 weights, f32 accumulate"}[w.wtype],
+        "data": "synthetic",
+        "config": {"workload": w.name + " two-tier: cache arena in HBM, all weights in pinned host memory",
+                   "n_layers": L, "d_model": w.d_model, "d_ff": w.d_ff, "keep_ratio": keep_ratio, "k_x": r["k_x"],
+                   "k_h": r["k_h"], "cache_budget": budget, "gamma": w.gamma, "cache_policy": args.policy,
+                   "token_correlation": args.token_correlation,
+                   "step": "one decode token through %d layers = %d MLP-steps" % (L, L),
+                   "l2": "inputs larger than L2: %.1f GB of arenas, %.1f GB of host weights"
+                         % (r["arena_bytes"] / 1e9, r["backing_bytes"] / 1e9),
+                   "launch": "CUDA graph of dip_mlp_step_tiered + dip_residual_rmsnorm per layer",
+                   "parallelism": "replicas only"},
+        "mlp_step_us": r["ms_per_step"] * 1e3 / L, "hit_rate": r["hit_rate"], "clocks": r["clocks"],
+        "e2e": r["e2e"],
+        # per layer: 2 selects, 2 cache updates, 2 slot assignments, 2 fetches, 4 GEMVs, 2 combines, 1 rmsnorm
+        "gpu_launches": 15 * L * args.steps,
+        # the fetch kernel: bytes it brought in / its own device time (timeline of 8 replays); the
+        # same bytes over the whole step's time are in fetch_gbs_over_step
+        "roofline": {"bound": "host_link", "kernel": "tier_fetch_kernel", "achieved": r["fetch_kernel_gbs"],
+                     "peak": link, "peak_kind": "of a pinned host-to-device copy measured in this run",
+                     "unit": "GB/s", "frac": r["fetch_kernel_gbs"] / link,
+                     "bytes_per_launch": r["fetch_kernel_bytes"], "us_per_launch": r["fetch_kernel_us"],
+                     "traffic": None},
+        "fetch_gbs_over_step": r["fetch_gbs"],
+        "fetched_bytes_per_mlp_step": r["fetched_bytes"] / (L * args.steps),
+    }
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = {k: v for k, v in oracle_rate(w, keep_ratio, budget, 1, 60).items()
+                                if k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line))
+
+
 def print_timeline(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget):
     """One decode token through the stack as a CUDA graph, with the library's device-side
     timeline on: per kernel, when it started, when its inputs were ready, when it ended."""
@@ -396,10 +614,7 @@ def print_timeline(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget):
     recs = ctx.trace_read()
     ctx.trace_end()
     print("# %s keep_ratio %g cache_budget %s: one graph replay of %d layers; times in us" % (w.name, keep_ratio, budget, L))
-    print("%-14s %9s %9s %9s %9s %9s" % ("kernel", "start", "ready", "stream", "end", "end-ready"))
-    for r in recs:
-        print("%-14s %9.2f %9.2f %9s %9.2f %9.2f" % (r["kind"], r["start"], r["ready"],
-              "%.2f" % r["aux"] if r["aux"] is not None else "-", r["end"], r["end"] - r["ready"]))
+    print_records(recs)
     main_path = [r for r in recs if r["kind"] != "cache_update"]
     print("# critical path per layer: %.2f us" % ((main_path[-1]["end"] - main_path[0]["ready"]) / L))
 
@@ -525,6 +740,8 @@ def main():
     if args.report:
         write_report(dip, ctx, torch, args.report, min(args.steps, 128))
         return
+    if args.two_tier:
+        return main_two_tier(args, dip, ctx, torch, w, keep_ratio, budget, rank, world, local)
     L = args.layers if args.layers else w.n_layers
     layers = build_stack(dip, ctx, torch, w, L, rank)
     n_tok = min(w.n_tokens, args.steps + args.warmup)

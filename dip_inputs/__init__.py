@@ -184,11 +184,13 @@ def layer_weights(w: Workload, layer: int) -> LayerWeights:
 # activations
 # ----------------------------------------------------------------------------
 def token_inputs(w: Workload, n_tokens: Optional[int] = None, batch: Optional[int] = None,
-                 d: Optional[int] = None) -> np.ndarray:
+                 d: Optional[int] = None, correlation: float = 0.0) -> np.ndarray:
     """First-layer inputs x_0 for every decode step: float32 [n_tokens, batch, d].
 
     student_t3: Student-t with 3 degrees of freedom, each vector scaled to unit RMS
     in fp64 and rounded to binary32.  laplace: Laplace(0, 1), rounded to binary32.
+    correlation c > 0: consecutive tokens of a sequence are mixed, x_t = c x_{t-1} +
+    sqrt(1 - c^2) draw_t (real activations are correlated over time; independent draws are not).
     """
     n = w.n_tokens if n_tokens is None else n_tokens
     b = w.batch if batch is None else batch
@@ -196,11 +198,16 @@ def token_inputs(w: Workload, n_tokens: Optional[int] = None, batch: Optional[in
     rng = _rng(w, 0, "x")
     if w.dist == "student_t3":
         v = rng.standard_t(3.0, size=(n, b, dd))
-        v /= np.sqrt((v * v).mean(axis=2, keepdims=True))
     elif w.dist == "laplace":
         v = rng.laplace(0.0, 1.0, size=(n, b, dd))
     else:
         raise ValueError(w.dist)
+    if correlation > 0.0:
+        fresh = float(np.sqrt(1.0 - correlation * correlation))
+        for t in range(1, n):
+            v[t] = correlation * v[t - 1] + fresh * v[t]
+    if w.dist == "student_t3":
+        v /= np.sqrt((v * v).mean(axis=2, keepdims=True))
     return v.astype(np.float32)
 
 

@@ -349,20 +349,26 @@ dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
                      ctx->mask, ctx->mask_h, false, stream);
 }
 
-// One masked input of the two-tier step: cache update, slot assignment, then the hits' product
-// on the main stream beside the misses' fetch on a side stream, the misses' product, the sum.
+// One masked input of the two-tier step: the hits' product on the main stream beside the cache
+// update, the slot assignment and the misses' fetch on a side stream; then the misses' product
+// and the sum of both.
 static dip_status tiered_half(dip_ctx *ctx, const dip_mlp_weights *w, int which, const dip_tier *t,
                               const dip_cache_state *c, const float *v, const uint32_t *mask_bits, int k,
                               float *out, cudaStream_t s)
 {
-    dip_status st = dip_launch_cache_update(ctx, mask_bits, c->d, c->stamp, c->policy == DIP_CACHE_LFU ? c->count : nullptr,
-                                            c->meta, c->capacity, s);
+    // the hits need neither the update nor the fetch: their product starts right away, while the
+    // side stream updates the cache, assigns slots and brings the misses in
+    dip_status st = dip_launch_tier_split(ctx, t, mask_bits, s);
     if (st != DIP_OK) return st;
-    if ((st = dip_launch_tier_assign(ctx, t, mask_bits, c->stamp, s)) != DIP_OK) return st;
+    cudaStream_t side = ctx->side[which];
     DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork[which], s));
-    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side[which], ctx->ev_fork[which], 0));
-    if ((st = dip_launch_tier_fetch(ctx, t, ctx->side[which])) != DIP_OK) return st;
-    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join[which], ctx->side[which]));
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(side, ctx->ev_fork[which], 0));
+    st = dip_launch_cache_update(ctx, mask_bits, c->d, c->stamp, c->policy == DIP_CACHE_LFU ? c->count : nullptr,
+                                 c->meta, c->capacity, side);
+    if (st != DIP_OK) return st;
+    if ((st = dip_launch_tier_assign(ctx, t, mask_bits, c->stamp, side)) != DIP_OK) return st;
+    if ((st = dip_launch_tier_fetch(ctx, t, side)) != DIP_OK) return st;
+    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join[which], side));
     const int words = (t->d + 31) / 32;
     dip_gemv_rows rows = {t->arena, t->loc, 1};
     if ((st = dip_launch_gemv(ctx, w, which, v, 1, t->split, k, out, s, &rows)) != DIP_OK) return st;

@@ -154,8 +154,11 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
 // gemv.cu: bit set from an ascending index list.
 dip_status dip_launch_idx_to_mask(dip_ctx *ctx, const int32_t *idx, int n, int d, uint32_t *mask, cudaStream_t stream);
 
-// tier.cu: after the cache update of a mask: slots for the inserted columns, the step's row of
-// every kept column, the fetch list and the hit / miss split of the mask.
+// tier.cu: before the cache update of a mask: its hits (resident columns, with their arena rows)
+// and its misses.
+dip_status dip_launch_tier_split(dip_ctx *ctx, const dip_tier *t, const uint32_t *mask_bits, cudaStream_t stream);
+// tier.cu: after the cache update: slots for the inserted columns, the step's arena row of every
+// miss, and the fetch list.
 dip_status dip_launch_tier_assign(dip_ctx *ctx, const dip_tier *t, const uint32_t *mask_bits, const int32_t *stamp,
                                   cudaStream_t stream);
 // tier.cu: copy the rows of the fetch list from the slow tier into the arena.

@@ -135,13 +135,15 @@ __device__ __forceinline__ float half_bits_to_float(uint16_t h)
 constexpr int GV_STAGE_BYTES = 32768;
 constexpr int GV_SCALE_STAGE_BYTES = 32768;                // INT4: shared memory for staged scale rows
 
+static_assert(DIP_MAX_D <= 32768, "the row lists in shared memory are 16-bit");
 template <int SEG> struct __align__(16) GemvSmem {
     // [stage][row][SEG + 16]: rows are 16 bytes apart from a multiple of 2 KB, so that the 8 row
     // addresses of a transposing matrix load fall into different banks
     unsigned char ring[GV_STAGES][GV_STAGE_BYTES + (GV_STAGE_BYTES / SEG) * 16];
     uint64_t full[GV_STAGES];
     uint64_t empty[GV_STAGES];
-    int idx[GV_MAX_ROWS];
+    uint16_t idx[GV_MAX_ROWS];   // the round's columns (< DIP_MAX_D = 2^15)
+    uint16_t row[GV_MAX_ROWS];   // two-tier: the arena row of each (< 2 * DIP_MAX_D = 2^16)
     uint32_t words[DIP_MAX_D / 32];
     int pre[DIP_MAX_D / 32];
     int wsum[GV_SCAN_THREADS / 32];
@@ -286,12 +288,17 @@ gemv_kernel(const GemvParams p)
                 while (u) {
                     const int bit = __ffs(u) - 1;
                     u &= u - 1;
-                    if (rank >= lo_rank && rank < hi_rank) s.idx[rank - lo_rank] = w * 32 + bit;
+                    if (rank >= lo_rank && rank < hi_rank) s.idx[rank - lo_rank] = (uint16_t)(w * 32 + bit);
                     ++rank;
                 }
             }
         }
         __syncthreads();
+        if (p.loc) {
+            // two-tier: look the rows' places up together, ahead of the copies
+            for (int r = tid; r < n_rows; r += GV_THREADS) s.row[r] = (uint16_t)p.loc[s.idx[r]];
+            __syncthreads();
+        }
         const int n_stages = (n_rows + R - 1) / R;
 
         if (warp == GV_CONSUMER_WARPS) {
@@ -308,8 +315,7 @@ gemv_kernel(const GemvParams p)
                 if (lane == 0) mbar_expect_tx(&s.full[st], (unsigned)(rows_here * seg_bytes));
                 __syncwarp();
                 for (int r = lane; r < rows_here; r += 32) {
-                    const int idx = s.idx[i * R + r];
-                    const int row = p.loc ? p.loc[idx] : idx;
+                    const int row = p.loc ? s.row[i * R + r] : s.idx[i * R + r];
                     bulk_g2s(&s.ring[st][r * RS], p.W + (size_t)row * p.row_bytes + seg_off, (unsigned)seg_bytes,
                              &s.full[st]);
                 }

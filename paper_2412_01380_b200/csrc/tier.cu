@@ -14,9 +14,9 @@ struct TierParams {
     const uint32_t *mask;      // [words] the step's mask
     const int32_t *stamp;      // [d] cache state AFTER the step's update (>= 0: resident)
     int32_t *slot;             // [d] in: slots before the update; out: after it
-    int32_t *loc;              // [d] out: arena row of each kept column
+    int32_t *loc;              // [d] out: arena row of each kept column that was not resident
     int32_t *fetch;            // out: [0] = n, [4 ..) columns, [4 + staging ..) arena rows
-    uint32_t *split;           // out: [0][words] hits, [1][words] misses
+    uint32_t *split;           // [0][words] hits, [1][words] misses (written by tier_split_kernel)
     unsigned long long *counters;
     int *status;
     unsigned long long *tr;
@@ -53,10 +53,37 @@ __device__ __forceinline__ void block_scan3(int (&v)[3], int (&pre)[3], int (*s_
     __syncthreads();
 }
 
+// Before the cache update: the columns of the mask that are resident (hits) can be multiplied
+// right away, out of the slots they are in; the others (misses) have to be fetched first.
+// One thread per column, one mask word per warp.
+__global__ void __launch_bounds__(256)
+tier_split_kernel(const uint32_t *__restrict__ mask, const int32_t *__restrict__ slot, int32_t *__restrict__ loc,
+                  uint32_t *__restrict__ split, int d, unsigned long long *tr)
+{
+    DIP_TRACE_MIN(tr, 0);
+    dip_grid_dependency_wait();
+    DIP_TRACE_MIN(tr, 1);
+    dip_launch_dependents();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int words = (d + 31) / 32, w = i >> 5;
+    if (w < words) {                                           // whole warps: d is a multiple of 32
+        const uint32_t m = mask[w];
+        const int sl = i < d ? slot[i] : -1;
+        const bool hit = ((m >> (i & 31)) & 1u) && sl >= 0;
+        if (hit) loc[i] = sl;
+        const uint32_t hw = __ballot_sync(0xffffffffu, hit);
+        if ((i & 31) == 0) {
+            split[w] = hw;
+            split[words + w] = m & ~hw;
+        }
+    }
+    DIP_TRACE_MAX(tr, 2);
+}
+
 // One CTA.  Compares the slot table (residency before the update) with the stamps (residency
 // after it): evicted columns give up their slots, inserted columns take the lowest free slots in
 // ascending column order, kept columns that did not become resident get a staging row for this
-// step.  Writes the list of rows to fetch and splits the mask into hits and misses.
+// step.  Writes the list of rows to fetch.
 __global__ void __launch_bounds__(TA_THREADS, 1)
 tier_assign_kernel(const TierParams t)
 {
@@ -74,24 +101,32 @@ tier_assign_kernel(const TierParams t)
     dip_launch_dependents();
     __syncthreads();
 
-    for (int base = warp * 32; base < t.d; base += TA_THREADS) {
-        const int i = base + lane;
-        int sl = -1, st = -1;
-        if (i < t.d) {
-            sl = t.slot[i];
-            st = t.stamp[i];
+    constexpr int TU = 8;                  // iterations whose loads are issued together
+    for (int base0 = warp * 32; base0 < t.d; base0 += TA_THREADS * TU) {
+        int slv[TU], stv[TU];
+#pragma unroll
+        for (int u = 0; u < TU; ++u) {
+            const int i = base0 + u * TA_THREADS + lane;
+            slv[u] = i < t.d ? t.slot[i] : -1;
+            stv[u] = i < t.d ? t.stamp[i] : -1;
         }
-        const bool before = sl >= 0, after = st >= 0;
-        const uint32_t bw = __ballot_sync(0xffffffffu, before), aw = __ballot_sync(0xffffffffu, after);
-        if (lane == 0) {
-            s_before[base >> 5] = bw;
-            s_after[base >> 5] = aw;
+#pragma unroll
+        for (int u = 0; u < TU; ++u) {
+            const int base = base0 + u * TA_THREADS, i = base + lane;
+            if (base >= t.d) break;                            // uniform over the warp
+            const int sl = slv[u];
+            const bool before = sl >= 0, after = stv[u] >= 0;
+            const uint32_t bw = __ballot_sync(0xffffffffu, before), aw = __ballot_sync(0xffffffffu, after);
+            if (lane == 0) {
+                s_before[base >> 5] = bw;
+                s_after[base >> 5] = aw;
+            }
+            if (before && after) {
+                if (sl < t.capacity) atomicOr(&s_occ[sl >> 5], 1u << (sl & 31));
+                else s_bad = 1;                                // a slot outside the arena
+            }
+            if (before && !after) t.slot[i] = -1;              // evicted
         }
-        if (before && after) {
-            if (sl < t.capacity) atomicOr(&s_occ[sl >> 5], 1u << (sl & 31));
-            else s_bad = 1;                                    // a slot outside the arena
-        }
-        if (before && !after) t.slot[i] = -1;                  // evicted
     }
     __syncthreads();
 
@@ -107,17 +142,16 @@ tier_assign_kernel(const TierParams t)
         if (t.capacity - w * 32 < 32) fr &= (1u << (t.capacity - w * 32)) - 1u;
     }
     const uint32_t ins = ~B & A;           // became resident in this step
-    const uint32_t hit = m & B & A;        // kept and already there
     const uint32_t byp = m & ~A;           // kept, not resident afterwards: one-step staging row
-    if (ins & ~m) s_bad = 1;               // only columns of the mask are ever inserted
+    if ((ins & ~m) | (byp & B)) s_bad = 1; // only columns of the mask are inserted; its hits stay
     int v[3] = {__popc(ins), __popc(byp), __popc(fr)}, pre[3];
     block_scan3(v, pre, s_ws, s_tot);
     const int n_ins = s_tot[0], n_byp = s_tot[1], n_free = s_tot[2];
     const bool bad = s_bad || n_ins > n_free || n_ins + n_byp > t.staging;
     int32_t *cols = t.fetch + 4, *dsts = t.fetch + 4 + t.staging;
     if (bad) {
-        // the table and the cache state disagree: fetch nothing, multiply nothing, say so
-        if (w < words) t.split[w] = t.split[words + w] = 0u;
+        // the table and the cache state disagree: fetch nothing, multiply no fetched row, say so
+        if (w < words) t.split[words + w] = 0u;
         if (tid == 0) {
             t.fetch[0] = 0;
             atomicExch(t.status, 2);
@@ -135,16 +169,8 @@ tier_assign_kernel(const TierParams t)
             dsts[n_ins + q] = t.capacity + q;
             t.loc[i] = t.capacity + q;
         }
-        for (uint32_t u = hit; u; u &= u - 1) {
-            const int i = w * 32 + __ffs(u) - 1;
-            t.loc[i] = t.slot[i];
-        }
         int f = pre[2];
         for (uint32_t u = fr; u && f < n_ins; u &= u - 1) dsts[f++] = w * 32 + __ffs(u) - 1;
-        if (w < words) {
-            t.split[w] = hit;
-            t.split[words + w] = m & ~hit;
-        }
     }
     __syncthreads();
     for (int r = tid; r < n_ins; r += TA_THREADS) {
@@ -221,6 +247,14 @@ dip_status dip_launch_tier_assign(dip_ctx *ctx, const dip_tier *t, const uint32_
     p.status = ctx->status;
     p.tr = dip_trace_slot(ctx, 6);
     DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_assign_kernel, dim3(1), dim3(TA_THREADS), 0, stream, p));
+    return DIP_OK;
+}
+
+dip_status dip_launch_tier_split(dip_ctx *ctx, const dip_tier *t, const uint32_t *mask_bits, cudaStream_t stream)
+{
+    unsigned long long *tr = dip_trace_slot(ctx, 8);
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_split_kernel, dim3((t->d + 255) / 256), dim3(256), 0, stream, mask_bits,
+                                     (const int32_t *)t->slot, t->loc, t->split, (int)t->d, tr));
     return DIP_OK;
 }
 

@@ -449,20 +449,36 @@ cache_update_kernel(const uint32_t *__restrict__ mask_bits, int d, int32_t *stam
     const unsigned lt = lanemask_lt();
 
     int hits = 0, misses = 0;
-    for (int it = 0; it < span && base + it < d; it += 32) {
-        const int e = base + it + lane;
-        const bool valid = e < d;
-        const unsigned mw = mask_bits[(base + it) >> 5];
-        const bool keep = valid && ((mw >> lane) & 1u);
-        const int st = valid ? stamp[e] : -1;
-        const bool res = st >= 0;
-        // LRU: age of the last use.  LFU (count given): t + 1 - uses, so that the most rarely
-        // used column has the largest key (a column is used at most once per update: uses <= t)
-        uint32_t ek = 0u;
-        if (res && !keep) ek = count ? (uint32_t)(t_now - count[e]) : (uint32_t)(t_now - st);
-        if (valid) keys[e] = (res ? 0x80000000u : 0u) | ek;
-        hits += __popc(__ballot_sync(0xffffffffu, keep && res));
-        misses += __popc(mw) - __popc(__ballot_sync(0xffffffffu, keep && res));
+    constexpr int CU = 8;             // iterations whose loads are issued together
+    for (int it0 = 0; it0 < span && base + it0 < d; it0 += 32 * CU) {
+        unsigned mwv[CU];
+        int stv[CU], cnv[CU];
+#pragma unroll
+        for (int u = 0; u < CU; ++u) {
+            const int it = it0 + 32 * u, e = base + it + lane;
+            const bool in_span = it < span && base + it < d;
+            mwv[u] = in_span ? mask_bits[(base + it) >> 5] : 0u;
+            stv[u] = in_span && e < d ? stamp[e] : -1;
+            cnv[u] = count && in_span && e < d ? count[e] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < CU; ++u) {
+            const int it = it0 + 32 * u, e = base + it + lane;
+            if (!(it < span && base + it < d)) break;          // uniform over the warp
+            const bool valid = e < d;
+            const unsigned mw = mwv[u];
+            const bool keep = valid && ((mw >> lane) & 1u);
+            const int st = stv[u];
+            const bool res = st >= 0;
+            // LRU: age of the last use.  LFU (count given): t + 1 - uses, so that the most rarely
+            // used column has the largest key (a column is used at most once per update: uses <= t)
+            uint32_t ek = 0u;
+            if (res && !keep) ek = count ? (uint32_t)(t_now - cnv[u]) : (uint32_t)(t_now - st);
+            if (valid) keys[e] = (res ? 0x80000000u : 0u) | ek;
+            const int hw = __popc(__ballot_sync(0xffffffffu, keep && res));
+            hits += hw;
+            misses += __popc(mw) - hw;
+        }
     }
     if (lane == 0) {
         s.wa[warp] = hits;
