@@ -50,6 +50,9 @@ _lib.orc_dense_mlp.argtypes = [_i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _
 _lib.orc_mlp_step.restype = _i32
 _lib.orc_mlp_step.argtypes = ([_i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _i32, _f32]
                               + [_vp, _vp, _vp, _vp, _i32, _vp] * 2 + [_vp] * 6)
+_lib.orc_neuron_pruned_step.restype = _i32
+_lib.orc_neuron_pruned_step.argtypes = [_i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _i32,
+                                        _vp, _vp, _vp, _vp, _vp]
 _lib.orc_residual_rmsnorm.restype = None
 _lib.orc_residual_rmsnorm.argtypes = [_vp, _vp, _i32, _vp]
 _lib.orc_mask_union.restype = _i32
@@ -243,6 +246,30 @@ def mlp_step(Wg: Matrix, Wu: Matrix, Wd: Matrix, x: np.ndarray, k_x: int, k_h: i
                            _p(r.m_x), _p(r.idx_x), _p(r.h32), _p(r.m_h), _p(r.idx_h), _p(r.y))
     if rc:
         raise ValueError("invalid k or capacity")
+    return r
+
+
+@dataclass
+class NeuronPrunedResult:
+    p32: np.ndarray
+    m: np.ndarray
+    idx: np.ndarray
+    h32: np.ndarray
+    y: np.ndarray
+
+
+def neuron_pruned_step(Wg: Matrix, Wu: Matrix, Wd: Matrix, x: np.ndarray, k: int, by: str) -> NeuronPrunedResult:
+    """Gate pruning (by="gate") or Up pruning (by="up") of Sec. 3.2 / Eq. 5 for one token."""
+    assert by in ("gate", "up")
+    d_ff, d_model = Wg.d_out, Wg.d_in
+    x = _chk(np.ascontiguousarray(x), np.float32, d_model)
+    r = NeuronPrunedResult(np.empty(d_ff, np.float32), np.empty(d_ff, np.uint8), np.empty(k, np.int32),
+                           np.empty(d_ff, np.float32), np.empty(d_model, np.float64))
+    rc = _lib.orc_neuron_pruned_step(Wg.type, _p(Wg.w), _p(Wg.scales), _p(Wu.w), _p(Wu.scales), _p(Wd.w),
+                                     _p(Wd.scales), d_model, d_ff, _p(x), int(k), 0 if by == "gate" else 1,
+                                     _p(r.p32), _p(r.m), _p(r.idx), _p(r.h32), _p(r.y))
+    if rc:
+        raise ValueError("invalid k")
     return r
 
 

@@ -539,6 +539,62 @@ int orc_mlp_step(int type,
 }
 
 /* ------------------------------------------------------------------ *
+ * Gate pruning and Up pruning (Sec. 3.2, Eq. 5): one of the two d_ff-sized
+ * partial activations is computed densely and ranks the MLP's neurons; the
+ * rows of the other first-layer matrix and the columns of W^d that belong
+ * to neurons outside the top-k are zero, and the MLP is Eq. 1-2 with those
+ * pruned matrices.
+ *   by = 0 (Gate pruning):  p = silu(W^g x),  m = topK(|p|),
+ *                           h_j = p_j * (W^u x)_j        for j in m, else 0
+ *   by = 1 (Up pruning):    p = W^u x,        m = topK(|p|),
+ *                           h_j = p_j * silu((W^g x)_j)  for j in m, else 0
+ *   y = sum_{j in m} W^d[:, j] h_j
+ * As in the DIP step, an activation that is both ranked and multiplied is
+ * held in binary32: p32 = (float) p and h32 = (float) h; sums are fp64.
+ * Ties of |p32| go to the lower neuron index.
+ * ------------------------------------------------------------------ */
+int orc_neuron_pruned_step(int type,
+                           const void *Wg, const uint16_t *Sg,
+                           const void *Wu, const uint16_t *Su,
+                           const void *Wd, const uint16_t *Sd,
+                           int d_model, int d_ff, const float *x, int k, int by,
+                           float *p32, uint8_t *m, int32_t *idx, float *h32, double *y)
+{
+    if (by != 0 && by != 1)
+        return -1;
+    const void *Wp = by == 0 ? Wg : Wu;          /* the dense, ranking matrix */
+    const uint16_t *Sp = by == 0 ? Sg : Su;
+    const void *Wo = by == 0 ? Wu : Wg;          /* the other one, pruned by rows */
+    const uint16_t *So = by == 0 ? Su : Sg;
+    int j;
+#pragma omp parallel for schedule(static)
+    for (j = 0; j < d_ff; ++j) {
+        double acc = 0.0;
+        for (int i = 0; i < d_model; ++i)
+            acc += orc_weight(type, Wp, Sp, d_ff, d_model, j, i) * (double)x[i];
+        p32[j] = (float)(by == 0 ? orc_silu(acc) : acc);
+    }
+    uint32_t *key = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)d_ff);
+    for (j = 0; j < d_ff; ++j)
+        key[j] = orc_rank_key(p32[j], 1, 1.0f);
+    int rc = orc_topk_mask(key, d_ff, k, m, idx);
+    free(key);
+    if (rc)
+        return rc;
+#pragma omp parallel for schedule(static)
+    for (j = 0; j < d_ff; ++j) {
+        double acc = 0.0;
+        if (m[j])
+            for (int i = 0; i < d_model; ++i)
+                acc += orc_weight(type, Wo, So, d_ff, d_model, j, i) * (double)x[i];
+        /* a pruned row gives 0: Gate pruning 0 * p, Up pruning p * silu(0) */
+        h32[j] = m[j] ? (float)((double)p32[j] * (by == 0 ? acc : orc_silu(acc))) : 0.0f;
+    }
+    orc_masked_matvec(type, Wd, Sd, d_model, d_ff, h32, m, y);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ *
  * Layer chaining used by the multi-layer workloads (not in the paper, which
  * evaluates inside full models): x_next = (x + y) / rms(x + y), fp64, rounded
  * once to binary32.  An all-zero sum is passed through unchanged.

@@ -1,6 +1,6 @@
 """Planted mistakes: each mutant is a copy of the oracle's C source with one plausible error
 (a swapped operand, a wrong tie-break, a wrong eviction order, ...).  The pins of
-test_oracle_pins.py / test_oracle_policies.py must fail on every one of them -- that is what
+test_oracle_pins.py / test_oracle_policies.py / test_oracle_neuron_pruning.py must fail on every one of them -- that is what
 makes them pins.  The mistakes are planted in the CPU oracle only."""
 import os
 import subprocess
@@ -27,6 +27,10 @@ MUTANTS = {
                                "    int misses = k - hits;\n    int free_slots = capacity - *n_resident;\n    int n_evict = misses;\n    if (n_evict < 0)\n        n_evict = 0;\n    int evictable = *n_resident - hits;\n    if (n_evict > evictable)\n        n_evict = evictable;\n\n    /* least recently used first"),
     "lfu_evicts_most_used": ("            v[nv].stamp = count[i];", "            v[nv].stamp = -count[i];"),
     "belady_evicts_soonest": ("                if (next > far) {", "                if (far < 0 || next < far) {"),
+    "gate_pruning_ranks_raw_gate": ("p32[j] = (float)(by == 0 ? orc_silu(acc) : acc);", "p32[j] = (float)acc;"),
+    "gate_and_up_pruning_swapped": ("const void *Wp = by == 0 ? Wg : Wu;", "const void *Wp = by == 0 ? Wu : Wg;"),
+    "pruned_neurons_reach_down": ("    orc_masked_matvec(type, Wd, Sd, d_model, d_ff, h32, m, y);\n    return 0;\n}\n\n/* ------------------------------------------------------------------ *\n * Layer chaining",
+                                  "    memset(m, 1, (size_t)d_ff);\n    orc_masked_matvec(type, Wd, Sd, d_model, d_ff, h32, m, y);\n    return 0;\n}\n\n/* ------------------------------------------------------------------ *\n * Layer chaining"),
 }
 
 
@@ -43,7 +47,8 @@ def test_pins_kill_mutant(name, tmp_path):
     env = dict(os.environ, DIP_ORACLE_LIB=str(lib))
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                         os.path.join(ROOT, "tests", "test_oracle_pins.py"),
-                        os.path.join(ROOT, "tests", "test_oracle_policies.py")],
+                        os.path.join(ROOT, "tests", "test_oracle_policies.py"),
+                        os.path.join(ROOT, "tests", "test_oracle_neuron_pruning.py")],
                        cwd=ROOT, env=env, capture_output=True, text=True)
     assert r.returncode != 0, "the pins passed on a broken oracle (%s)" % name
     assert "failed" in r.stdout
