@@ -98,7 +98,8 @@ dip_status dip_device_status(dip_ctx *ctx, int *status_out, void *stream);
  * dip_trace_read returns the records of the launches that ran since.  These
  * calls synchronise the device; the stamps cost one atomic per CTA.
  *   kind: 1 select (DIP), 2 select (cache-aware), 3 cache update, 4 gate/up GEMV,
- *         5 down GEMV.
+ *         5 down GEMV, 6 slot assignment, 7 fetch, 8 hit/miss split (two-tier step),
+ *         9 neuron-major product (Gate / Up pruning).
  * ------------------------------------------------------------------------ */
 typedef struct {
     int32_t kind;
@@ -299,6 +300,38 @@ dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *lay
                           const float *x_in, int batch, int k_x, int k_h, float gamma,
                           const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
                           float *x_out, float *y_last, void *stream);
+
+/* ------------------------------------------------------------------------
+ * Gate pruning and Up pruning (Sec. 3.2, Eq. 5), the neuron-wise schedules the
+ * paper compares DIP with: one of the two first-layer products is computed
+ * densely and ranks the d_ff neurons, p = silu(W^g x) (Gate pruning) or
+ * p = W^u x (Up pruning); only the k neurons of largest |p| (ties to the lower
+ * index) are evaluated in the other first-layer matrix and in W^d:
+ *   h_j = p_j * (W^u x)_j   resp.   p_j * silu((W^g x)_j)   for kept j, else 0
+ *   y   = sum over kept j of W^d[:, j] h_j
+ * A neuron is a ROW of W^g / W^u and a COLUMN of W^d, so the layout differs
+ * from dip_mlp_weights: gate and up are the matrices' own row-major
+ * [d_ff][d_model] arrays (row j = neuron j), down is [d_ff][d_model] with row
+ * j = W^d[:, j] (the `down` array of dip_pack_weights).  F32 or BF16; INT4
+ * returns DIP_ERR_UNSUPPORTED.  One token per call.
+ *   x [d_model] in, y [d_model] out; optional outputs (device, may be NULL):
+ *   p_out [d_ff] the ranking activation, mask_out [ceil(d_ff/32)], idx_out [k]
+ *   ascending, h_out [d_ff].  p and h are binary32, sums binary32.
+ * ------------------------------------------------------------------------ */
+typedef struct {
+    int32_t wtype;
+    int32_t d_model;
+    int32_t d_ff;
+    int32_t reserved;
+    const void *gate;
+    const void *up;
+    const void *down;
+} dip_neuron_weights;
+enum { DIP_PRUNE_BY_GATE = 0, DIP_PRUNE_BY_UP = 1 };
+dip_status dip_mlp_step_neuron_pruned(dip_ctx *ctx, const dip_neuron_weights *w, int prune_by,
+                                      const float *x, int k, float *y,
+                                      float *p_out, uint32_t *mask_out, int32_t *idx_out, float *h_out,
+                                      void *stream);
 
 /* ------------------------------------------------------------------------
  * Two-tier execution (Sec. 5 and its diagram of a single linear layer; the

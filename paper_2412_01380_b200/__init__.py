@@ -89,6 +89,17 @@ _lib.dip_mlp_step_tiered.restype = _i32
 _lib.dip_mlp_step_tiered.argtypes = [_vp, C.POINTER(MlpWeightsStruct), C.POINTER(TierStruct), C.POINTER(TierStruct),
                                      _vp, _i32, _i32, _f32, C.POINTER(CacheStateStruct),
                                      C.POINTER(CacheStateStruct), _vp, C.POINTER(StepOutputsStruct), _vp]
+
+
+class NeuronWeightsStruct(C.Structure):
+    _fields_ = [("wtype", C.c_int32), ("d_model", C.c_int32), ("d_ff", C.c_int32), ("reserved", C.c_int32),
+                ("gate", _vp), ("up", _vp), ("down", _vp)]
+
+
+PRUNE_BY_GATE, PRUNE_BY_UP = 0, 1
+_lib.dip_mlp_step_neuron_pruned.restype = _i32
+_lib.dip_mlp_step_neuron_pruned.argtypes = [_vp, C.POINTER(NeuronWeightsStruct), _i32, _vp, _i32, _vp,
+                                            _vp, _vp, _vp, _vp, _vp]
 _lib.dip_sparse_gemv_down_noalloc.restype = _i32
 _lib.dip_sparse_gemv_down_noalloc.argtypes = [C.POINTER(MlpWeightsStruct), _vp, _vp, _i32, _vp, _vp]
 
@@ -96,7 +107,8 @@ EXPORTED = ["dip_create", "dip_destroy", "dip_status_string", "dip_last_error", 
             "dip_device_status", "dip_trace_begin", "dip_trace_reset", "dip_trace_read", "dip_trace_end",
             "dip_packed_bytes", "dip_pack_weights", "dip_mask_topk", "dip_ca_mask",
             "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_mlp_step",
-            "dip_residual_rmsnorm", "dip_stack_step", "dip_mlp_step_tiered", "dip_sparse_gemv_down_noalloc"]
+            "dip_residual_rmsnorm", "dip_stack_step", "dip_mlp_step_tiered", "dip_mlp_step_neuron_pruned",
+            "dip_sparse_gemv_down_noalloc"]
 
 
 class TraceRecord(C.Structure):
@@ -105,7 +117,7 @@ class TraceRecord(C.Structure):
 
 
 TRACE_KINDS = {1: "select", 2: "select_ca", 3: "cache_update", 4: "gemv_gate_up", 5: "gemv_down",
-               6: "tier_assign", 7: "tier_fetch", 8: "tier_split"}
+               6: "tier_assign", 7: "tier_fetch", 8: "tier_split", 9: "rowdot"}
 for _name in ("dip_trace_begin", "dip_trace_reset", "dip_trace_end"):
     getattr(_lib, _name).restype = _i32
     getattr(_lib, _name).argtypes = [_vp]
@@ -316,6 +328,29 @@ def dip_mlp_step_tiered(ctx: Context, w: MlpWeights, tier_gu: Tier, tier_d: Tier
                                        C.byref(tier_d.struct), _ptr(x), int(k_x), int(k_h), float(gamma),
                                        C.byref(tier_gu.cache.struct), C.byref(tier_d.cache.struct),
                                        _ptr(y), C.byref(outs), _stream()))
+
+
+class NeuronWeights:
+    """Weights of one block laid out by neuron for Gate / Up pruning: gate and up as their own
+    row-major [d_ff, d_model] matrices, down as [d_ff, d_model] with row j = W^d[:, j]."""
+
+    def __init__(self, wtype: int, gate: torch.Tensor, up: torch.Tensor, down_t: torch.Tensor):
+        d_ff, d_model = gate.shape
+        assert up.shape == gate.shape and tuple(down_t.shape) == (d_ff, d_model)
+        for t in (gate, up, down_t):
+            assert t.is_cuda and t.is_contiguous()
+        self.wtype, self.d_model, self.d_ff = int(wtype), int(d_model), int(d_ff)
+        self.gate, self.up, self.down = gate, up, down_t
+        self.struct = NeuronWeightsStruct(self.wtype, self.d_model, self.d_ff, 0, _ptr(gate), _ptr(up), _ptr(down_t))
+
+
+def dip_mlp_step_neuron_pruned(ctx: Context, w: NeuronWeights, prune_by: str, x: torch.Tensor, k: int,
+                               y: torch.Tensor, p=None, mask=None, idx=None, h=None) -> None:
+    """Gate pruning (prune_by="gate") or Up pruning ("up") of one token through one block."""
+    assert prune_by in ("gate", "up")
+    ctx.check(_lib.dip_mlp_step_neuron_pruned(ctx.handle, C.byref(w.struct),
+                                              PRUNE_BY_GATE if prune_by == "gate" else PRUNE_BY_UP, _ptr(x), int(k),
+                                              _ptr(y), _ptr(p), _ptr(mask), _ptr(idx), _ptr(h), _stream()))
 
 
 def dip_residual_rmsnorm(ctx: Context, x: torch.Tensor, y: torch.Tensor, x_next: torch.Tensor) -> None:

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdip.so")
-SOURCES = ["api.cu", "topk.cu", "gemv.cu", "gemv_noalloc.cu", "pack.cu", "tier.cu"]
+SOURCES = ["api.cu", "topk.cu", "gemv.cu", "gemv_noalloc.cu", "pack.cu", "tier.cu", "rowdot.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "dip.h")]
 
 NVCC_FLAGS = [

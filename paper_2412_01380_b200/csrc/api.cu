@@ -110,6 +110,7 @@ dip_status dip_create(dip_ctx **out, int device)
     if ((st = dev_alloc(ctx, &ctx->y2, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->xa, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->xb, vec)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->p, (size_t)DIP_MAX_D)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask, vec / 32)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->idx, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask_h, vec / 32)) != DIP_OK) return fail(st);
@@ -143,6 +144,7 @@ dip_status dip_destroy(dip_ctx *ctx)
     cudaFree(ctx->y2);
     cudaFree(ctx->xa);
     cudaFree(ctx->xb);
+    cudaFree(ctx->p);
     cudaFree(ctx->mask);
     cudaFree(ctx->idx);
     cudaFree(ctx->mask_h);
@@ -414,6 +416,47 @@ dip_status dip_mlp_step_tiered(dip_ctx *ctx, const dip_mlp_weights *w,
     if (out && out->idx_h && (st = dip_launch_mask_to_idx(ctx, mask_h, 1, 1, w->d_ff, out->idx_h, k_h, nullptr, s)) != DIP_OK)
         return st;
     return DIP_OK;
+}
+
+dip_status dip_mlp_step_neuron_pruned(dip_ctx *ctx, const dip_neuron_weights *w, int prune_by,
+                                      const float *x, int k, float *y,
+                                      float *p_out, uint32_t *mask_out, int32_t *idx_out, float *h_out,
+                                      void *stream)
+{
+    if (!ctx || !w || !x || !y || !dip_aligned16(x) || !dip_aligned16(y)) return DIP_ERR_INVALID_ARG;
+    if (w->wtype == DIP_W_INT4_G128) return DIP_ERR_UNSUPPORTED;
+    if (!dims_ok(w->wtype, w->d_model, w->d_ff)) return DIP_ERR_INVALID_ARG;
+    if (!w->gate || !w->up || !w->down || !dip_aligned16(w->gate) || !dip_aligned16(w->up) || !dip_aligned16(w->down))
+        return DIP_ERR_INVALID_ARG;
+    if (prune_by != DIP_PRUNE_BY_GATE && prune_by != DIP_PRUNE_BY_UP) return DIP_ERR_INVALID_ARG;
+    if (k < 1 || k > w->d_ff) return DIP_ERR_INVALID_ARG;
+    if ((p_out && !dip_aligned16(p_out)) || (h_out && !dip_aligned16(h_out))) return DIP_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    float *p = p_out ? p_out : ctx->p;
+    float *h = h_out ? h_out : ctx->h;
+    uint32_t *mask = mask_out ? mask_out : ctx->mask_h;
+    int32_t *idx = idx_out ? idx_out : ctx->idx_h;
+    const bool by_gate = prune_by == DIP_PRUNE_BY_GATE;
+    dip_status st;
+    // the dense, ranking activation: p = silu(W^g x) (Gate pruning) or W^u x (Up pruning)
+    st = dip_launch_rowdot(ctx, w->wtype, by_gate ? w->gate : w->up, w->d_model, w->d_ff, x, nullptr, w->d_ff,
+                           by_gate ? 1 : 0, nullptr, p, s);
+    if (st != DIP_OK) return st;
+    // m = topK(|p|) over the neurons (Eq. 5), as a bit set and as an ascending list
+    if ((st = dip_launch_select(ctx, p, nullptr, nullptr, 1, w->d_ff, k, 1.0f, nullptr, mask, s)) != DIP_OK) return st;
+    if ((st = dip_launch_mask_to_idx(ctx, mask, 1, 1, w->d_ff, idx, k, nullptr, s)) != DIP_OK) return st;
+    // the kept rows of the other matrix: h_j = p_j * (W^u x)_j, or p_j * silu((W^g x)_j); 0 elsewhere
+    DIP_CUDA_TRY(ctx, cudaMemsetAsync(h, 0, sizeof(float) * (size_t)w->d_ff, s));
+    st = dip_launch_rowdot(ctx, w->wtype, by_gate ? w->up : w->gate, w->d_model, w->d_ff, x, idx, k,
+                           by_gate ? 0 : 1, p, h, s);
+    if (st != DIP_OK) return st;
+    // y = sum over the kept neurons of W^d[:, j] h_j
+    dip_mlp_weights wd = {};
+    wd.wtype = w->wtype;
+    wd.d_model = w->d_model;
+    wd.d_ff = w->d_ff;
+    wd.down = w->down;
+    return dip_launch_gemv(ctx, &wd, 1, h, 1, mask, k, y, s);
 }
 
 dip_status dip_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y,

@@ -28,6 +28,7 @@ struct dip_ctx {
     float *y2;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner, odd layers)
     float *xa;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner ping)
     float *xb;           // [DIP_MAX_BATCH][DIP_MAX_D]   (stack runner pong)
+    float *p;            // [DIP_MAX_D]   ranking activation of Gate / Up pruning
     uint32_t *mask;      // [DIP_MAX_BATCH][DIP_MAX_D/32]  masks of x
     int32_t *idx;        // [DIP_MAX_BATCH][DIP_MAX_D]     kept indices of x
     uint32_t *mask_h;    // same for h
@@ -163,6 +164,12 @@ dip_status dip_launch_tier_assign(dip_ctx *ctx, const dip_tier *t, const uint32_
                                   cudaStream_t stream);
 // tier.cu: copy the rows of the fetch list from the slow tier into the arena.
 dip_status dip_launch_tier_fetch(dip_ctx *ctx, const dip_tier *t, cudaStream_t stream);
+
+// rowdot.cu: out_j = [silu](W[j, :] . x) [* mul_j] for the listed rows (rows == nullptr: rows
+// 0 .. n_rows-1) of a row-major [d_ff][d_model] matrix; F32 or BF16.
+dip_status dip_launch_rowdot(dip_ctx *ctx, int wtype, const void *W, int d_model, int d_ff, const float *x,
+                             const int32_t *rows, int n_rows, int silu, const float *mul, float *out,
+                             cudaStream_t stream);
 
 // pack.cu
 dip_status dip_launch_pack(dip_ctx *ctx, int wtype, int d_model, int d_ff,
