@@ -53,6 +53,8 @@ def parse_args():
                     help="run every workload of the five configurations (fewer steps) and write a markdown table")
     ap.add_argument("--two-tier", action="store_true",
                     help="time the two-tier step instead: cache arena in HBM, all weights in pinned host memory")
+    ap.add_argument("--schedule", default="dip", choices=["dip", "gate", "up"],
+                    help="dip: input pruning (the headline); gate / up: Gate / Up pruning of Eq. 5 (neuron-wise)")
     ap.add_argument("--token-correlation", type=float, default=0.0,
                     help="mix consecutive tokens (x_t = c x_{t-1} + sqrt(1-c^2) draw); 0 = independent tokens")
     ap.add_argument("--timeline", action="store_true",
@@ -530,6 +532,124 @@ def run_two_tier(dip, ctx, torch, w, L, rank, xs_host, keep_ratio, budget, steps
                     "d2h_bytes_per_step": 4 * d_model}}
 
 
+def main_neuron_pruned(args, dip, ctx, torch, w, keep_ratio, rank, world, local):
+    """Gate pruning / Up pruning (Eq. 5): per layer one dense neuron-major product ranks the
+    neurons, the other first-layer matrix and W^d are read for the kept neurons only."""
+    from dip_inputs import device as dd
+    if world > 1 or args.batch > 1 or w.wtype == di.W_INT4_G128:
+        raise SystemExit("--schedule gate|up is a single-GPU, single-token, F32/BF16 measurement")
+    by = args.schedule
+    L = args.layers if args.layers else w.n_layers
+    d_model, d_ff = w.d_model, w.d_ff
+    k = di.keep_count(keep_ratio, d_ff)
+    layers = []
+    for l in range(L):
+        g, _ = dd.matrix(w, l, "gate", d_ff, d_model, "cuda", rank)
+        u, _ = dd.matrix(w, l, "up", d_ff, d_model, "cuda", rank)
+        d_, _ = dd.matrix(w, l, "down", d_model, d_ff, "cuda", rank)
+        layers.append(dip.NeuronWeights(w.wtype, g, u, d_.t().contiguous()))
+        del d_
+    n_tok = min(w.n_tokens, args.steps + args.warmup)
+    xs_dev = torch.from_numpy(di.token_inputs(w, n_tokens=n_tok, batch=1)[:, 0].copy()).cuda()
+    xa, xb = torch.empty(d_model, device="cuda"), torch.empty(d_model, device="cuda")
+    y = torch.empty(d_model, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def token():
+        cur, nxt = xa, xb
+        for l in range(L):
+            dip.dip_mlp_step_neuron_pruned(ctx, layers[l], by, cur, k, y)
+            dip.dip_residual_rmsnorm(ctx, cur, y, nxt)
+            cur, nxt = nxt, cur
+        return cur
+
+    xa.copy_(xs_dev[0])
+    token()
+    torch.cuda.synchronize()
+    ctx.trace_begin()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        x_last = token()
+    # per-kernel durations from the device-side timeline of two replays
+    dense_us = kept_us = 0.0
+    for t in range(2):
+        xa.copy_(xs_dev[t % n_tok])
+        torch.cuda.synchronize()
+        ctx.trace_reset()
+        graph.replay()
+        recs = [r for r in ctx.trace_read() if r["kind"] == "rowdot"]
+        dense_us += sum(r["end"] - r["ready"] for r in recs[0::2])
+        kept_us += sum(r["end"] - r["ready"] for r in recs[1::2])
+    dense_us /= 2 * L
+    kept_us /= 2 * L
+    if args.timeline:
+        print_records(ctx.trace_read()[:10])
+        ctx.trace_end()
+        return
+    ctx.trace_end()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        x_last = token()
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
+                           else int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local]))
+    for t in range(args.warmup):
+        xa.copy_(xs_dev[t % n_tok], non_blocking=True)
+        graph.replay()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for t in range(args.steps):
+        xa.copy_(xs_dev[(args.warmup + t) % n_tok], non_blocking=True)
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    xs_pin = xs_dev.cpu().pin_memory()
+    out_host = torch.empty(d_model).pin_memory()
+    n_e2e = min(args.steps, 128)
+    e0.record(stream)
+    for t in range(n_e2e):
+        xa.copy_(xs_pin[t % n_tok], non_blocking=True)
+        graph.replay()
+        out_host.copy_(x_last, non_blocking=True)
+        stream.synchronize()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_e = e0.elapsed_time(e1)
+    bw = weight_bytes(w.wtype)
+    dense_bytes = d_ff * d_model * bw + 4 * (d_model + d_ff)
+    step_bytes = dense_bytes + 2 * k * d_model * bw + 4 * (3 * d_ff + 2 * d_model + k)
+    peak, peak_kind = measured_peak()
+    step_gbs = step_bytes * L * args.steps / (ms * 1e-3) / 1e9
+    achieved = dense_bytes / (dense_us * 1e-6) / 1e9
+    line = {
+        "metric": METRIC, "value": L * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": {di.W_F32: "f32", di.W_BF16: "bf16 weights, f32 accumulate"}[w.wtype], "data": "synthetic",
+        "config": {"workload": "%s, %s pruning (Eq. 5)" % (w.name, by), "n_layers": L, "d_model": d_model,
+                   "d_ff": d_ff, "keep_ratio": keep_ratio, "k": k,
+                   "step": "one decode token through %d layers = %d MLP-steps" % (L, L),
+                   "l2": "inputs larger than L2: %.1f GB of distinct layer weights cycled"
+                         % (3 * L * d_ff * d_model * bw / 1e9),
+                   "launch": "CUDA graph of dip_mlp_step_neuron_pruned + dip_residual_rmsnorm per layer",
+                   "parallelism": "replicas only"},
+        "mlp_step_us": ms * 1e3 / (L * args.steps), "step_gbs": step_gbs, "step_frac_of_measured_hbm": step_gbs / peak,
+        "clocks": clocks,
+        "e2e": {"value": L * n_e2e / (ms_e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * d_model,
+                "d2h_bytes_per_step": 4 * d_model},
+        # per layer: 2 row products, select, mask->list, memset, down GEMV, rmsnorm
+        "gpu_launches": 6 * L * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "rowdot_kernel (dense ranking product)", "achieved": achieved,
+                     "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "bytes_per_launch": dense_bytes, "us_per_launch": dense_us, "traffic": None},
+        "kernels_us": {"rowdot_dense": dense_us, "rowdot_kept": kept_us},
+    }
+    print(json.dumps(line))
+
+
 def main_two_tier(args, dip, ctx, torch, w, keep_ratio, budget, rank, world, local):
     if world > 1 or args.batch > 1 or budget is None:
         raise SystemExit("--two-tier is a single-GPU, single-token, cache-aware measurement")
@@ -740,6 +860,8 @@ def main():
     if args.report:
         write_report(dip, ctx, torch, args.report, min(args.steps, 128))
         return
+    if args.schedule != "dip":
+        return main_neuron_pruned(args, dip, ctx, torch, w, keep_ratio, rank, world, local)
     if args.two_tier:
         return main_two_tier(args, dip, ctx, torch, w, keep_ratio, budget, rank, world, local)
     L = args.layers if args.layers else w.n_layers
