@@ -101,6 +101,8 @@ dip_status dip_create(dip_ctx **out, int device)
         const int v = atoi(e);
         if (v == 512 || v == 1024 || v == 2048) ctx->gemv_seg = v;
     }
+    ctx->gemv_direct = 1;
+    if (const char *e = getenv("DIP_GEMV_DIRECT")) ctx->gemv_direct = atoi(e) != 0;   // tuning aid: 0 = copy-ring kernel
     ctx->n_tickets = N_TICKETS;
     const size_t vec = (size_t)DIP_MAX_BATCH * DIP_MAX_D;
     if ((st = dev_alloc(ctx, &ctx->partials, ctx->partials_floats)) != DIP_OK) return fail(st);

@@ -16,6 +16,7 @@ struct dip_ctx {
     int device;
     int sm_count;
     int gemv_seg;        // 0 = choose per launch; else force the GEMV segment width (tuning aid)
+    int gemv_direct;     // one token, F32/BF16: plain-load kernel instead of the copy ring
     // split-row partial sums of the two GEMVs (binary32)
     float *partials;
     size_t partials_floats;
