@@ -144,13 +144,12 @@ class ClockSampler:
 
 def ncu_traffic(w, keep_ratio, batch, algorithmic):
     """dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMV launch, from the ncu capture
-    summarised in profiles/kernels_phi3_medium_4layers_rho025.md (91.82 MB read + 2.51 MB written at
+    summarised in profiles/kernels_phi3_medium_4layers_rho025.md (91.79 MB read + 2.21 MB written at
     Phi-3-Medium shapes, keep ratio 0.25, one token).  Other keep ratios of the same workload scale
-    with the kept bytes (the traffic is the kept rows plus the split-row partial sums); anything
-    else has no capture."""
+    with the kept bytes (the traffic is the kept rows); anything else has no capture."""
     if w.name != "phi3_medium" or batch != 1:
         return None
-    return 94.33e6 if abs(keep_ratio - 0.25) < 1e-9 else algorithmic * (94.33e6 / 91.85e6)
+    return 94.00e6 if abs(keep_ratio - 0.25) < 1e-9 else algorithmic * (94.00e6 / 91.85e6)
 
 
 def max_over_ranks(ms, dist, torch, device):
@@ -926,7 +925,7 @@ def main():
         "clocks": head["clocks"],
         "e2e": {k: head["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
         "gpu_launches": launches_per_step * args.steps,
-        "roofline": {"bound": "hbm", "kernel": "gemv_kernel (gate/up bundle)", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "gemv_direct_kernel (gate/up bundle)" if args.batch == 1 and w.wtype != di.W_INT4_G128 else "gemv_kernel (gate/up bundle)", "achieved": achieved, "peak": peak,
                      "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS, "bytes_per_launch": gu_bytes,
                      "us_per_launch": gu_us, "traffic": ncu_traffic(w, keep_ratio, args.batch, gu_bytes)},

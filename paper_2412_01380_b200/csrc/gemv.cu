@@ -14,6 +14,9 @@
 //      part order by the last CTA to arrive at the slab (an arrival counter).
 // The order of every sum is fixed, so results are bit-reproducible; no float atomics.
 //
+// One token with F32 / BF16 weights takes gemv_direct_kernel further down instead: plain loads, a
+// 512-byte segment per CTA, and for gate/up no row parts at all.
+//
 // which = 0 (gate/up bundle): the epilogue applies silu(gate) * up (Eq. 2).  which = 1: down.
 // Every wait on an mbarrier is bounded; on expiry the kernel records a status word and leaves.
 #include <cuda_bf16.h>
