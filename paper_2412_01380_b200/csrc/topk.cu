@@ -336,6 +336,7 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
         // writes the certain bits and collects the bin's keys with their columns.
         s.hist[2 * tid] = 0;          // free again: refilled below with the candidates' next digit
         s.hist[2 * tid + 1] = 0;
+#pragma unroll 4
         for (int it = 0; it < span && base + it < d; it += 32) {
             const int e = base + it + lane;
             const uint32_t key = e < d ? keys[e] : 0u;
