@@ -107,7 +107,7 @@ __device__ __forceinline__ void find_bin(TkShared &s, int krem)
 __device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask, int top_bit, int k,
                                    TkShared &s, uint32_t &T, int &quota, int &n_eq)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
     uint32_t prefix = 0, prefmask = 0;
     int krem = k;
     int hi = top_bit;
