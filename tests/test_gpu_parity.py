@@ -186,6 +186,7 @@ GEMV_SHAPES = [
     (di.W_BF16, 64, 160, 0.5),         # rows of 640 and 128 bytes: segments with idle lanes
     (di.W_F32, 96, 32, 0.4),           # a row shorter than one 512-byte segment
     (di.W_BF16, 8192, 96, 0.6),        # more kept rows than one round of the in-kernel row list
+    (di.W_BF16, 128, 32768, 0.5),      # more gate/up segments than SMs; down rows of half a segment, 148 row parts
     (di.W_INT4_G128, 1024, 2816, 0.25), (di.W_INT4_G128, 384, 640, 0.5), (di.W_INT4_G128, 256, 512, 1.0),
     (di.W_INT4_G128, 4096, 14336, 0.25), (di.W_INT4_G128, 512, 1024, 0.01),
 ]
