@@ -896,10 +896,12 @@ __global__ void idx_to_mask_kernel(const int32_t *__restrict__ idx, int n, int d
     }
 }
 
-// Sum of the row parts in part order and the epilogue, one thread per four outputs: the same
-// arithmetic as the last-CTA path of gemv_kernel, as a kernel of its own (used when the batch is
-// large).  partials: [nparts][n_slabs][bt][slab]; gate/up rows are interleaved in chunks of c.
-template <int WHICH>
+// Sum of the row parts and the epilogue as a kernel of its own (large batches; the two launches
+// of the two-tier step).  CP_LANES (1 or 8) neighbouring lanes share four outputs: lane l adds the
+// parts l, l + CP_LANES, ... (its loads in flight together), then the lanes' sums meet in a fixed
+// shuffle tree, so the result is reproducible.  Eight lanes pay when there are many parts.  partials: [nparts][n_slabs][bt][slab]; gate/up rows are
+// interleaved in chunks of c.
+template <int WHICH, int CP_LANES>
 __global__ void __launch_bounds__(256)
 combine_parts_kernel(const float *__restrict__ partials, int nparts, int n_slabs, int bt, int slab_elems, int c,
                      int batch, int d_out, float *__restrict__ out)
@@ -910,24 +912,30 @@ combine_parts_kernel(const float *__restrict__ partials, int nparts, int n_slabs
     const int groups = out_per_slab / 4;
     const long long total = (long long)n_slabs * batch * groups;
     const size_t stride = (size_t)n_slabs * bt * slab_elems;
-    for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
-        const int o = (int)(t % groups) * 4;
-        const int b = (int)((t / groups) % batch);
-        const int slab = (int)(t / ((long long)groups * batch));
+    const int pl = threadIdx.x % CP_LANES;
+    const long long first = (blockIdx.x * (long long)blockDim.x + threadIdx.x) / CP_LANES;
+    const long long step = (long long)gridDim.x * blockDim.x / CP_LANES;
+    // whole warps iterate together (the bound is rounded up to the warp's four groups)
+    for (long long t0 = first - (threadIdx.x % 32) / CP_LANES; t0 < total; t0 += step) {
+        const long long t = t0 + (threadIdx.x % 32) / CP_LANES;
+        const bool live = t < total;
+        const int o = live ? (int)(t % groups) * 4 : 0;
+        const int b = live ? (int)((t / groups) % batch) : 0;
+        const int slab = live ? (int)(t / ((long long)groups * batch)) : 0;
         const int j = slab * out_per_slab + o;
-        if (j >= d_out) continue;
         const int e0 = WHICH == 0 ? (o / c) * 2 * c + (o % c) : o;
         const int e1 = e0 + c;
         const float *pp = partials + ((size_t)slab * bt + b) * slab_elems;
         float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
-        for (int q0 = 0; q0 < nparts; q0 += 8) {
+        for (int q0 = pl; q0 < nparts; q0 += 8 * CP_LANES) {
             float4 a0[8], a1[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 a0[q] = a1[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (q0 + q < nparts) {
-                    a0[q] = __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(q0 + q) * stride + e0));
-                    if (WHICH == 0) a1[q] = __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(q0 + q) * stride + e1));
+                const int part = q0 + q * CP_LANES;
+                if (live && part < nparts) {
+                    a0[q] = __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)part * stride + e0));
+                    if (WHICH == 0) a1[q] = __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)part * stride + e1));
                 }
             }
 #pragma unroll
@@ -936,9 +944,21 @@ combine_parts_kernel(const float *__restrict__ partials, int nparts, int n_slabs
                 s1.x += a1[q].x; s1.y += a1[q].y; s1.z += a1[q].z; s1.w += a1[q].w;
             }
         }
-        float4 r = s0;
-        if (WHICH == 0) r = make_float4(silu_f32(s0.x) * s1.x, silu_f32(s0.y) * s1.y, silu_f32(s0.z) * s1.z, silu_f32(s0.w) * s1.w);
-        *reinterpret_cast<float4 *>(out + (size_t)b * d_out + j) = r;
+#pragma unroll
+        for (int m = 1; m < CP_LANES; m <<= 1) {
+            s0.x += __shfl_xor_sync(0xffffffffu, s0.x, m); s0.y += __shfl_xor_sync(0xffffffffu, s0.y, m);
+            s0.z += __shfl_xor_sync(0xffffffffu, s0.z, m); s0.w += __shfl_xor_sync(0xffffffffu, s0.w, m);
+            if (WHICH == 0) {
+                s1.x += __shfl_xor_sync(0xffffffffu, s1.x, m); s1.y += __shfl_xor_sync(0xffffffffu, s1.y, m);
+                s1.z += __shfl_xor_sync(0xffffffffu, s1.z, m); s1.w += __shfl_xor_sync(0xffffffffu, s1.w, m);
+            }
+        }
+        if (live && pl == 0 && j < d_out) {
+            float4 r = s0;
+            if (WHICH == 0)
+                r = make_float4(silu_f32(s0.x) * s1.x, silu_f32(s0.y) * s1.y, silu_f32(s0.z) * s1.z, silu_f32(s0.w) * s1.w);
+            *reinterpret_cast<float4 *>(out + (size_t)b * d_out + j) = r;
+        }
     }
 }
 
@@ -964,10 +984,17 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, int 
     DIP_CUDA_TRY(ctx, dip_launch_pdl(gemv_kernel<WT, WHICH, BT, SEG>, grid, dim3(GV_THREADS), smem, stream, p));
     if ((BT >= 8 && nparts > 1 && !mode) || mode == 2) {
         const long long groups = (long long)n_slabs * p.batch * ((WHICH == 0 ? SLAB / 2 : SLAB) / 4);
-        const int blocks = (int)((groups + 255) / 256);
-        DIP_CUDA_TRY(ctx, dip_launch_pdl(combine_parts_kernel<WHICH>, dim3(blocks), dim3(256), 0, stream,
-                                         (const float *)p.partials, total_parts, n_slabs, BT, SLAB, WTraits<WT>::C, p.batch,
-                                         p.d_out, p.out));
+        if (total_parts >= 16) {
+            const int blocks = (int)((groups * 8 + 255) / 256);
+            DIP_CUDA_TRY(ctx, dip_launch_pdl(combine_parts_kernel<WHICH, 8>, dim3(blocks), dim3(256), 0, stream,
+                                             (const float *)p.partials, total_parts, n_slabs, BT, SLAB, WTraits<WT>::C,
+                                             p.batch, p.d_out, p.out));
+        } else {
+            const int blocks = (int)((groups + 255) / 256);
+            DIP_CUDA_TRY(ctx, dip_launch_pdl(combine_parts_kernel<WHICH, 1>, dim3(blocks), dim3(256), 0, stream,
+                                             (const float *)p.partials, total_parts, n_slabs, BT, SLAB, WTraits<WT>::C,
+                                             p.batch, p.d_out, p.out));
+        }
     }
     return DIP_OK;
 }
