@@ -154,7 +154,7 @@ __device__ void block_radix_select(const uint32_t *keys, int d, uint32_t keymask
 
 
 constexpr int TK_VEC_ITERS = DIP_MAX_D / 4 / TK_THREADS;   // float4 loads per thread at the largest d
-constexpr int TK_VEC_BATCH = 4;                            // of which this many are in flight together
+constexpr int TK_VEC_BATCH = 5;                            // of which this many are in flight together
 
 // scale = 1 / rms(xa + xb) over d elements, the same bits on every thread of the CTA.  The sums
 // r = xa + xb are optionally parked in stash[] (as bit patterns).  Summation order: each thread
