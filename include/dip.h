@@ -98,8 +98,8 @@ dip_status dip_device_status(dip_ctx *ctx, int *status_out, void *stream);
  * dip_trace_read returns the records of the launches that ran since.  These
  * calls synchronise the device; the stamps cost one atomic per CTA.
  *   kind: 1 select (DIP), 2 select (cache-aware), 3 cache update, 4 gate/up GEMV,
- *         5 down GEMV, 6 slot assignment, 7 fetch, 8 hit/miss split (two-tier step),
- *         9 neuron-major product (Gate / Up pruning).
+ *         5 down GEMV, 6 slot assignment, 7 fetch, 8 hit/miss split, 10 install (two-tier
+ *         step), 9 neuron-major product (Gate / Up pruning).
  * ------------------------------------------------------------------------ */
 typedef struct {
     int32_t kind;
@@ -349,14 +349,16 @@ dip_status dip_mlp_step_neuron_pruned(dip_ctx *ctx, const dip_neuron_weights *w,
  *   backing  slow tier: the d packed rows of the matrix ([d][row_bytes], the
  *            layout of dip_pack_weights: gate_up or down), device-accessible
  *   arena    fast tier, device: (capacity + staging) rows of row_bytes; rows
- *            0 .. capacity-1 are cache slots, the rest hold, for one step,
- *            columns that are used without being kept (more misses than room)
+ *            0 .. capacity-1 are cache slots; the rest are staging rows: a
+ *            step's misses land there (the j-th miss in ascending column order
+ *            in row capacity + j) and are multiplied from there; those that the
+ *            cache keeps are then moved into their slots
  *   slot     device int32[d]: cache slot of column i, -1 = not resident.  Must
  *            agree with the cache state: slot[i] >= 0 exactly where
  *            stamp[i] >= 0; start both cold (all -1)
  *   loc      device int32[d]: scratch; arena row of each column of the current mask
- *   fetch    device int32[4 + 2 * staging]: scratch; [0] = rows fetched this
- *            step, then their columns, then their arena rows
+ *   fetch    device int32[4 + 2 * staging]: scratch; [0] = misses of the step,
+ *            [1] = rows moved into slots, then the misses' columns, then the moves
  *   split    device uint32[2][ceil(d/32)]: scratch; the mask's hits and its misses
  *   counters device uint64[2], accumulated: rows fetched, bytes fetched
  * Which slot a new column gets is the library's choice (the lowest free slots,
@@ -382,15 +384,18 @@ typedef struct {
 /* ------------------------------------------------------------------------
  * dip_mlp_step_tiered — dip_mlp_step for one token with both masked inputs
  * cache-aware and their weights two-tiered.  Per input: mask (Algorithm 1's
- * ranking), cache update, slot assignment, then the mask's hits are multiplied
- * out of the arena while a second stream copies its misses from the slow tier
- * into their slots; the misses' product follows and the two partial results
- * are added in row order groups (hits first).  w gives the format and shapes
- * (and the INT4 scales); w->gate_up and w->down are not read and may be NULL.
- * Results equal dip_mlp_step's on the same cache states up to the order of
- * the binary32 sums.  k_x <= tier_gu->staging and k_h <= tier_d->staging.
- * A slot table that disagrees with the cache state (fewer free slots than
- * columns to insert) sets the sticky device status to 2 and fetches nothing.
+ * ranking); the mask's hits are multiplied out of the arena at once while one
+ * stream of the context copies its misses from the slow tier into the staging
+ * rows and another keeps the books (cache update, slot assignment, the move of
+ * the staged rows that the cache keeps into their slots); the misses' product
+ * follows the copy and the two partial results are added (hits first).  The
+ * book-keeping is joined into `stream` before the call's work ends.  w gives
+ * the format and shapes (and the INT4 scales); w->gate_up and w->down are not
+ * read and may be NULL.  Results equal dip_mlp_step's on the same cache states
+ * up to the order of the binary32 sums.  k_x <= tier_gu->staging and
+ * k_h <= tier_d->staging.  A slot table that disagrees with the cache state
+ * (fewer free slots than columns to insert, a resident column the table does
+ * not know) sets the sticky device status to 2 and installs nothing.
  * ------------------------------------------------------------------------ */
 dip_status dip_mlp_step_tiered(dip_ctx *ctx, const dip_mlp_weights *w,
                                const dip_tier *tier_gu, const dip_tier *tier_d,

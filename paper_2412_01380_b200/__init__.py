@@ -117,7 +117,7 @@ class TraceRecord(C.Structure):
 
 
 TRACE_KINDS = {1: "select", 2: "select_ca", 3: "cache_update", 4: "gemv_gate_up", 5: "gemv_down",
-               6: "tier_assign", 7: "tier_fetch", 8: "tier_split", 9: "rowdot"}
+               6: "tier_assign", 7: "tier_fetch", 8: "tier_split", 9: "rowdot", 10: "tier_install"}
 for _name in ("dip_trace_begin", "dip_trace_reset", "dip_trace_end"):
     getattr(_lib, _name).restype = _i32
     getattr(_lib, _name).argtypes = [_vp]

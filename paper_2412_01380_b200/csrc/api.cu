@@ -125,6 +125,13 @@ dip_status dip_create(dip_ctx **out, int device)
     if (cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if ((st = dev_alloc(ctx, &ctx->trace, (size_t)DIP_TRACE_SLOTS * DIP_TRACE_WORDS)) != DIP_OK) return fail(st);
     for (int i = 0; i < 2; ++i) {
+        if (cudaStreamCreateWithFlags(&ctx->tier_fetch[i], cudaStreamNonBlocking) != cudaSuccess) return fail(DIP_ERR_CUDA);
+        if (cudaStreamCreateWithFlags(&ctx->tier_book[i], cudaStreamNonBlocking) != cudaSuccess) return fail(DIP_ERR_CUDA);
+        if (cudaEventCreateWithFlags(&ctx->ev_tier_fork[i], cudaEventDisableTiming) != cudaSuccess) return fail(DIP_ERR_CUDA);
+        if (cudaEventCreateWithFlags(&ctx->ev_tier_fetched[i], cudaEventDisableTiming) != cudaSuccess) return fail(DIP_ERR_CUDA);
+        if (cudaEventCreateWithFlags(&ctx->ev_tier_booked[i], cudaEventDisableTiming) != cudaSuccess) return fail(DIP_ERR_CUDA);
+    }
+    for (int i = 0; i < 2; ++i) {
         if (cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking) != cudaSuccess) return fail(DIP_ERR_CUDA);
         if (cudaEventCreateWithFlags(&ctx->ev_fork[i], cudaEventDisableTiming) != cudaSuccess) return fail(DIP_ERR_CUDA);
         if (cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming) != cudaSuccess) return fail(DIP_ERR_CUDA);
@@ -161,6 +168,11 @@ dip_status dip_destroy(dip_ctx *ctx)
         if (ctx->side[i]) cudaStreamDestroy(ctx->side[i]);
         if (ctx->ev_fork[i]) cudaEventDestroy(ctx->ev_fork[i]);
         if (ctx->ev_join[i]) cudaEventDestroy(ctx->ev_join[i]);
+        if (ctx->tier_fetch[i]) cudaStreamDestroy(ctx->tier_fetch[i]);
+        if (ctx->tier_book[i]) cudaStreamDestroy(ctx->tier_book[i]);
+        if (ctx->ev_tier_fork[i]) cudaEventDestroy(ctx->ev_tier_fork[i]);
+        if (ctx->ev_tier_fetched[i]) cudaEventDestroy(ctx->ev_tier_fetched[i]);
+        if (ctx->ev_tier_booked[i]) cudaEventDestroy(ctx->ev_tier_booked[i]);
     }
     delete ctx;
     return DIP_OK;
@@ -353,30 +365,36 @@ dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
                      ctx->mask, ctx->mask_h, false, stream);
 }
 
-// One masked input of the two-tier step: the hits' product on the main stream beside the cache
-// update, the slot assignment and the misses' fetch on a side stream; then the misses' product
-// and the sum of both.
+// One masked input of the two-tier step.  On the step's path: the hit / miss split, the list of
+// the misses, the hits' product; beside it one stream fetches the misses into the staging rows
+// (the misses' product waits for that) and another keeps the books: cache update, slot
+// assignment, and the move of the staged rows of the inserted columns into their slots.  The
+// book-keeping is joined at the end of the call.
 static dip_status tiered_half(dip_ctx *ctx, const dip_mlp_weights *w, int which, const dip_tier *t,
                               const dip_cache_state *c, const float *v, const uint32_t *mask_bits, int k,
                               float *out, cudaStream_t s)
 {
-    // the hits need neither the update nor the fetch: their product starts right away, while the
-    // side stream updates the cache, assigns slots and brings the misses in
+    const int words = (t->d + 31) / 32;
     dip_status st = dip_launch_tier_split(ctx, t, mask_bits, s);
     if (st != DIP_OK) return st;
-    cudaStream_t side = ctx->side[which];
-    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork[which], s));
-    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(side, ctx->ev_fork[which], 0));
+    // the misses as an ascending list: fetch[0] = how many, fetch[4 ..] = their columns
+    if ((st = dip_launch_mask_to_idx(ctx, t->split + words, 1, 1, t->d, t->fetch + 4, 0, t->fetch, s)) != DIP_OK) return st;
+    cudaStream_t sf = ctx->tier_fetch[which], sb = ctx->tier_book[which];
+    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_tier_fork[which], s));
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(sf, ctx->ev_tier_fork[which], 0));
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(sb, ctx->ev_tier_fork[which], 0));
+    if ((st = dip_launch_tier_fetch(ctx, t, sf)) != DIP_OK) return st;
+    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_tier_fetched[which], sf));
     st = dip_launch_cache_update(ctx, mask_bits, c->d, c->stamp, c->policy == DIP_CACHE_LFU ? c->count : nullptr,
-                                 c->meta, c->capacity, side);
+                                 c->meta, c->capacity, sb);
     if (st != DIP_OK) return st;
-    if ((st = dip_launch_tier_assign(ctx, t, mask_bits, c->stamp, side)) != DIP_OK) return st;
-    if ((st = dip_launch_tier_fetch(ctx, t, side)) != DIP_OK) return st;
-    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join[which], side));
-    const int words = (t->d + 31) / 32;
+    if ((st = dip_launch_tier_assign(ctx, t, mask_bits, c->stamp, sb)) != DIP_OK) return st;
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(sb, ctx->ev_tier_fetched[which], 0));
+    if ((st = dip_launch_tier_install(ctx, t, sb)) != DIP_OK) return st;
+    DIP_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_tier_booked[which], sb));
     dip_gemv_rows rows = {t->arena, t->loc, 1};
     if ((st = dip_launch_gemv(ctx, w, which, v, 1, t->split, k, out, s, &rows)) != DIP_OK) return st;
-    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->ev_join[which], 0));
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->ev_tier_fetched[which], 0));
     rows.mode = 2;
     return dip_launch_gemv(ctx, w, which, v, 1, t->split + words, k, out, s, &rows);
 }
@@ -417,6 +435,9 @@ dip_status dip_mlp_step_tiered(dip_ctx *ctx, const dip_mlp_weights *w,
         return st;
     if (out && out->idx_h && (st = dip_launch_mask_to_idx(ctx, mask_h, 1, 1, w->d_ff, out->idx_h, k_h, nullptr, s)) != DIP_OK)
         return st;
+    // the book-keeping of both inputs has to be through before the call's work ends
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->ev_tier_booked[0], 0));
+    DIP_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->ev_tier_booked[1], 0));
     return DIP_OK;
 }
 

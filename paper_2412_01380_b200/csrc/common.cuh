@@ -43,6 +43,9 @@ struct dip_ctx {
     cudaStream_t side[2];
     cudaEvent_t ev_fork[2], ev_join[2];
     bool side_busy[2];
+    // two-tier step, per masked input: a stream that fetches the misses and one that keeps the books
+    cudaStream_t tier_fetch[2], tier_book[2];
+    cudaEvent_t ev_tier_fork[2], ev_tier_fetched[2], ev_tier_booked[2];
     // device-side timeline (diagnostics): one slot of DIP_TRACE_WORDS words per launch
     unsigned long long *trace;
     int trace_on;
@@ -159,12 +162,15 @@ dip_status dip_launch_idx_to_mask(dip_ctx *ctx, const int32_t *idx, int n, int d
 // tier.cu: before the cache update of a mask: its hits (resident columns, with their arena rows)
 // and its misses.
 dip_status dip_launch_tier_split(dip_ctx *ctx, const dip_tier *t, const uint32_t *mask_bits, cudaStream_t stream);
-// tier.cu: after the cache update: slots for the inserted columns, the step's arena row of every
-// miss, and the fetch list.
+// tier.cu: after the cache update: evicted columns free their slots, inserted columns get slots,
+// and the install list says which staging rows move where.
 dip_status dip_launch_tier_assign(dip_ctx *ctx, const dip_tier *t, const uint32_t *mask_bits, const int32_t *stamp,
                                   cudaStream_t stream);
-// tier.cu: copy the rows of the fetch list from the slow tier into the arena.
+// tier.cu: copy the rows of the miss list (fetch[0] columns at fetch + 4) from the slow tier into
+// the staging rows of the arena, in list order, and point loc at them.
 dip_status dip_launch_tier_fetch(dip_ctx *ctx, const dip_tier *t, cudaStream_t stream);
+// tier.cu: move the staged rows of the inserted columns into their cache slots (install list).
+dip_status dip_launch_tier_install(dip_ctx *ctx, const dip_tier *t, cudaStream_t stream);
 
 // rowdot.cu: out_j = [silu](W[j, :] . x) [* mul_j] for the listed rows (rows == nullptr: rows
 // 0 .. n_rows-1) of a row-major [d_ff][d_model] matrix; F32 or BF16.

@@ -14,8 +14,9 @@ struct TierParams {
     const uint32_t *mask;      // [words] the step's mask
     const int32_t *stamp;      // [d] cache state AFTER the step's update (>= 0: resident)
     int32_t *slot;             // [d] in: slots before the update; out: after it
-    int32_t *loc;              // [d] out: arena row of each kept column that was not resident
-    int32_t *fetch;            // out: [0] = n, [4 ..) columns, [4 + staging ..) arena rows
+    int32_t *loc;              // [d] arena row of each kept column (not touched here)
+    int32_t *fetch;            // [0] = misses fetched, [1] = out: rows to install, [4 ..) the misses' columns,
+                               // [4 + staging ..) out: install list
     uint32_t *split;           // [0][words] hits, [1][words] misses (written by tier_split_kernel)
     unsigned long long *counters;
     int *status;
@@ -80,10 +81,11 @@ tier_split_kernel(const uint32_t *__restrict__ mask, const int32_t *__restrict__
     DIP_TRACE_MAX(tr, 2);
 }
 
-// One CTA.  Compares the slot table (residency before the update) with the stamps (residency
-// after it): evicted columns give up their slots, inserted columns take the lowest free slots in
-// ascending column order, kept columns that did not become resident get a staging row for this
-// step.  Writes the list of rows to fetch.
+// One CTA, after the cache update, beside the products (nothing on the step's path waits for it).
+// Compares the slot table (residency before the update) with the stamps (residency after it):
+// evicted columns give up their slots, inserted columns take the lowest free slots in ascending
+// column order.  Every miss of the step has been fetched into the staging row of its rank among
+// the misses; the install list says which staging rows move into which slots.
 __global__ void __launch_bounds__(TA_THREADS, 1)
 tier_assign_kernel(const TierParams t)
 {
@@ -142,47 +144,42 @@ tier_assign_kernel(const TierParams t)
         if (t.capacity - w * 32 < 32) fr &= (1u << (t.capacity - w * 32)) - 1u;
     }
     const uint32_t ins = ~B & A;           // became resident in this step
-    const uint32_t byp = m & ~A;           // kept, not resident afterwards: one-step staging row
-    if ((ins & ~m) | (byp & B)) s_bad = 1; // only columns of the mask are inserted; its hits stay
-    int v[3] = {__popc(ins), __popc(byp), __popc(fr)}, pre[3];
+    const uint32_t miss = m & ~B;          // kept and not resident before: fetched into staging
+    if ((ins & ~miss) | (m & B & ~A)) s_bad = 1;   // only misses are inserted; the mask's hits stay
+    int v[3] = {__popc(ins), __popc(miss), __popc(fr)}, pre[3];
     block_scan3(v, pre, s_ws, s_tot);
-    const int n_ins = s_tot[0], n_byp = s_tot[1], n_free = s_tot[2];
-    const bool bad = s_bad || n_ins > n_free || n_ins + n_byp > t.staging;
-    int32_t *cols = t.fetch + 4, *dsts = t.fetch + 4 + t.staging;
+    const int n_ins = s_tot[0], n_miss = s_tot[1], n_free = s_tot[2];
+    const bool bad = s_bad || n_ins > n_free || n_miss > t.staging;
+    int32_t *inst = t.fetch + 4 + t.staging;                   // install list: (rank among the misses) << 16 | slot
     if (bad) {
-        // the table and the cache state disagree: fetch nothing, multiply no fetched row, say so
-        if (w < words) t.split[words + w] = 0u;
+        // the table and the cache state disagree: install nothing, say so
         if (tid == 0) {
-            t.fetch[0] = 0;
+            t.fetch[1] = 0;
             atomicExch(t.status, 2);
         }
         DIP_TRACE_MAX(t.tr, 2);
         return;
     }
     {
-        int r = pre[0];
-        for (uint32_t u = ins; u; u &= u - 1) cols[r++] = w * 32 + __ffs(u) - 1;
-        int q = pre[1];
-        for (uint32_t u = byp; u; u &= u - 1, ++q) {
-            const int i = w * 32 + __ffs(u) - 1;
-            cols[n_ins + q] = i;
-            dsts[n_ins + q] = t.capacity + q;
-            t.loc[i] = t.capacity + q;
-        }
+        // the j-th free slot (ascending) goes to the j-th inserted column (ascending)
         int f = pre[2];
-        for (uint32_t u = fr; u && f < n_ins; u &= u - 1) dsts[f++] = w * 32 + __ffs(u) - 1;
+        for (uint32_t u = fr; u && f < n_ins; u &= u - 1) inst[f++] = w * 32 + __ffs(u) - 1;
     }
     __syncthreads();
-    for (int r = tid; r < n_ins; r += TA_THREADS) {
-        const int c = cols[r], s = dsts[r];
-        t.slot[c] = s;
-        t.loc[c] = s;
+    {
+        int r = pre[0];
+        for (uint32_t u = ins; u; u &= u - 1, ++r) {
+            const int bit = __ffs(u) - 1, col = w * 32 + bit;
+            const int rank = pre[1] + __popc(miss & ((1u << bit) - 1u));   // the column's staging row
+            const int sl = inst[r];
+            t.slot[col] = sl;
+            inst[r] = (rank << 16) | sl;
+        }
     }
     if (tid == 0) {
-        const int n = n_ins + n_byp;
-        t.fetch[0] = n;
-        t.counters[0] += (unsigned long long)n;
-        t.counters[1] += (unsigned long long)n * t.row_bytes;
+        t.fetch[1] = n_ins;
+        t.counters[0] += (unsigned long long)n_miss;
+        t.counters[1] += (unsigned long long)n_miss * t.row_bytes;
     }
     DIP_TRACE_MAX(t.tr, 2);
 }
@@ -191,27 +188,36 @@ constexpr int TF_THREADS = 256;
 constexpr int TF_UNROLL = 4;
 constexpr int TF_CHUNK = TF_THREADS * 16 * TF_UNROLL;     // bytes one CTA moves per turn
 
-// Copies the listed rows from the slow tier into their arena rows: a grid-stride loop over
+// Copies `n` rows src_row(e) -> dst_row(e) of row_bytes each: a grid-stride loop over
 // (row, 16 KB chunk) units, 16 bytes per thread and four loads in flight per thread.  Plain loads:
 // the source may be host memory mapped into the device's address space.
+//   INSTALL = false (fetch): row e of the miss list: slow tier row cols[e] -> staging row
+//             capacity + e, and loc[cols[e]] = that row for the product over the misses;
+//   INSTALL = true: entry e of the install list: staging row -> cache slot, inside the arena.
+template <bool INSTALL>
 __global__ void __launch_bounds__(TF_THREADS)
-tier_fetch_kernel(const char *__restrict__ backing, char *__restrict__ arena, const int32_t *__restrict__ fetch,
-                  int staging, unsigned long long row_bytes, unsigned long long *tr)
+tier_copy_kernel(const char *__restrict__ backing, char *arena, const int32_t *__restrict__ fetch,
+                 int32_t *__restrict__ loc, int capacity, int staging, unsigned long long row_bytes,
+                 unsigned long long *tr)
 {
     DIP_TRACE_MIN(tr, 0);
     dip_grid_dependency_wait();
     DIP_TRACE_MIN(tr, 1);
     dip_launch_dependents();
-    const int n = fetch[0];
-    const int32_t *cols = fetch + 4, *dsts = fetch + 4 + staging;
+    const int n = INSTALL ? fetch[1] : min(fetch[0], staging);
+    const int32_t *list = fetch + 4 + (INSTALL ? staging : 0);
     const int cpr = (int)((row_bytes + TF_CHUNK - 1) / TF_CHUNK);
     const long long total = (long long)n * cpr;
     for (long long u = blockIdx.x; u < total; u += gridDim.x) {
         const int e = (int)(u / cpr), c = (int)(u % cpr);
+        const int v = list[e];
         const size_t off = (size_t)c * TF_CHUNK;
         const int vecs = (int)(min((unsigned long long)TF_CHUNK, row_bytes - off) / 16);
-        const uint4 *src = reinterpret_cast<const uint4 *>(backing + (size_t)cols[e] * row_bytes + off);
-        uint4 *dst = reinterpret_cast<uint4 *>(arena + (size_t)dsts[e] * row_bytes + off);
+        const char *src_row = INSTALL ? arena + (size_t)(capacity + (v >> 16)) * row_bytes : backing + (size_t)v * row_bytes;
+        const int dst_row = INSTALL ? (v & 0xffff) : capacity + e;
+        const uint4 *src = reinterpret_cast<const uint4 *>(src_row + off);
+        uint4 *dst = reinterpret_cast<uint4 *>(arena + (size_t)dst_row * row_bytes + off);
+        if (!INSTALL && c == 0 && threadIdx.x == 0) loc[v] = dst_row;
         uint4 q[TF_UNROLL];
 #pragma unroll
         for (int j = 0; j < TF_UNROLL; ++j) {
@@ -261,8 +267,17 @@ dip_status dip_launch_tier_split(dip_ctx *ctx, const dip_tier *t, const uint32_t
 dip_status dip_launch_tier_fetch(dip_ctx *ctx, const dip_tier *t, cudaStream_t stream)
 {
     unsigned long long *tr = dip_trace_slot(ctx, 7);
-    DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_fetch_kernel, dim3(2 * ctx->sm_count), dim3(TF_THREADS), 0, stream,
-                                     (const char *)t->backing, (char *)t->arena, (const int32_t *)t->fetch, t->staging,
-                                     (unsigned long long)t->row_bytes, tr));
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_copy_kernel<false>, dim3(2 * ctx->sm_count), dim3(TF_THREADS), 0, stream,
+                                     (const char *)t->backing, (char *)t->arena, (const int32_t *)t->fetch, t->loc,
+                                     (int)t->capacity, (int)t->staging, (unsigned long long)t->row_bytes, tr));
+    return DIP_OK;
+}
+
+dip_status dip_launch_tier_install(dip_ctx *ctx, const dip_tier *t, cudaStream_t stream)
+{
+    unsigned long long *tr = dip_trace_slot(ctx, 10);
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_copy_kernel<true>, dim3(2 * ctx->sm_count), dim3(TF_THREADS), 0, stream,
+                                     (const char *)t->backing, (char *)t->arena, (const int32_t *)t->fetch, t->loc,
+                                     (int)t->capacity, (int)t->staging, (unsigned long long)t->row_bytes, tr));
     return DIP_OK;
 }
