@@ -184,12 +184,14 @@ tier_assign_kernel(const TierParams t)
     DIP_TRACE_MAX(t.tr, 2);
 }
 
-constexpr int TF_THREADS = 256;
+constexpr int TF_THREADS = 512;
 constexpr int TF_UNROLL = 4;
 constexpr int TF_CHUNK = TF_THREADS * 16 * TF_UNROLL;     // bytes one CTA moves per turn
 
 // Copies `n` rows src_row(e) -> dst_row(e) of row_bytes each: a grid-stride loop over
-// (row, 16 KB chunk) units, 16 bytes per thread and four loads in flight per thread.  Plain loads:
+// (row, 32 KB chunk) units, 16 bytes per thread and four loads in flight per thread.  The grid
+// leaves a few SMs without a CTA of this long-running kernel: the single-CTA book-keeping kernels
+// beside it need a whole SM's registers.  Plain loads:
 // the source may be host memory mapped into the device's address space.
 //   INSTALL = false (fetch): row e of the miss list: slow tier row cols[e] -> staging row
 //             capacity + e, and loc[cols[e]] = that row for the product over the misses;
@@ -267,7 +269,8 @@ dip_status dip_launch_tier_split(dip_ctx *ctx, const dip_tier *t, const uint32_t
 dip_status dip_launch_tier_fetch(dip_ctx *ctx, const dip_tier *t, cudaStream_t stream)
 {
     unsigned long long *tr = dip_trace_slot(ctx, 7);
-    DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_copy_kernel<false>, dim3(2 * ctx->sm_count), dim3(TF_THREADS), 0, stream,
+    const dim3 grid(ctx->sm_count > 16 ? ctx->sm_count - 8 : ctx->sm_count);
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(tier_copy_kernel<false>, grid, dim3(TF_THREADS), 0, stream,
                                      (const char *)t->backing, (char *)t->arena, (const int32_t *)t->fetch, t->loc,
                                      (int)t->capacity, (int)t->staging, (unsigned long long)t->row_bytes, tr));
     return DIP_OK;
