@@ -26,11 +26,10 @@ struct TkShared {
     int wc[TK_WARPS];
     float wf[TK_WARPS];
     float scale;
-    int n_cand, n_cand2;
+    int n_cand2;
     uint32_t last_key[32];
     int last_idx[32];
 };
-constexpr int TK_CAND_CAP = 2048;   // candidates of the threshold bin kept for the refinement passes
 
 __device__ __forceinline__ unsigned lanemask_lt()
 {
@@ -226,7 +225,7 @@ __device__ float block_residual_scale(const float *__restrict__ xa, const float 
 //   NORM == true: the row is first formed as x = (xa + xb) / rms(xa + xb) (the layer chaining
 //                of a stack) and written to x_out; the summation order is that of
 //                residual_rmsnorm_kernel, so both give the same bits.
-// keys[] is dynamic shared memory: d words.
+// keys[] is dynamic shared memory: d words rounded up to a multiple of four.
 // ---------------------------------------------------------------------------------------
 template <bool CA, bool NORM>
 __global__ void __launch_bounds__(TK_THREADS, 1)
@@ -237,9 +236,8 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
     DIP_TRACE_MIN(tr, 0);
     extern __shared__ uint32_t keys[];
     __shared__ TkShared s;
-    __shared__ uint32_t cand_key[TK_CAND_CAP];
-    __shared__ int cand_idx[TK_CAND_CAP];
-    __shared__ unsigned int s_maskw[DIP_MAX_D / 32];
+    __shared__ unsigned int s_maskw[DIP_MAX_D / 32];   // the mask being built
+    __shared__ unsigned int s_candw[DIP_MAX_D / 32];   // columns whose key falls in the threshold's bin
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x;
     const int n_words = (d + 31) >> 5;
@@ -253,7 +251,6 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
     s.hist[2 * tid] = 0;
     s.hist[2 * tid + 1] = 0;
     if (tid == 0) {
-        s.n_cand = 0;
         s.n_cand2 = 0;
     }
     dip_grid_dependency_wait();        // the inputs come from the previous kernel in the stream
@@ -323,50 +320,77 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
     __syncthreads();
     find_bin(s, k);
     const uint32_t b1 = (uint32_t)s.bcast[0];
-    const int krem1 = s.bcast[1], cnt1 = s.bcast[2];
+    const int krem1 = s.bcast[1];
 
     // warp w owns columns [w*span, (w+1)*span), span a multiple of 32: one ballot = one mask word
     const int span = ((d + TK_THREADS - 1) / TK_THREADS) * 32;
     const int base = warp * span;
 
-    bool fast = cnt1 <= TK_CAND_CAP;
-    if (fast) {
-        // Every key in a bin above b1 is kept, every key below is dropped; the krem1 largest of the
-        // cnt1 keys in bin b1 (lower index first among equals) complete the mask.  One sweep
-        // writes the certain bits and collects the bin's keys with their columns.
-        s.hist[2 * tid] = 0;          // free again: refilled below with the candidates' next digit
-        s.hist[2 * tid + 1] = 0;
-#pragma unroll 4
-        for (int it = 0; it < span && base + it < d; it += 32) {
-            const int e = base + it + lane;
-            const uint32_t key = e < d ? keys[e] : 0u;
-            const uint32_t dg = key >> 20;
-            const unsigned bk = __ballot_sync(0xffffffffu, e < d && dg > b1);
-            if (lane == 0) s_maskw[(base + it) >> 5] = bk;
-            if (e < d && dg == b1) {
-                const int pos = atomicAdd(&s.n_cand, 1);
-                cand_key[pos] = key & 0xfffffu;
-                cand_idx[pos] = e;
+    // Every key in a bin above b1 is kept, every key below is dropped; the krem1 largest of the
+    // keys in bin b1 (lower index first among equals) complete the mask.  One sweep, four keys
+    // per lane, builds two bit sets in the mask's layout: the certain columns and the columns of
+    // bin b1.  A lane's four flags are a nibble; eight neighbouring lanes OR theirs into a word.
+    s.hist[2 * tid] = 0;          // free again: refilled below with the candidates' next digit
+    s.hist[2 * tid + 1] = 0;
+    {
+        const int n4 = (d + 3) >> 2;
+        const int sh = (lane & 7) * 4;
+        for (int q0 = warp * 32; q0 < n4; q0 += TK_THREADS) {
+            const int q = q0 + lane;
+            uint4 kk = make_uint4(0u, 0u, 0u, 0u);
+            unsigned live = 0u;                                // which of the four columns exist
+            if (q < n4) {
+                kk = *reinterpret_cast<const uint4 *>(keys + 4 * q);
+                live = 4 * q + 4 <= d ? 0xfu : (1u << (d - 4 * q)) - 1u;
+            }
+            const uint32_t d0 = kk.x >> 20, d1 = kk.y >> 20, d2 = kk.z >> 20, d3 = kk.w >> 20;
+            unsigned gt = (d0 > b1 ? 1u : 0u) | (d1 > b1 ? 2u : 0u) | (d2 > b1 ? 4u : 0u) | (d3 > b1 ? 8u : 0u);
+            unsigned eq = (d0 == b1 ? 1u : 0u) | (d1 == b1 ? 2u : 0u) | (d2 == b1 ? 4u : 0u) | (d3 == b1 ? 8u : 0u);
+            gt = (gt & live) << sh;
+            eq = (eq & live) << sh;
+#pragma unroll
+            for (int o = 1; o < 8; o <<= 1) {
+                gt |= __shfl_xor_sync(0xffffffffu, gt, o);
+                eq |= __shfl_xor_sync(0xffffffffu, eq, o);
+            }
+            if ((lane & 7) == 0 && q < n4) {
+                s_maskw[q >> 3] = gt;
+                s_candw[q >> 3] = eq;
             }
         }
-        __syncthreads();
-        // second digit (bits 19..9) of the candidates
-        for (int c = tid; c < cnt1; c += TK_THREADS) atomicAdd(&s.hist[cand_key[c] >> 9], 1u);
+    }
+    __syncthreads();
+    {
+        // second digit (bits 19..9) of the candidates; a thread walks the candidate bits of a word
+        for (int w = tid; w < n_words; w += TK_THREADS) {
+            unsigned u = s_candw[w];
+            while (u) {
+                const int col = w * 32 + __ffs(u) - 1;
+                u &= u - 1;
+                atomicAdd(&s.hist[(keys[col] & 0xfffffu) >> 9], 1u);
+            }
+        }
         __syncthreads();
         find_bin(s, krem1);
         const uint32_t b2 = (uint32_t)s.bcast[0];
         const int krem2 = s.bcast[1], cnt2 = s.bcast[2];
-        fast = cnt2 <= 32;
-        if (fast) {
-            for (int c = tid; c < cnt1; c += TK_THREADS) {
-                const uint32_t dg = cand_key[c] >> 9;
-                if (dg > b2) {
-                    atomicOr(&s_maskw[cand_idx[c] >> 5], 1u << (cand_idx[c] & 31));
-                } else if (dg == b2) {
-                    const int pos = atomicAdd(&s.n_cand2, 1);
-                    s.last_key[pos] = cand_key[c] & 0x1ffu;
-                    s.last_idx[pos] = cand_idx[c];
+        if (cnt2 <= 32) {
+            for (int w = tid; w < n_words; w += TK_THREADS) {
+                unsigned u = s_candw[w], keep = 0u;
+                while (u) {
+                    const int bit = __ffs(u) - 1;
+                    u &= u - 1;
+                    const uint32_t low = keys[w * 32 + bit] & 0xfffffu;
+                    const uint32_t dg = low >> 9;
+                    if (dg > b2) {
+                        keep |= 1u << bit;
+                    } else if (dg == b2) {
+                        const int pos = atomicAdd(&s.n_cand2, 1);
+                        s.last_key[pos] = low & 0x1ffu;
+                        s.last_idx[pos] = w * 32 + bit;
+                    }
                 }
+                if (keep) s_maskw[w] |= keep;                  // the word is this thread's
             }
             __syncthreads();
             if (warp == 0) {
@@ -620,7 +644,7 @@ residual_rmsnorm_kernel(const float *x, const float *y, int d, float *x_next)
 dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d, int k,
                              float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream)
 {
-    const size_t smem = (size_t)d * sizeof(uint32_t);
+    const size_t smem = (size_t)((d + 3) & ~3) * sizeof(uint32_t);
     const dim3 grid(batch), block(TK_THREADS);
     unsigned long long *tr = dip_trace_slot(ctx, d <= 0 ? 0 : (stamp ? 2 : 1));
     cudaError_t e;
