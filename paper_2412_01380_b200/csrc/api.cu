@@ -121,6 +121,7 @@ dip_status dip_create(dip_ctx **out, int device)
     if ((st = dev_alloc(ctx, &ctx->counts, (size_t)8)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask_ring, (size_t)2 * DIP_RING_LAYERS * (DIP_MAX_D / 32))) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask_tmp, (size_t)(DIP_MAX_D / 32))) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->coarse, (size_t)DIP_MAX_D)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->status, (size_t)1)) != DIP_OK) return fail(st);
     if (cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if ((st = dev_alloc(ctx, &ctx->trace, (size_t)DIP_TRACE_SLOTS * DIP_TRACE_WORDS)) != DIP_OK) return fail(st);
@@ -162,6 +163,7 @@ dip_status dip_destroy(dip_ctx *ctx)
     cudaFree(ctx->counts);
     cudaFree(ctx->mask_ring);
     cudaFree(ctx->mask_tmp);
+    cudaFree(ctx->coarse);
     cudaFree(ctx->status);
     cudaFree(ctx->trace);
     for (int i = 0; i < 2; ++i) {
@@ -333,11 +335,13 @@ static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
     // c' = cache_update(c, m_x)       (Algorithm 1; beside the products, which do not need it)
     if (cache_gu && (st = fork_cache_update(ctx, 0, mask_x, cache_gu, s)) != DIP_OK) return st;
     // h = (W~u x) * silu(W~g x)       (Eq. 2 inside Eq. 3)
-    st = dip_launch_gemv(ctx, w, 0, x, batch, mask_x, nmax_x, h, s);
+    // (a single-token product also leaves the top bits of the rank keys of h for the next launch)
+    dip_gemv_keys hk = {ctx->coarse, cache_d ? cache_d->stamp : nullptr, gamma, 0};
+    st = dip_launch_gemv(ctx, w, 0, x, batch, mask_x, nmax_x, h, s, nullptr, batch == 1 ? &hk : nullptr);
     if (st != DIP_OK) return st;
     // m_h = topK(score(h))            (Eq. 8: the GLU of the already sparsified gate/up)
     st = dip_launch_select(ctx, h, nullptr, nullptr, batch, w->d_ff, k_h, gamma,
-                           cache_d ? cache_d->stamp : nullptr, mask_h, s);
+                           cache_d ? cache_d->stamp : nullptr, mask_h, s, hk.written ? ctx->coarse : nullptr);
     if (st != DIP_OK) return st;
     if (cache_d && (st = fork_cache_update(ctx, 1, mask_h, cache_d, s)) != DIP_OK) return st;
     // y = W~d h                       (Eq. 1 inside Eq. 3)

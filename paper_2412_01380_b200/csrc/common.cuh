@@ -38,6 +38,7 @@ struct dip_ctx {
     int32_t *counts;     // [8] device scalars (union sizes)
     uint32_t *mask_ring; // [2][DIP_RING_LAYERS][DIP_MAX_D/32] per-layer mask slots of the stack runner
     uint32_t *mask_tmp;  // [DIP_MAX_D/32] list-based GEMV entry points
+    uint16_t *coarse;    // [DIP_MAX_D] top 16 bits of the rank keys of h, left by the gate/up GEMV
     int *status;         // sticky device status word (0 = fine)
     // the cache updates run beside the GEMVs: one side stream per cache kind
     cudaStream_t side[2];
@@ -119,8 +120,12 @@ static inline bool dip_aligned16(const void *p) { return (((uintptr_t)p) & 15u) 
 
 // topk.cu: mask of each row: k largest rank keys (|x|, or |x| * (resident ? 1 : gamma) when stamp
 // is given).  xb != nullptr: the row is first formed as (xa + xb) / rms(xa + xb), written to x_out.
+// coarse != nullptr (one row, no xb, d % 32 == 0): the producer of xa has left the top 16 bits of
+// every column's rank key there (dip_gemv_keys), and the launch reads those instead of all of
+// xa and stamp.
 dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d, int k,
-                             float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream);
+                             float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream,
+                             const uint16_t *coarse = nullptr);
 
 // topk.cu: LRU cache update from (mask, state).
 // count != nullptr: LFU (use counters), else LRU.
@@ -152,9 +157,20 @@ struct dip_gemv_rows {
     const int32_t *loc;
     int mode;            // 0 = a launch of its own
 };
+// keys != nullptr (which = 0): the caller ranks h next and wants the top 16 bits of every rank key
+// |h_j| * (stamp[j] >= 0 ? 1 : gamma) (stamp == nullptr: |h_j|) in keys->coarse[j].  Only the
+// single-token F32 / BF16 launch writes them; keys->written says whether it did.  The stamps are
+// read while the product runs, so nothing may change them between this launch and the ranking.
+struct dip_gemv_keys {
+    uint16_t *coarse;        // [d_ff]
+    const int32_t *stamp;    // cache state of the down input, or nullptr
+    float gamma;
+    int written;             // out
+};
 dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                            const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
-                           float *out, cudaStream_t stream, const dip_gemv_rows *rows = nullptr);
+                           float *out, cudaStream_t stream, const dip_gemv_rows *rows = nullptr,
+                           dip_gemv_keys *keys = nullptr);
 
 // gemv.cu: bit set from an ascending index list.
 dip_status dip_launch_idx_to_mask(dip_ctx *ctx, const int32_t *idx, int n, int d, uint32_t *mask, cudaStream_t stream);

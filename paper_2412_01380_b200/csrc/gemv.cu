@@ -55,6 +55,12 @@ struct GemvParams {
     const int32_t *loc;        // two-tier: packed row of column i is W + loc[i] * row_bytes (nullptr: row i)
     int defer;                 // 1: leave the row parts in `partials` for combine_parts_kernel
     int part_base;             // first part index of this launch inside `partials`
+    // gate/up, gemv_direct_kernel only: top 16 bits of the rank key of every h_j for the select
+    // that follows (nullptr: not wanted); the key is |h_j| * (key_stamp[j] >= 0 ? 1 : key_gamma),
+    // or |h_j| without stamps
+    uint16_t *key_coarse;
+    const int32_t *key_stamp;
+    float key_gamma;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -713,6 +719,11 @@ gemv_direct_kernel(const GemvParams p)
     DIP_TRACE_MIN(p.tr, 1);
     dip_launch_dependents();
 
+    // the stamp that the epilogue's rank key needs travels while the rows stream
+    int key_stamp = 0;
+    if (WHICH == 0 && p.key_coarse && p.key_stamp && tid < OUT_PER_SLAB && slab * OUT_PER_SLAB + tid < p.d_out)
+        key_stamp = __ldcg(p.key_stamp + slab * OUT_PER_SLAB + tid);
+
     // ---- 1. the mask words and their popcount prefix (as in gemv_kernel) ----
     if (tid < GV_SCAN_THREADS) {
         uint32_t u[4] = {0u, 0u, 0u, 0u};
@@ -853,6 +864,12 @@ gemv_direct_kernel(const GemvParams p)
                 r = s.sum[o];
             }
             p.out[j] = r;
+            if (WHICH == 0 && p.key_coarse) {
+                // what the select would form from h_j and the stamp, cut to its top 16 bits
+                float a = fabsf(r);
+                if (p.key_stamp) a = __fmul_rn(a, key_stamp >= 0 ? 1.0f : p.key_gamma);
+                p.key_coarse[j] = (uint16_t)((__float_as_uint(a) & 0x7fffffffu) >> 16);
+            }
         }
     }
     DIP_TRACE_MAX(p.tr, 2);
@@ -1045,9 +1062,10 @@ dip_status launch_bt(dip_ctx *ctx, GemvParams &p, int n_kept_max, int mode, cuda
 
 dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                            const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
-                           float *out, cudaStream_t stream, const dip_gemv_rows *rows)
+                           float *out, cudaStream_t stream, const dip_gemv_rows *rows, dip_gemv_keys *keys)
 {
     const int mode = rows ? rows->mode : 0;
+    if (keys) keys->written = 0;
     if (mode && batch != 1) return DIP_ERR_UNSUPPORTED;
     const bool int4 = w->wtype == DIP_W_INT4_G128;
     if (int4 && batch > 1) return DIP_ERR_UNSUPPORTED;      // the 4-bit path is single-token
@@ -1064,6 +1082,9 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
     p.partials = ctx->partials;
     p.tickets = ctx->tickets;
     p.status = ctx->status;
+    p.key_coarse = nullptr;
+    p.key_stamp = nullptr;
+    p.key_gamma = 1.0f;
     // all tokens of the batch in one launch (up to 16 sets of accumulators in registers): the
     // union of their rows is read once
     for (int b0 = 0; b0 < batch; b0 += 16) {
@@ -1074,6 +1095,12 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
         p.tr = dip_trace_slot(ctx, which == 0 ? 4 : 5);
         dip_status st;
         if (ctx->gemv_direct && !int4 && p.batch == 1 && !rows) {
+            if (keys && which == 0 && batch == 1 && keys->coarse) {
+                p.key_coarse = keys->coarse;
+                p.key_stamp = keys->stamp;
+                p.key_gamma = keys->gamma;
+                keys->written = 1;
+            }
             if (w->wtype == DIP_W_F32)
                 st = which == 0 ? launch_direct<DIP_W_F32, 0>(ctx, p, n_kept_max, stream)
                                 : launch_direct<DIP_W_F32, 1>(ctx, p, n_kept_max, stream);

@@ -217,6 +217,108 @@ __device__ float block_residual_scale(const float *__restrict__ xa, const float 
     return *scale_slot;
 }
 
+// Second half of the fast path.  s_maskw holds the columns whose key lies in a bin above the
+// threshold's, s_candw those in the threshold's bin (both in the mask's layout, complete and
+// visible), keys[] the rank key of every candidate column at least, s.hist is zero.  The krem1
+// largest candidates (lower column first among equals) complete the mask.  Returns false when
+// more than 32 candidates share the threshold's top 22 bits; nothing has been written then.
+__device__ bool refine_candidates(const uint32_t *keys, TkShared &s, unsigned int *s_maskw, const unsigned int *s_candw,
+                                  int n_words, int krem1, uint32_t *__restrict__ mask_bits)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // second digit (bits 19..9) of the candidates; a thread walks the candidate bits of a word
+    for (int w = tid; w < n_words; w += TK_THREADS) {
+        unsigned u = s_candw[w];
+        while (u) {
+            const int col = w * 32 + __ffs(u) - 1;
+            u &= u - 1;
+            atomicAdd(&s.hist[(keys[col] & 0xfffffu) >> 9], 1u);
+        }
+    }
+    __syncthreads();
+    find_bin(s, krem1);
+    const uint32_t b2 = (uint32_t)s.bcast[0];
+    const int krem2 = s.bcast[1], cnt2 = s.bcast[2];
+    if (cnt2 > 32) return false;
+    for (int w = tid; w < n_words; w += TK_THREADS) {
+        unsigned u = s_candw[w], keep = 0u;
+        while (u) {
+            const int bit = __ffs(u) - 1;
+            u &= u - 1;
+            const uint32_t low = keys[w * 32 + bit] & 0xfffffu;
+            const uint32_t dg = low >> 9;
+            if (dg > b2) {
+                keep |= 1u << bit;
+            } else if (dg == b2) {
+                const int pos = atomicAdd(&s.n_cand2, 1);
+                s.last_key[pos] = low & 0x1ffu;
+                s.last_idx[pos] = w * 32 + bit;
+            }
+        }
+        if (keep) s_maskw[w] |= keep;                  // the word is this thread's
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // at most 32 keys share the threshold's top 22 bits: rank them by (key descending,
+        // column ascending) and keep the first krem2
+        const uint32_t kv = lane < cnt2 ? s.last_key[lane] : 0u;
+        const int iv = lane < cnt2 ? s.last_idx[lane] : 0x7fffffff;
+        int rank = 0;
+        for (int j = 0; j < cnt2; ++j) {
+            const uint32_t kj = __shfl_sync(0xffffffffu, kv, j);
+            const int ij = __shfl_sync(0xffffffffu, iv, j);
+            rank += (kj > kv) || (kj == kv && ij < iv);
+        }
+        if (lane < cnt2 && rank < krem2) atomicOr(&s_maskw[iv >> 5], 1u << (iv & 31));
+    }
+    __syncthreads();
+    for (int w = tid; w < n_words; w += TK_THREADS) mask_bits[w] = s_maskw[w];
+    return true;
+}
+
+// General path (very many keys tied around the threshold): full radix select on all d keys in
+// keys[], then an ordered sweep that ranks the ties by column.
+__device__ void general_select(const uint32_t *keys, int d, int k, TkShared &s, uint32_t *__restrict__ mask_bits)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // warp w owns columns [w*span, (w+1)*span), span a multiple of 32: one ballot = one mask word
+    const int span = ((d + TK_THREADS - 1) / TK_THREADS) * 32;
+    const int base = warp * span;
+    uint32_t T;
+    int quota, n_eq;
+    block_radix_select(keys, d, 0x7fffffffu, 31, k, s, T, quota, n_eq);
+    if (quota == n_eq) {
+        // every column tied with the threshold is kept: the mask is key >= T
+        for (int it = 0; it < span && base + it < d; it += 32) {
+            const int e = base + it + lane;
+            const unsigned bk = __ballot_sync(0xffffffffu, e < d && keys[e] >= T);
+            if (lane == 0) mask_bits[(base + it) >> 5] = bk;
+        }
+        return;
+    }
+    // only the first `quota` tied columns (by index) are kept: rank the ties in order
+    const unsigned lt = lanemask_lt();
+    int eq = 0;
+    for (int it = 0; it < span; it += 32) {
+        const int e = base + it + lane;
+        eq += __popc(__ballot_sync(0xffffffffu, e < d && keys[e] == T));
+    }
+    if (lane == 0) s.wb[warp] = eq;
+    __syncthreads();
+    int tot;
+    int eq_before = warp_array_prefix(s.wb, warp, lane, tot);
+    for (int it = 0; it < span && base + it < d; it += 32) {
+        const int e = base + it + lane;
+        const uint32_t key = e < d ? keys[e] : 0u;
+        const bool q = e < d && key == T;
+        const unsigned bq = __ballot_sync(0xffffffffu, q);
+        const bool keep = (e < d && key > T) || (q && (eq_before + __popc(bq & lt)) < quota);
+        const unsigned bk = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) mask_bits[(base + it) >> 5] = bk;
+        eq_before += __popc(bq);
+    }
+}
+
 // ---------------------------------------------------------------------------------------
 // select_kernel: the mask of one row.
 //   CA == false: key = bits(|x|)                              (DIP, Eq. 7-8)
@@ -322,10 +424,6 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
     const uint32_t b1 = (uint32_t)s.bcast[0];
     const int krem1 = s.bcast[1];
 
-    // warp w owns columns [w*span, (w+1)*span), span a multiple of 32: one ballot = one mask word
-    const int span = ((d + TK_THREADS - 1) / TK_THREADS) * 32;
-    const int base = warp * span;
-
     // Every key in a bin above b1 is kept, every key below is dropped; the krem1 largest of the
     // keys in bin b1 (lower index first among equals) complete the mask.  One sweep, four keys
     // per lane, builds two bit sets in the mask's layout: the certain columns and the columns of
@@ -360,95 +458,129 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
         }
     }
     __syncthreads();
-    {
-        // second digit (bits 19..9) of the candidates; a thread walks the candidate bits of a word
-        for (int w = tid; w < n_words; w += TK_THREADS) {
-            unsigned u = s_candw[w];
-            while (u) {
-                const int col = w * 32 + __ffs(u) - 1;
-                u &= u - 1;
-                atomicAdd(&s.hist[(keys[col] & 0xfffffu) >> 9], 1u);
-            }
-        }
-        __syncthreads();
-        find_bin(s, krem1);
-        const uint32_t b2 = (uint32_t)s.bcast[0];
-        const int krem2 = s.bcast[1], cnt2 = s.bcast[2];
-        if (cnt2 <= 32) {
-            for (int w = tid; w < n_words; w += TK_THREADS) {
-                unsigned u = s_candw[w], keep = 0u;
-                while (u) {
-                    const int bit = __ffs(u) - 1;
-                    u &= u - 1;
-                    const uint32_t low = keys[w * 32 + bit] & 0xfffffu;
-                    const uint32_t dg = low >> 9;
-                    if (dg > b2) {
-                        keep |= 1u << bit;
-                    } else if (dg == b2) {
-                        const int pos = atomicAdd(&s.n_cand2, 1);
-                        s.last_key[pos] = low & 0x1ffu;
-                        s.last_idx[pos] = w * 32 + bit;
-                    }
-                }
-                if (keep) s_maskw[w] |= keep;                  // the word is this thread's
-            }
-            __syncthreads();
-            if (warp == 0) {
-                // at most 32 keys share the threshold's top 22 bits: rank them by (key descending,
-                // column ascending) and keep the first krem2
-                const uint32_t kv = lane < cnt2 ? s.last_key[lane] : 0u;
-                const int iv = lane < cnt2 ? s.last_idx[lane] : 0x7fffffff;
-                int rank = 0;
-                for (int j = 0; j < cnt2; ++j) {
-                    const uint32_t kj = __shfl_sync(0xffffffffu, kv, j);
-                    const int ij = __shfl_sync(0xffffffffu, iv, j);
-                    rank += (kj > kv) || (kj == kv && ij < iv);
-                }
-                if (lane < cnt2 && rank < krem2) atomicOr(&s_maskw[iv >> 5], 1u << (iv & 31));
-            }
-            __syncthreads();
-            for (int w = tid; w < n_words; w += TK_THREADS) mask_bits[w] = s_maskw[w];
-            DIP_TRACE_MAX(tr, 2);
-            return;
-        }
-    }
-
-    // General path (very many keys tied around the threshold): full radix select on all keys,
-    // then an ordered sweep that ranks the ties by column.
-    uint32_t T;
-    int quota, n_eq;
-    block_radix_select(keys, d, 0x7fffffffu, 31, k, s, T, quota, n_eq);
-    if (quota == n_eq) {
-        // every column tied with the threshold is kept: the mask is key >= T
-        for (int it = 0; it < span && base + it < d; it += 32) {
-            const int e = base + it + lane;
-            const unsigned bk = __ballot_sync(0xffffffffu, e < d && keys[e] >= T);
-            if (lane == 0) mask_bits[(base + it) >> 5] = bk;
-        }
+    if (refine_candidates(keys, s, s_maskw, s_candw, n_words, krem1, mask_bits)) {
         DIP_TRACE_MAX(tr, 2);
         return;
     }
-    // only the first `quota` tied columns (by index) are kept: rank the ties in order
-    const unsigned lt = lanemask_lt();
-    int eq = 0;
-    for (int it = 0; it < span; it += 32) {
-        const int e = base + it + lane;
-        eq += __popc(__ballot_sync(0xffffffffu, e < d && keys[e] == T));
+    general_select(keys, d, k, s, mask_bits);
+    DIP_TRACE_MAX(tr, 2);
+}
+
+// ---------------------------------------------------------------------------------------
+// select_coarse_kernel: the same mask as select_kernel<CA, false> for one row whose producer has
+// already left the top 16 bits of every rank key in coarse[] (the gate/up GEMV does, in its
+// epilogue).  One SM reads global memory at a fraction of the device's rate, so the bytes this CTA
+// has to pull in are its floor: two bytes per column here instead of the eight of value + stamp.
+// The first radix digit (top 11 bits) and the classification sweep work on the coarse keys, eight
+// per lane, held in registers; the full key is formed only for the few hundred columns of the
+// threshold's bin.  Needs d % 8 == 0 and d <= 8 * TK_COARSE_ITERS * TK_THREADS.
+// ---------------------------------------------------------------------------------------
+constexpr int TK_COARSE_ITERS = DIP_MAX_D / 8 / TK_THREADS;    // 16-byte loads per thread at the largest d
+
+template <bool CA>
+__device__ __forceinline__ uint32_t rank_key(float v, int stamp, float gamma)
+{
+    float a = fabsf(v);
+    if (CA) a = __fmul_rn(a, stamp >= 0 ? 1.0f : gamma);
+    return __float_as_uint(a) & 0x7fffffffu;
+}
+
+template <bool CA>
+__global__ void __launch_bounds__(TK_THREADS, 1)
+select_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ coarse, int d, int k, float gamma,
+                     const int32_t *__restrict__ stamp, uint32_t *__restrict__ mask_bits, unsigned long long *tr)
+{
+    DIP_TRACE_MIN(tr, 0);
+    extern __shared__ uint32_t keys[];
+    __shared__ TkShared s;
+    __shared__ unsigned int s_maskw[DIP_MAX_D / 32];
+    __shared__ unsigned int s_candw[DIP_MAX_D / 32];
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int n_words = d >> 5;
+    const int n8 = d >> 3;
+
+    s.hist[2 * tid] = 0;
+    s.hist[2 * tid + 1] = 0;
+    if (tid == 0) s.n_cand2 = 0;
+    dip_grid_dependency_wait();
+    DIP_TRACE_MIN(tr, 1);
+    dip_launch_dependents();
+
+    // coarse keys to registers (all loads in flight together)
+    uint4 ck[TK_COARSE_ITERS];
+#pragma unroll
+    for (int j = 0; j < TK_COARSE_ITERS; ++j) {
+        const int q = tid + j * TK_THREADS;
+        ck[j] = make_uint4(0u, 0u, 0u, 0u);
+        if (q < n8) ck[j] = __ldcg(reinterpret_cast<const uint4 *>(coarse) + q);
     }
-    if (lane == 0) s.wb[warp] = eq;
+    __syncthreads();                                               // histogram zeroed
+#pragma unroll
+    for (int j = 0; j < TK_COARSE_ITERS; ++j) {
+        if (tid + j * TK_THREADS < n8) {
+            const uint32_t wv[4] = {ck[j].x, ck[j].y, ck[j].z, ck[j].w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                atomicAdd(&s.hist[(wv[t] & 0xffffu) >> 4], 1u);
+                atomicAdd(&s.hist[wv[t] >> 20], 1u);
+            }
+        }
+    }
     __syncthreads();
-    int tot;
-    int eq_before = warp_array_prefix(s.wb, warp, lane, tot);
-    for (int it = 0; it < span && base + it < d; it += 32) {
-        const int e = base + it + lane;
-        const uint32_t key = e < d ? keys[e] : 0u;
-        const bool q = e < d && key == T;
-        const unsigned bq = __ballot_sync(0xffffffffu, q);
-        const bool keep = (e < d && key > T) || (q && (eq_before + __popc(bq & lt)) < quota);
-        const unsigned bk = __ballot_sync(0xffffffffu, keep);
-        if (lane == 0) mask_bits[(base + it) >> 5] = bk;
-        eq_before += __popc(bq);
+    find_bin(s, k);
+    const uint32_t b1 = (uint32_t)s.bcast[0];
+    const int krem1 = s.bcast[1];
+
+    // classification: a lane's eight flags are a byte, four neighbouring lanes make a mask word
+    s.hist[2 * tid] = 0;
+    s.hist[2 * tid + 1] = 0;
+    {
+        const int sh = (lane & 3) * 8;
+#pragma unroll
+        for (int j = 0; j < TK_COARSE_ITERS; ++j) {
+            const int q = tid + j * TK_THREADS;
+            if ((tid & ~31) + j * TK_THREADS < n8) {                  // the whole warp or none of it
+                const uint32_t wv[4] = {ck[j].x, ck[j].y, ck[j].z, ck[j].w};
+                unsigned gt = 0u, eq = 0u;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const uint32_t lo = (wv[t] & 0xffffu) >> 4, hi = wv[t] >> 20;
+                    gt |= (lo > b1 ? 1u : 0u) << (2 * t) | (hi > b1 ? 2u : 0u) << (2 * t);
+                    eq |= (lo == b1 ? 1u : 0u) << (2 * t) | (hi == b1 ? 2u : 0u) << (2 * t);
+                }
+                if (q >= n8) gt = eq = 0u;
+                gt <<= sh;
+                eq <<= sh;
+                gt |= __shfl_xor_sync(0xffffffffu, gt, 1);
+                eq |= __shfl_xor_sync(0xffffffffu, eq, 1);
+                gt |= __shfl_xor_sync(0xffffffffu, gt, 2);
+                eq |= __shfl_xor_sync(0xffffffffu, eq, 2);
+                if ((lane & 3) == 0 && q < n8) {
+                    s_maskw[q >> 2] = gt;
+                    s_candw[q >> 2] = eq;
+                }
+            }
+        }
     }
+    __syncthreads();
+    // the full rank keys of the candidates (a word's candidates belong to one thread, here and in
+    // the refinement)
+    for (int w = tid; w < n_words; w += TK_THREADS) {
+        unsigned u = s_candw[w];
+        while (u) {
+            const int col = w * 32 + __ffs(u) - 1;
+            u &= u - 1;
+            keys[col] = rank_key<CA>(__ldcg(x + col), CA ? __ldcg(stamp + col) : 0, gamma);
+        }
+    }
+    if (refine_candidates(keys, s, s_maskw, s_candw, n_words, krem1, mask_bits)) {
+        DIP_TRACE_MAX(tr, 2);
+        return;
+    }
+    // heavy ties: all keys in full, then the general path
+    for (int e = tid; e < d; e += TK_THREADS) keys[e] = rank_key<CA>(x[e], CA ? stamp[e] : 0, gamma);
+    __syncthreads();
+    general_select(keys, d, k, s, mask_bits);
     DIP_TRACE_MAX(tr, 2);
 }
 
@@ -642,13 +774,22 @@ residual_rmsnorm_kernel(const float *x, const float *y, int d, float *x_next)
 // host launchers
 // ---------------------------------------------------------------------------------------
 dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d, int k,
-                             float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream)
+                             float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream,
+                             const uint16_t *coarse)
 {
     const size_t smem = (size_t)((d + 3) & ~3) * sizeof(uint32_t);
     const dim3 grid(batch), block(TK_THREADS);
     unsigned long long *tr = dip_trace_slot(ctx, d <= 0 ? 0 : (stamp ? 2 : 1));
     cudaError_t e;
-    if (xb) {
+    if (coarse) {
+        if (xb || batch != 1 || (d & 31)) return DIP_ERR_INVALID_ARG;
+        if (stamp)
+            e = dip_launch_pdl(select_coarse_kernel<true>, grid, block, smem, stream, xa, coarse, d, k, gamma, stamp,
+                               mask_bits, tr);
+        else
+            e = dip_launch_pdl(select_coarse_kernel<false>, grid, block, smem, stream, xa, coarse, d, k, 1.0f,
+                               (const int32_t *)nullptr, mask_bits, tr);
+    } else if (xb) {
         if (stamp)
             e = dip_launch_pdl(select_kernel<true, true>, grid, block, smem, stream, xa, xb, x_out, d, k, gamma, stamp, mask_bits, tr);
         else
@@ -683,6 +824,8 @@ dip_status dip_init_mask_kernels(dip_ctx *ctx)
     DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_coarse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_coarse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(cache_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     return DIP_OK;
 }
