@@ -103,6 +103,9 @@ dip_status dip_create(dip_ctx **out, int device)
     }
     ctx->gemv_direct = 1;
     if (const char *e = getenv("DIP_GEMV_DIRECT")) ctx->gemv_direct = atoi(e) != 0;   // tuning aid: 0 = copy-ring kernel
+    // below ~4096 columns the whole of h and its stamps is a few KB and the plain select is as fast
+    ctx->coarse_min_d = 4096;
+    if (const char *e = getenv("DIP_COARSE_MIN_D")) ctx->coarse_min_d = atoi(e);       // tuning aid: smallest d_ff that ranks h from coarse keys
     ctx->n_tickets = N_TICKETS;
     const size_t vec = (size_t)DIP_MAX_BATCH * DIP_MAX_D;
     if ((st = dev_alloc(ctx, &ctx->partials, ctx->partials_floats)) != DIP_OK) return fail(st);
@@ -337,7 +340,8 @@ static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
     // h = (W~u x) * silu(W~g x)       (Eq. 2 inside Eq. 3)
     // (a single-token product also leaves the top bits of the rank keys of h for the next launch)
     dip_gemv_keys hk = {ctx->coarse, cache_d ? cache_d->stamp : nullptr, gamma, 0};
-    st = dip_launch_gemv(ctx, w, 0, x, batch, mask_x, nmax_x, h, s, nullptr, batch == 1 ? &hk : nullptr);
+    st = dip_launch_gemv(ctx, w, 0, x, batch, mask_x, nmax_x, h, s, nullptr,
+                         batch == 1 && w->d_ff >= ctx->coarse_min_d ? &hk : nullptr);
     if (st != DIP_OK) return st;
     // m_h = topK(score(h))            (Eq. 8: the GLU of the already sparsified gate/up)
     st = dip_launch_select(ctx, h, nullptr, nullptr, batch, w->d_ff, k_h, gamma,

@@ -39,6 +39,7 @@ struct dip_ctx {
     uint32_t *mask_ring; // [2][DIP_RING_LAYERS][DIP_MAX_D/32] per-layer mask slots of the stack runner
     uint32_t *mask_tmp;  // [DIP_MAX_D/32] list-based GEMV entry points
     uint16_t *coarse;    // [DIP_MAX_D] top 16 bits of the rank keys of h, left by the gate/up GEMV
+    int coarse_min_d;    // smallest d_ff for which the step ranks h from those
     int *status;         // sticky device status word (0 = fine)
     // the cache updates run beside the GEMVs: one side stream per cache kind
     cudaStream_t side[2];

@@ -568,9 +568,22 @@ select_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ c
     for (int w = tid; w < n_words; w += TK_THREADS) {
         unsigned u = s_candw[w];
         while (u) {
-            const int col = w * 32 + __ffs(u) - 1;
-            u &= u - 1;
-            keys[col] = rank_key<CA>(__ldcg(x + col), CA ? __ldcg(stamp + col) : 0, gamma);
+            // four columns at a time, their loads in flight together
+            int col[4], sv[4];
+            float xv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                col[i] = -1;
+                if (u) {
+                    col[i] = w * 32 + __ffs(u) - 1;
+                    u &= u - 1;
+                    xv[i] = __ldcg(x + col[i]);
+                    sv[i] = CA ? __ldcg(stamp + col[i]) : 0;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (col[i] >= 0) keys[col[i]] = rank_key<CA>(xv[i], sv[i], gamma);
         }
     }
     if (refine_candidates(keys, s, s_maskw, s_candw, n_words, krem1, mask_bits)) {

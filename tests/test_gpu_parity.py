@@ -259,6 +259,40 @@ def test_mlp_step_matches_oracle(dip, ctx, wtype, d_model, d_ff, rho, beta):
         assert rel_err(y, y_dense) <= REL_TOL
 
 
+@pytest.mark.parametrize("wtype,d_model,d_ff,rho,beta", [
+    (di.W_F32, 1024, 2816, 0.5, None),      # no cache: keys are |h|
+    (di.W_BF16, 1024, 4096, 0.1, 0.25),
+    (di.W_BF16, 1024, 2048, 0.5, 0.25),     # k > capacity: bypass
+    (di.W_BF16, 512, 1536, 1.0, 0.5),       # keep ratio 1: every column kept
+    (di.W_BF16, 256, 32, 0.25, 0.5),        # a single mask word
+])
+def test_mlp_step_ranking_h_from_the_gemv_keys(dip, wtype, d_model, d_ff, rho, beta, monkeypatch):
+    """A context that ranks h from the 16-bit keys left by the gate/up product at every size
+    (by default only wide layers do): same bit-exact masks and cache state."""
+    monkeypatch.setenv("DIP_COARSE_MIN_D", "0")
+    c = dip.Context(0)
+    try:
+        lw = _layer(31 + d_ff, d_model, d_ff, wtype)
+        w = upload_layer(dip, c, lw)
+        k_x, k_h = di.keep_count(rho, d_model), di.keep_count(rho, d_ff)
+        gamma = 0.2 if beta is not None else 1.0
+        ref_gu = ref_d = g_gu = g_d = None
+        if beta is not None:
+            ref_gu = oracle.Cache(d_model, di.cache_capacity(beta, d_model))
+            ref_d = oracle.Cache(d_ff, di.cache_capacity(beta, d_ff))
+            g_gu = dip.CacheState(d_model, ref_gu.capacity, "cuda")
+            g_d = dip.CacheState(d_ff, ref_d.capacity, "cuda")
+        wl = di.WORKLOADS["phi3_mini"].scaled(seed=d_ff + 1)
+        xs = di.token_inputs(wl, n_tokens=5, batch=1, d=d_model)[:, 0]
+        for x in xs:
+            _check_step(dip, c, lw, w, x, k_x, k_h, gamma, ref_gu, ref_d, g_gu, g_d)
+        # x = 0 makes every h_j zero: all rank keys tie and the lowest columns win (general path)
+        _check_step(dip, c, lw, w, np.zeros(d_model, dtype=np.float32), k_x, k_h, gamma, ref_gu, ref_d, g_gu, g_d)
+    finally:
+        torch.cuda.synchronize()
+        c.close()
+
+
 def test_full_size_phi3_medium_layer(dip, ctx):
     """One Phi-3-Medium-shaped block at the benchmark's keep ratios, all outputs checked."""
     wl = di.WORKLOADS["phi3_medium"]
