@@ -144,12 +144,12 @@ class ClockSampler:
 
 def ncu_traffic(w, keep_ratio, batch, algorithmic):
     """dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMV launch, from the ncu capture
-    summarised in profiles/kernels_phi3_medium_4layers_rho025.md (91.79 MB read + 2.21 MB written at
+    summarised in profiles/kernels_phi3_medium_4layers_rho025.md (91.87 MB read + 2.54 MB written at
     Phi-3-Medium shapes, keep ratio 0.25, one token).  Other keep ratios of the same workload scale
     with the kept bytes (the traffic is the kept rows); anything else has no capture."""
     if w.name != "phi3_medium" or batch != 1:
         return None
-    return 94.00e6 if abs(keep_ratio - 0.25) < 1e-9 else algorithmic * (94.00e6 / 91.85e6)
+    return 94.40e6 if abs(keep_ratio - 0.25) < 1e-9 else algorithmic * (94.40e6 / 91.85e6)
 
 
 def max_over_ranks(ms, dist, torch, device):
