@@ -142,14 +142,31 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def ncu_traffic(w, keep_ratio, batch, algorithmic):
-    """dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMV launch, from the ncu capture
-    summarised in profiles/kernels_phi3_medium_4layers_rho025.md (91.87 MB read + 2.54 MB written at
-    Phi-3-Medium shapes, keep ratio 0.25, one token).  Other keep ratios of the same workload scale
-    with the kept bytes (the traffic is the kept rows); anything else has no capture."""
-    if w.name != "phi3_medium" or batch != 1:
+# dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMV launch at Phi-3-Medium shapes, keep
+# ratio 0.25, one token, from the committed ncu capture (profiles/): bytes, and the kernel it is of.
+NCU_TRAFFIC = {"kernel": "gemv_direct_kernel", "bytes": 94.40e6,
+               "source": "profiles/kernels_phi3_medium_4layers_rho025.md"}
+
+
+def ncu_traffic(w, keep_ratio, batch, kernel_name):
+    """The committed capture's DRAM traffic per launch, only for the exact kernel, workload and keep
+    ratio it was taken on; null for anything else (nothing is extrapolated)."""
+    if w.name != "phi3_medium" or batch != 1 or abs(keep_ratio - 0.25) > 1e-9:
         return None
-    return 94.40e6 if abs(keep_ratio - 0.25) < 1e-9 else algorithmic * (94.40e6 / 91.85e6)
+    if not kernel_name.startswith(NCU_TRAFFIC["kernel"]):
+        return None
+    return NCU_TRAFFIC["bytes"]
+
+
+def median_repeat(ms_list):
+    """The median of the repeats' times (the upper one for an even count, so it is a measured repeat)."""
+    s = sorted(ms_list)
+    return s[len(s) // 2]
+
+
+def GATE_UP_KERNEL(w, batch):
+    """Name of the kernel that computes the gate/up product for this workload."""
+    return "gemv_direct_kernel" if batch == 1 and w.wtype != di.W_INT4_G128 else "gemv_kernel"
 
 
 def max_over_ranks(ms, dist, torch, device):
@@ -201,7 +218,7 @@ def build_stack(dip, ctx, torch, w, n_layers, rank):
 
 
 def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, warmup, use_graph=True,
-               kernel_pass=True, e2e_pass=True, sampler=None, dist=None, policy="lru"):
+               kernel_pass=True, e2e_pass=True, sampler=None, dist=None, policy="lru", min_timed_s=0.5, min_repeats=3):
     """Time `steps` decode tokens through the stack at one (keep ratio, cache budget)."""
     L, d_model, d_ff = len(layers), w.d_model, w.d_ff
     k_x, k_h = di.keep_count(keep_ratio, d_model), di.keep_count(keep_ratio, d_ff)
@@ -249,23 +266,37 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
             dist.barrier()
             torch.cuda.synchronize()
 
-    # ---- device-resident timing ----
+    def check_status(where):
+        st = ctx.device_status()
+        if st != 0:
+            raise SystemExit("device status %d after %s: a kernel gave up a bounded wait; no number is printed"
+                             % (st, where))
+
+    # ---- device-resident timing: the region of `steps` steps is repeated until at least
+    #      min_timed_s have been timed (and at least 3 times); the median repeat is reported ----
     for t in range(warmup):
         one_step(t)
     barrier()
     if sampler:
         sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for t in range(steps):
-        one_step(warmup + t)
-    e1.record(stream)
-    barrier()
+    reps, tok = [], warmup
+    while len(reps) < min_repeats or (sum(reps) < min_timed_s * 1e3 and len(reps) < 64):
+        barrier()
+        e0.record(stream)
+        for t in range(steps):
+            one_step(tok + t)
+        e1.record(stream)
+        barrier()
+        tok += steps
+        reps.append(max_over_ranks(e0.elapsed_time(e1), dist, torch, "cuda"))
     clocks = sampler.stop() if sampler else None
-    ms = e0.elapsed_time(e1)
-    ms = max_over_ranks(ms, dist, torch, "cuda")
+    check_status("the timed region")
+    ms = median_repeat(reps)
     res = {"keep_ratio": keep_ratio, "cache_budget": budget, "k_x": k_x, "k_h": k_h, "ms_total": ms,
            "ms_per_step": ms / steps, "mlp_steps_per_s": L * steps / (ms * 1e-3), "clocks": clocks,
+           "repeats": {"n": len(reps), "ms_min": min(reps), "ms_median": ms, "ms_max": max(reps),
+                       "timed_s": sum(reps) * 1e-3},
            "bytes": algorithmic_bytes(w, k_x, k_h, ca)}
     res["step_gbs"] = res["bytes"]["step"] * L * steps / (ms * 1e-3) / 1e9
     res["batch"] = batch
@@ -307,6 +338,7 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
         barrier()
         ms_e = e0.elapsed_time(e1)
         ms_e = max_over_ranks(ms_e, dist, torch, "cuda")
+        check_status("the end-to-end region")
         res["e2e"] = {"value": L * n_e2e / (ms_e * 1e-3), "unit": UNIT, "steps": n_e2e,
                       "h2d_bytes_per_step": 4 * d_model * batch, "d2h_bytes_per_step": 4 * d_model * batch,
                       "wall_ms": (time.perf_counter() - t0) * 1e3}
@@ -365,6 +397,7 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
             eb.record(stream)
             torch.cuda.synchronize()
             kern[name + "_train_us"] = ea.elapsed_time(eb) * 1e3 / (2 * L)
+        check_status("the per-kernel pass")
         res["kernels"] = kern
     return res
 
@@ -760,7 +793,7 @@ def write_report(dip, ctx, torch, path, steps):
                 xs = torch.from_numpy(di.token_inputs(w, n_tokens=n_tok, batch=B).copy())
                 xs = xs[:, 0] if B == 1 else xs
                 r = run_config(dip, ctx, torch, w, layers, xs, w.keep_ratio, None, min(steps, 64), 4,
-                               kernel_pass=False, e2e_pass=False)
+                               kernel_pass=False, e2e_pass=False, min_timed_s=0.1)
                 ud = r.get("union_density")
                 row(name, r, L, "union density x %.2f h %.2f" % (ud["x"], ud["h"]) if ud else "")
         else:
@@ -769,7 +802,8 @@ def write_report(dip, ctx, torch, path, steps):
             if name == "phi3_medium":
                 combos = [(r_, b_) for r_ in di.PHI3_MEDIUM_KEEP_RATIOS for b_ in di.PHI3_MEDIUM_CACHE_BUDGETS]
             for rho, beta in combos:
-                r = run_config(dip, ctx, torch, w, layers, xs, rho, beta, steps, 4, kernel_pass=False, e2e_pass=False)
+                r = run_config(dip, ctx, torch, w, layers, xs, rho, beta, steps, 4, kernel_pass=False, e2e_pass=False,
+                               min_timed_s=0.1)
                 extra = "hit rate %.2f" % r["hit_rate"] if "hit_rate" in r else ""
                 if name == "block_f32":
                     extra = "8 distinct blocks cycled (one block alone fits L2)"
@@ -782,10 +816,14 @@ def write_report(dip, ctx, torch, path, steps):
         f.write("\n".join(rows) + "\n")
 
 
-def oracle_rate(w, keep_ratio, budget, n_layers_sample, n_steps, warmup=0):
+def oracle_rate(w, keep_ratio, budget, n_layers_sample, n_steps, warmup=0, threads=None):
     """The CPU oracle as it stands, timed on this machine's host cores on a bounded sample of the
-    workload: `n_steps` MLP-steps cycling over `n_layers_sample` host-generated layers."""
+    workload: `n_steps` MLP-steps cycling over `n_layers_sample` host-generated layers.
+    threads: None = all cores the OpenMP runtime gives it; 1 = the single-thread leg."""
     import oracle
+    all_threads = oracle.num_threads()
+    if threads is not None:
+        oracle.set_num_threads(threads)
     k_x, k_h = di.keep_count(keep_ratio, w.d_model), di.keep_count(keep_ratio, w.d_ff)
     ca = budget is not None
     gamma = w.gamma if ca else 1.0
@@ -809,7 +847,10 @@ def oracle_rate(w, keep_ratio, budget, n_layers_sample, n_steps, warmup=0):
         if s >= warmup:
             times.append(time.perf_counter() - t0)
     total = float(np.sum(times))
-    return {"value": n_steps / total, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    used = oracle.num_threads()
+    if threads is not None:
+        oracle.set_num_threads(all_threads)
+    return {"value": n_steps / total, "unit": UNIT, "cores": used, "kind": "oracle",
             "sample": "%d MLP-steps over %d host-generated layer(s) of %s, keep ratio %g, cache budget %s"
                       % (n_steps, n_layers_sample, w.name, keep_ratio, budget),
             "ms_per_mlp_step": total / n_steps * 1e3}
@@ -865,7 +906,7 @@ def main():
         return main_two_tier(args, dip, ctx, torch, w, keep_ratio, budget, rank, world, local)
     L = args.layers if args.layers else w.n_layers
     layers = build_stack(dip, ctx, torch, w, L, rank)
-    n_tok = min(w.n_tokens, args.steps + args.warmup)
+    n_tok = w.n_tokens                                  # the repeats cycle through the workload's tokens
     wl_rank = w.scaled(seed=w.seed + 1000 * rank)
     if args.batch > 1:
         budget = None                                   # Algorithm 1 is per token
@@ -886,7 +927,7 @@ def main():
         for rho in di.PHI3_MEDIUM_KEEP_RATIOS:
             for beta in di.PHI3_MEDIUM_CACHE_BUDGETS:
                 r = run_config(dip, ctx, torch, w, layers, xs_host, rho, beta, min(args.steps, 64), 4,
-                               kernel_pass=True, e2e_pass=False)
+                               kernel_pass=True, e2e_pass=False, min_timed_s=0.1)
                 sweep.append(r)
 
     if rank != 0:
@@ -904,6 +945,7 @@ def main():
         gu_us = None
         achieved = head.get("union_gbs", head["step_gbs"])
     launches_per_step = L * (4 + (2 if budget is not None else 0)) + 1
+    kernel_name = GATE_UP_KERNEL(w, args.batch) + " (gate/up bundle)"
     line = {
         "metric": METRIC, "value": whole_job_rate(L * args.steps, world, head["ms_total"]), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["ms_per_step"],
@@ -917,6 +959,7 @@ def main():
                    "l2": "inputs larger than L2: %.1f GB of distinct layer weights cycled" % (sum(l.nbytes for l in layers) / 1e9),
                    "launch": "CUDA graph of dip_stack_step", "parallelism": "replicas only"},
         "mlp_step_us": head["ms_per_step"] * 1e3 / L,
+        "repeats": head["repeats"],
         "step_gbs": head["step_gbs"] * world,
         "step_frac_of_measured_hbm": head["step_gbs"] / peak,
         "step_frac_of_nominal_8tbs": head["step_gbs"] / NOMINAL_HBM_GBS,
@@ -925,10 +968,12 @@ def main():
         "clocks": head["clocks"],
         "e2e": {k: head["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
         "gpu_launches": launches_per_step * args.steps,
-        "roofline": {"bound": "hbm", "kernel": "gemv_direct_kernel (gate/up bundle)" if args.batch == 1 and w.wtype != di.W_INT4_G128 else "gemv_kernel (gate/up bundle)", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                      "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS, "bytes_per_launch": gu_bytes,
-                     "us_per_launch": gu_us, "traffic": ncu_traffic(w, keep_ratio, args.batch, gu_bytes)},
+                     "us_per_launch": gu_us, "traffic": ncu_traffic(w, keep_ratio, args.batch, kernel_name),
+                     "traffic_source": "committed ncu capture (%s); null when this run's kernel or workload differs"
+                                       % NCU_TRAFFIC["source"]},
         "kernels_us": head.get("kernels"),
         "union_density": head.get("union_density"),
     }
@@ -946,6 +991,8 @@ def main():
         torch.cuda.empty_cache()
         line["cpu_baseline"] = {k: v for k, v in oracle_rate(w, keep_ratio, budget, 1, 60).items()
                                 if k in ("value", "unit", "cores", "kind", "sample")}
+        one = oracle_rate(w, keep_ratio, budget, 1, 8, threads=1)
+        line["cpu_baseline"]["single_thread"] = {k: one[k] for k in ("value", "unit", "cores", "sample")}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -27,7 +27,8 @@
  *    it, and is joined back into `stream` before the call's work ends.
  *  - Arguments are validated on the host before anything is launched; a failed
  *    validation returns an error code and launches nothing.
- *  - Data pointers must be 16-byte aligned.
+ *  - Data pointers (vectors, masks, cache state, weights) must be 16-byte
+ *    aligned; a misaligned one is DIP_ERR_INVALID_ARG.
  *  - Float vectors are binary32.  Masks are bit sets: bit (i & 31) of word
  *    (i >> 5) is column i.  Kept-index lists are int32 in ascending order.
  *  - Top-k ties are resolved in favour of the lower column index, so every
@@ -68,10 +69,38 @@ enum {
 
 typedef struct dip_ctx dip_ctx;   /* opaque; owns scratch workspace on one device */
 
+/* Options of a context.  A zeroed struct gives the defaults; the library reads no
+ * environment variable and has no other global switch.
+ *   max_d, max_batch   size the workspace: the largest d_model / d_ff and the most tokens per
+ *                      call that this context will see (0 = DIP_MAX_D / DIP_MAX_BATCH).  A call
+ *                      beyond them returns DIP_ERR_WORKSPACE.
+ *   gemv_segment_bytes 0 = chosen per launch; 512, 1024 or 2048 force the segment of a packed
+ *                      row that one thread block of the copy-ring product kernel handles.
+ *   gemv_copy_ring     non-zero: single-token F32 / BF16 products also go through the
+ *                      copy-ring kernel (by default they use the plain-load kernel).
+ *   coarse_min_d       smallest d_ff for which a single-token step ranks h from the 16-bit keys
+ *                      that the gate/up product leaves behind: 0 = default (4096), negative =
+ *                      every size.  Either way the masks are the same bits.
+ *   wait_limit_us      bound of every in-kernel wait on an asynchronous copy, in microseconds
+ *                      (0 = one second); see dip_device_status. */
+typedef struct {
+    int32_t max_d;
+    int32_t max_batch;
+    int32_t gemv_segment_bytes;
+    int32_t gemv_copy_ring;
+    int32_t coarse_min_d;
+    int32_t wait_limit_us;
+    int32_t reserved[4];          /* keep zero */
+} dip_options;
+
 /* Create a context on `device` (a CUDA ordinal).  Allocates the scratch
- * workspace (a few MB) with cudaMalloc; no other call allocates.  *out is
- * NULL on failure. */
+ * workspace (about 50 MB at the default sizes) with cudaMalloc; no other call
+ * allocates.  *out is NULL on failure.  The calling thread's current device is
+ * left as it was.  Every later call on the context must be made with `device`
+ * current (DIP_ERR_INVALID_ARG otherwise). */
 dip_status dip_create(dip_ctx **out, int device);
+/* The same with options (NULL = defaults). */
+dip_status dip_create_ex(dip_ctx **out, int device, const dip_options *options);
 /* Frees the workspace.  The caller makes sure no work of this context is in flight. */
 dip_status dip_destroy(dip_ctx *ctx);
 /* Static description of a status code (host string, never NULL). */
@@ -83,9 +112,21 @@ const char *dip_last_error(const dip_ctx *ctx);
 int dip_sm_count(const dip_ctx *ctx);
 /* Every wait inside a kernel (on the arrival of an asynchronous copy) is bounded.  If one runs
  * out, the kernel stops early, its outputs are invalid and a sticky status word on the device
- * becomes non-zero.  This call waits for `stream`, then copies the word to *status_out (host):
- * 0 = no kernel of this context has given up a wait. */
+ * becomes non-zero.  This call waits for `stream`, then copies the word to *status_out (host). */
+typedef enum {
+    DIP_DEVICE_OK = 0,
+    DIP_DEVICE_WAIT_TIMEOUT = 1,        /* a kernel gave up a bounded wait                          */
+    DIP_DEVICE_TIER_INCONSISTENT = 2    /* two-tier step: slot table and cache state disagree       */
+} dip_device_status_word;
 dip_status dip_device_status(dip_ctx *ctx, int *status_out, void *stream);
+/* Clears the sticky word (enqueued on `stream`). */
+dip_status dip_reset_device_status(dip_ctx *ctx, void *stream);
+/* Self-test of the bounded wait (diagnostics): enqueues one tiny kernel that waits, with the
+ * given limit, for a copy that is never issued.  The wait runs out, the kernel returns, and the
+ * status word becomes DIP_DEVICE_WAIT_TIMEOUT; nothing else is touched and the context stays
+ * usable.  waited_ns (device uint64, may be NULL) receives how long the kernel waited.
+ * 1 <= limit_us <= 1000000. */
+dip_status dip_selftest_bounded_wait(dip_ctx *ctx, int limit_us, unsigned long long *waited_ns, void *stream);
 
 /* ------------------------------------------------------------------------
  * Timeline of the library's own kernels (diagnostics; off by default).  Between
@@ -301,6 +342,27 @@ dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *lay
                           const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
                           float *x_out, float *y_last, void *stream);
 
+/* dip_stack_step that also keeps every layer's intermediates (for checking a stack layer by
+ * layer against Eq. 7-8 and Algorithm 1): the same kernels in the same order, writing into the
+ * caller's arrays instead of the context's workspace.  All arrays are required, device memory,
+ * 16-byte aligned:
+ *   x      [n_layers][batch][d_model]   x_l, the input of layer l (x_0 = x_in)
+ *   mask_x [n_layers][batch][d_model/32]
+ *   h      [n_layers][batch][d_ff]
+ *   mask_h [n_layers][batch][d_ff/32]
+ *   y      [n_layers][batch][d_model]   the MLP output of layer l */
+typedef struct {
+    float *x;
+    uint32_t *mask_x;
+    float *h;
+    uint32_t *mask_h;
+    float *y;
+} dip_stack_probe;
+dip_status dip_stack_step_probed(dip_ctx *ctx, int n_layers, const dip_mlp_weights *layers,
+                                 const float *x_in, int batch, int k_x, int k_h, float gamma,
+                                 const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                                 float *x_out, const dip_stack_probe *probe, void *stream);
+
 /* ------------------------------------------------------------------------
  * Gate pruning and Up pruning (Sec. 3.2, Eq. 5), the neuron-wise schedules the
  * paper compares DIP with: one of the two first-layer products is computed
@@ -429,7 +491,9 @@ dip_status dip_mlp_step_tiered(dip_ctx *ctx, const dip_mlp_weights *w,
  * Limits: d_model <= 16384 (DIP_ERR_WORKSPACE beyond it: the fixed array
  * cannot hold the partial sums), d_model % 32 == 0, 1 <= n_kept <= d_ff <=
  * DIP_MAX_D; INT4 weights return DIP_ERR_UNSUPPORTED.  Only w->wtype,
- * w->d_model, w->d_ff and w->down are read.
+ * w->d_model, w->d_ff and w->down are read.  kept_idx lists each kept column
+ * once (ascending, as dip_mask_topk writes it); an entry outside [0, d_ff) is
+ * skipped, a repeated entry is counted as often as it appears.
  *
  * All calls on a device share the one array, which keeps the previous call's
  * contents (each call clears the counters it needs on `stream` first).  Two

@@ -25,8 +25,12 @@ _lib = C.CDLL(_os.environ.get("DIP_ORACLE_LIB") or _build.build())
 _vp, _i32, _f32, _f64 = C.c_void_p, C.c_int, C.c_float, C.c_double
 
 _lib.orc_num_threads.restype = _i32
+_lib.orc_set_num_threads.restype = None
+_lib.orc_set_num_threads.argtypes = [_i32]
 _lib.orc_silu.restype = _f64
 _lib.orc_silu.argtypes = [_f64]
+_lib.orc_glu.restype = None
+_lib.orc_glu.argtypes = [_vp, _vp, _i32, _vp]
 _lib.orc_weight.restype = _f64
 _lib.orc_weight.argtypes = [_i32, _vp, _vp, _i32, _i32, _i32, _i32]
 _lib.orc_rank_key.restype = C.c_uint32
@@ -75,8 +79,22 @@ def num_threads() -> int:
     return int(_lib.orc_num_threads())
 
 
+def set_num_threads(n: int) -> None:
+    """Threads the oracle's parallel loops use from now on (timing legs only; results do not change)."""
+    _lib.orc_set_num_threads(int(n))
+
+
 def silu(z: float) -> float:
     return float(_lib.orc_silu(float(z)))
+
+
+def glu(g: np.ndarray, u: np.ndarray) -> np.ndarray:
+    """Eq. 2 element-wise: u * silu(g), fp64."""
+    g = _chk(np.ascontiguousarray(g), np.float64)
+    u = _chk(np.ascontiguousarray(u), np.float64, g.size)
+    h = np.empty(g.size, dtype=np.float64)
+    _lib.orc_glu(_p(g), _p(u), g.size, _p(h))
+    return h
 
 
 def rank_key(x: float, resident: bool, gamma: float) -> int:

@@ -44,6 +44,18 @@ int orc_num_threads(void)
 #endif
 }
 
+/* Threads used by the parallel loops from now on (the benchmark's single-thread
+ * timing leg); every sum still runs in one thread, so results do not change. */
+void orc_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1)
+        omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /* ------------------------------------------------------------------ *
  * Stored-number decoding (formats, not method arithmetic).
  * ------------------------------------------------------------------ */
@@ -105,6 +117,14 @@ double orc_weight(int type, const void *w, const uint16_t *scales,
 double orc_silu(double z)
 {
     return z / (1.0 + exp(-z));
+}
+
+/* Eq. 2, element-wise: h_j = u_j * silu(g_j) for given pre-activations
+ * (u = W^u x, g = W^g x, dense or sparsified), in fp64. */
+void orc_glu(const double *g, const double *u, int n, double *h)
+{
+    for (int j = 0; j < n; ++j)
+        h[j] = u[j] * orc_silu(g[j]);
 }
 
 /* ------------------------------------------------------------------ *

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libdip.so")
 W_F32, W_BF16, W_INT4_G128 = 0, 1, 2
 MAX_D, MAX_BATCH, INT4_GROUP, CACHE_META_INTS = 32768, 16, 128, 8
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_WORKSPACE = 0, 1, 2, 3, 4
+DEVICE_OK, DEVICE_WAIT_TIMEOUT, DEVICE_TIER_INCONSISTENT = 0, 1, 2
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -43,8 +44,24 @@ class StepOutputsStruct(C.Structure):
                 ("union_counts", _vp)]
 
 
+class OptionsStruct(C.Structure):
+    _fields_ = [("max_d", C.c_int32), ("max_batch", C.c_int32), ("gemv_segment_bytes", C.c_int32),
+                ("gemv_copy_ring", C.c_int32), ("coarse_min_d", C.c_int32), ("wait_limit_us", C.c_int32),
+                ("reserved", C.c_int32 * 4)]
+
+
+class StackProbeStruct(C.Structure):
+    _fields_ = [("x", _vp), ("mask_x", _vp), ("h", _vp), ("mask_h", _vp), ("y", _vp)]
+
+
 _lib.dip_create.restype = _i32
 _lib.dip_create.argtypes = [C.POINTER(_vp), _i32]
+_lib.dip_create_ex.restype = _i32
+_lib.dip_create_ex.argtypes = [C.POINTER(_vp), _i32, C.POINTER(OptionsStruct)]
+_lib.dip_reset_device_status.restype = _i32
+_lib.dip_reset_device_status.argtypes = [_vp, _vp]
+_lib.dip_selftest_bounded_wait.restype = _i32
+_lib.dip_selftest_bounded_wait.argtypes = [_vp, _i32, _vp, _vp]
 _lib.dip_destroy.restype = _i32
 _lib.dip_destroy.argtypes = [_vp]
 _lib.dip_status_string.restype = C.c_char_p
@@ -76,7 +93,10 @@ _lib.dip_residual_rmsnorm.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp, _vp]
 _lib.dip_stack_step.restype = _i32
 _lib.dip_stack_step.argtypes = [_vp, _i32, C.POINTER(MlpWeightsStruct), _vp, _i32, _i32, _i32, _f32,
                                 C.POINTER(CacheStateStruct), C.POINTER(CacheStateStruct), _vp, _vp, _vp]
-
+_lib.dip_stack_step_probed.restype = _i32
+_lib.dip_stack_step_probed.argtypes = [_vp, _i32, C.POINTER(MlpWeightsStruct), _vp, _i32, _i32, _i32, _f32,
+                                       C.POINTER(CacheStateStruct), C.POINTER(CacheStateStruct), _vp,
+                                       C.POINTER(StackProbeStruct), _vp]
 
 
 class TierStruct(C.Structure):
@@ -103,8 +123,9 @@ _lib.dip_mlp_step_neuron_pruned.argtypes = [_vp, C.POINTER(NeuronWeightsStruct),
 _lib.dip_sparse_gemv_down_noalloc.restype = _i32
 _lib.dip_sparse_gemv_down_noalloc.argtypes = [C.POINTER(MlpWeightsStruct), _vp, _vp, _i32, _vp, _vp]
 
-EXPORTED = ["dip_create", "dip_destroy", "dip_status_string", "dip_last_error", "dip_sm_count",
-            "dip_device_status", "dip_trace_begin", "dip_trace_reset", "dip_trace_read", "dip_trace_end",
+EXPORTED = ["dip_create", "dip_create_ex", "dip_destroy", "dip_status_string", "dip_last_error", "dip_sm_count",
+            "dip_device_status", "dip_reset_device_status", "dip_selftest_bounded_wait", "dip_stack_step_probed",
+            "dip_trace_begin", "dip_trace_reset", "dip_trace_read", "dip_trace_end",
             "dip_packed_bytes", "dip_pack_weights", "dip_mask_topk", "dip_ca_mask",
             "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_mlp_step",
             "dip_residual_rmsnorm", "dip_stack_step", "dip_mlp_step_tiered", "dip_mlp_step_neuron_pruned",
@@ -143,13 +164,17 @@ def _stream() -> int:
 class Context:
     """A dip_ctx: scratch workspace on one device.  Not for concurrent use from several streams."""
 
-    def __init__(self, device: int = 0):
+    def __init__(self, device: int = 0, max_d: int = 0, max_batch: int = 0, gemv_segment_bytes: int = 0,
+                 gemv_copy_ring: bool = False, coarse_min_d: int = 0, wait_limit_us: int = 0):
+        """The keyword arguments are the fields of dip_options (0 = the library's default)."""
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2412_01380_b200 needs a CUDA device; there is no CPU path")
         h = _vp()
-        st = _lib.dip_create(C.byref(h), int(device))
+        opt = OptionsStruct(int(max_d), int(max_batch), int(gemv_segment_bytes), int(bool(gemv_copy_ring)),
+                            int(coarse_min_d), int(wait_limit_us))
+        st = _lib.dip_create_ex(C.byref(h), int(device), C.byref(opt))
         if st != OK:
-            raise DipError(st, "dip_create")
+            raise DipError(st, "dip_create_ex")
         self.handle = h
         self.device = int(device)
 
@@ -166,6 +191,13 @@ class Context:
         out = C.c_int(-1)
         self.check(_lib.dip_device_status(self.handle, C.byref(out), _stream()))
         return out.value
+
+    def reset_device_status(self) -> None:
+        self.check(_lib.dip_reset_device_status(self.handle, _stream()))
+
+    def selftest_bounded_wait(self, limit_us: int, waited_ns: Optional[torch.Tensor] = None) -> None:
+        """Enqueue the tiny kernel whose bounded wait runs out (device status becomes 1)."""
+        self.check(_lib.dip_selftest_bounded_wait(self.handle, int(limit_us), _ptr(waited_ns), _stream()))
 
     def trace_begin(self) -> None:
         self.check(_lib.dip_trace_begin(self.handle))
@@ -378,6 +410,26 @@ def dip_stack_step(ctx: Context, stack: Stack, x_in: torch.Tensor, k_x: int, k_h
     ctx.check(_lib.dip_stack_step(ctx.handle, len(stack.layers), stack.w_arr, _ptr(x_in), batch, int(k_x),
                                   int(k_h), float(gamma), stack.gu_arr, stack.d_arr, _ptr(x_out),
                                   _ptr(y_last), _stream()))
+
+
+class StackProbe:
+    """Per-layer intermediates of one dip_stack_step_probed call (device tensors owned here)."""
+
+    def __init__(self, n_layers: int, batch: int, d_model: int, d_ff: int, device):
+        self.x = torch.empty((n_layers, batch, d_model), device=device)
+        self.mask_x = torch.zeros((n_layers, batch, d_model // 32), dtype=torch.int32, device=device)
+        self.h = torch.empty((n_layers, batch, d_ff), device=device)
+        self.mask_h = torch.zeros((n_layers, batch, d_ff // 32), dtype=torch.int32, device=device)
+        self.y = torch.empty((n_layers, batch, d_model), device=device)
+        self.struct = StackProbeStruct(_ptr(self.x), _ptr(self.mask_x), _ptr(self.h), _ptr(self.mask_h), _ptr(self.y))
+
+
+def dip_stack_step_probed(ctx: Context, stack: Stack, x_in: torch.Tensor, k_x: int, k_h: int, gamma: float,
+                          x_out: torch.Tensor, probe: StackProbe) -> None:
+    batch = 1 if x_in.dim() == 1 else x_in.shape[0]
+    ctx.check(_lib.dip_stack_step_probed(ctx.handle, len(stack.layers), stack.w_arr, _ptr(x_in), batch, int(k_x),
+                                         int(k_h), float(gamma), stack.gu_arr, stack.d_arr, _ptr(x_out),
+                                         C.byref(probe.struct), _stream()))
 
 
 def dip_sparse_gemv_down_noalloc(w: MlpWeights, h: torch.Tensor, kept_idx: torch.Tensor, n_kept: int,

@@ -60,6 +60,26 @@ template <typename T> dip_status dev_alloc(dip_ctx *ctx, T **p, size_t n)
     return DIP_OK;
 }
 
+// The context exists and its device is the calling thread's current one.
+bool ctx_ok(const dip_ctx *ctx)
+{
+    int dev = -1;
+    return ctx && cudaGetDevice(&dev) == cudaSuccess && dev == ctx->device;
+}
+
+// Shapes within what the context's workspace was sized for.
+bool fits(const dip_ctx *ctx, int d_a, int d_b, int batch)
+{
+    return d_a <= ctx->max_d && d_b <= ctx->max_d && batch <= ctx->max_batch;
+}
+
+bool opt_aligned16(const void *p) { return !p || dip_aligned16(p); }
+
+bool outputs_aligned(const dip_step_outputs *o)
+{
+    return !o || (opt_aligned16(o->mask_x) && opt_aligned16(o->mask_h) && opt_aligned16(o->h));
+}
+
 }  // namespace
 
 extern "C" {
@@ -79,35 +99,45 @@ const char *dip_status_string(dip_status s)
 const char *dip_last_error(const dip_ctx *ctx) { return ctx ? ctx->err : ""; }
 int dip_sm_count(const dip_ctx *ctx) { return ctx ? ctx->sm_count : 0; }
 
-dip_status dip_create(dip_ctx **out, int device)
+dip_status dip_create(dip_ctx **out, int device) { return dip_create_ex(out, device, nullptr); }
+
+dip_status dip_create_ex(dip_ctx **out, int device, const dip_options *opt)
 {
     if (!out) return DIP_ERR_INVALID_ARG;
     *out = nullptr;
+    dip_options o = {};
+    if (opt) o = *opt;
+    if (o.max_d < 0 || o.max_d > DIP_MAX_D || o.max_batch < 0 || o.max_batch > DIP_MAX_BATCH) return DIP_ERR_INVALID_ARG;
+    if (o.gemv_segment_bytes != 0 && o.gemv_segment_bytes != 512 && o.gemv_segment_bytes != 1024 &&
+        o.gemv_segment_bytes != 2048)
+        return DIP_ERR_INVALID_ARG;
+    if (o.wait_limit_us < 0) return DIP_ERR_INVALID_ARG;
+    int prev_device = -1;
+    if (cudaGetDevice(&prev_device) != cudaSuccess) return DIP_ERR_CUDA;
     dip_ctx *ctx = new (std::nothrow) dip_ctx();
     if (!ctx) return DIP_ERR_CUDA;
     memset(ctx, 0, sizeof(*ctx));
     ctx->device = device;
     dip_status st = DIP_OK;
     auto fail = [&](dip_status s) {
-        // keep the message readable through a static copy: the context is about to go
         dip_destroy(ctx);
+        cudaSetDevice(prev_device);
         return s;
     };
     if (cudaSetDevice(device) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
         return fail(DIP_ERR_CUDA);
-    ctx->partials_floats = PARTIALS_FLOATS;
-    if (const char *e = getenv("DIP_GEMV_SEG")) {          // tuning aid: force the GEMV segment width
-        const int v = atoi(e);
-        if (v == 512 || v == 1024 || v == 2048) ctx->gemv_seg = v;
-    }
-    ctx->gemv_direct = 1;
-    if (const char *e = getenv("DIP_GEMV_DIRECT")) ctx->gemv_direct = atoi(e) != 0;   // tuning aid: 0 = copy-ring kernel
+    ctx->max_d = o.max_d ? (o.max_d + 127) / 128 * 128 : DIP_MAX_D;
+    ctx->max_batch = o.max_batch ? o.max_batch : DIP_MAX_BATCH;
+    ctx->gemv_seg = o.gemv_segment_bytes;
+    ctx->gemv_direct = o.gemv_copy_ring ? 0 : 1;
     // below ~4096 columns the whole of h and its stamps is a few KB and the plain select is as fast
-    ctx->coarse_min_d = 4096;
-    if (const char *e = getenv("DIP_COARSE_MIN_D")) ctx->coarse_min_d = atoi(e);       // tuning aid: smallest d_ff that ranks h from coarse keys
+    ctx->coarse_min_d = o.coarse_min_d == 0 ? 4096 : (o.coarse_min_d < 0 ? 0 : o.coarse_min_d);
+    ctx->wait_limit_ns = o.wait_limit_us ? 1000ull * (unsigned long long)o.wait_limit_us : 1000000000ull;
+    // split-row partial sums: up to one part per SM of a whole output row per token
+    ctx->partials_floats = PARTIALS_FLOATS;
     ctx->n_tickets = N_TICKETS;
-    const size_t vec = (size_t)DIP_MAX_BATCH * DIP_MAX_D;
+    const size_t vec = (size_t)ctx->max_batch * ctx->max_d;
     if ((st = dev_alloc(ctx, &ctx->partials, ctx->partials_floats)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->tickets, (size_t)N_TICKETS)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->h, vec)) != DIP_OK) return fail(st);
@@ -115,16 +145,16 @@ dip_status dip_create(dip_ctx **out, int device)
     if ((st = dev_alloc(ctx, &ctx->y2, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->xa, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->xb, vec)) != DIP_OK) return fail(st);
-    if ((st = dev_alloc(ctx, &ctx->p, (size_t)DIP_MAX_D)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->p, (size_t)ctx->max_d)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask, vec / 32)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->idx, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask_h, vec / 32)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->idx_h, vec)) != DIP_OK) return fail(st);
-    if ((st = dev_alloc(ctx, &ctx->union_idx, (size_t)DIP_MAX_D)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->union_idx, (size_t)ctx->max_d)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->counts, (size_t)8)) != DIP_OK) return fail(st);
-    if ((st = dev_alloc(ctx, &ctx->mask_ring, (size_t)2 * DIP_RING_LAYERS * (DIP_MAX_D / 32))) != DIP_OK) return fail(st);
-    if ((st = dev_alloc(ctx, &ctx->mask_tmp, (size_t)(DIP_MAX_D / 32))) != DIP_OK) return fail(st);
-    if ((st = dev_alloc(ctx, &ctx->coarse, (size_t)DIP_MAX_D)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->mask_ring, (size_t)2 * DIP_RING_LAYERS * (ctx->max_d / 32))) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->mask_tmp, (size_t)(ctx->max_d / 32))) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->coarse, (size_t)ctx->max_d)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->status, (size_t)1)) != DIP_OK) return fail(st);
     if (cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if ((st = dev_alloc(ctx, &ctx->trace, (size_t)DIP_TRACE_SLOTS * DIP_TRACE_WORDS)) != DIP_OK) return fail(st);
@@ -143,6 +173,7 @@ dip_status dip_create(dip_ctx **out, int device)
     if (cudaMemset(ctx->tickets, 0, N_TICKETS * sizeof(unsigned int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if (cudaMemset(ctx->counts, 0, 8 * sizeof(int32_t)) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if ((st = dip_init_mask_kernels(ctx)) != DIP_OK) return fail(st);
+    if (cudaSetDevice(prev_device) != cudaSuccess) return fail(DIP_ERR_CUDA);
     *out = ctx;
     return DIP_OK;
 }
@@ -199,7 +230,10 @@ dip_status dip_pack_weights(dip_ctx *ctx, int wtype, int d_model, int d_ff,
                             const void *Sg, const void *Su, const void *Sd,
                             const dip_mlp_weights *out, void *stream)
 {
-    if (!ctx || !Wg || !Wu || !Wd || !out) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx) || !Wg || !Wu || !Wd || !out) return DIP_ERR_INVALID_ARG;
+    if (!dip_aligned16(Wg) || !dip_aligned16(Wu) || !dip_aligned16(Wd) || !opt_aligned16(Sg) || !opt_aligned16(Su) ||
+        !opt_aligned16(Sd))
+        return DIP_ERR_INVALID_ARG;
     if (!weights_ok(out) || out->wtype != wtype || out->d_model != d_model || out->d_ff != d_ff)
         return DIP_ERR_INVALID_ARG;
     if (wtype == DIP_W_INT4_G128 && (!Sg || !Su || !Sd)) return DIP_ERR_INVALID_ARG;
@@ -208,10 +242,23 @@ dip_status dip_pack_weights(dip_ctx *ctx, int wtype, int d_model, int d_ff,
 
 dip_status dip_device_status(dip_ctx *ctx, int *status_out, void *stream)
 {
-    if (!ctx || !status_out) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx) || !status_out) return DIP_ERR_INVALID_ARG;
     DIP_CUDA_TRY(ctx, cudaMemcpyAsync(status_out, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     DIP_CUDA_TRY(ctx, cudaStreamSynchronize((cudaStream_t)stream));
     return DIP_OK;
+}
+
+dip_status dip_reset_device_status(dip_ctx *ctx, void *stream)
+{
+    if (!ctx_ok(ctx)) return DIP_ERR_INVALID_ARG;
+    DIP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->status, 0, sizeof(int), (cudaStream_t)stream));
+    return DIP_OK;
+}
+
+dip_status dip_selftest_bounded_wait(dip_ctx *ctx, int limit_us, unsigned long long *waited_ns, void *stream)
+{
+    if (!ctx_ok(ctx) || limit_us < 1 || limit_us > 1000000) return DIP_ERR_INVALID_ARG;
+    return dip_launch_bounded_wait_selftest(ctx, 1000ull * (unsigned long long)limit_us, waited_ns, (cudaStream_t)stream);
 }
 
 // Run the cache update of one masked input beside the main stream (side stream `which`).
@@ -241,8 +288,9 @@ static dip_status join_cache_updates(dip_ctx *ctx, cudaStream_t main)
 dip_status dip_mask_topk(dip_ctx *ctx, const float *x, int batch, int d, int k,
                          uint32_t *mask_bits, int32_t *kept_idx, void *stream)
 {
-    if (!ctx || !x || !dip_aligned16(x)) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx) || !x || !dip_aligned16(x) || !opt_aligned16(mask_bits)) return DIP_ERR_INVALID_ARG;
     if (batch < 1 || batch > DIP_MAX_BATCH || d < 1 || d > DIP_MAX_D || k < 1 || k > d) return DIP_ERR_INVALID_ARG;
+    if (!fits(ctx, d, 0, batch)) return DIP_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
     uint32_t *m = mask_bits ? mask_bits : ctx->mask;
     dip_status st = dip_launch_select(ctx, x, nullptr, nullptr, batch, d, k, 1.0f, nullptr, m, s);
@@ -254,10 +302,11 @@ dip_status dip_ca_mask(dip_ctx *ctx, const float *x, int d, int k, float gamma,
                        const dip_cache_state *st,
                        uint32_t *mask_bits, int32_t *kept_idx, void *stream)
 {
-    if (!ctx || !x || !dip_aligned16(x)) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx) || !x || !dip_aligned16(x) || !opt_aligned16(mask_bits)) return DIP_ERR_INVALID_ARG;
     if (d < 1 || d > DIP_MAX_D || k < 1 || k > d) return DIP_ERR_INVALID_ARG;
     if (!(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
     if (!cache_ok(st, d)) return DIP_ERR_INVALID_ARG;
+    if (!fits(ctx, d, 0, 1)) return DIP_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
     uint32_t *m = mask_bits ? mask_bits : ctx->mask;
     dip_status rc = dip_launch_select(ctx, x, nullptr, nullptr, 1, d, k, gamma, st->stamp, m, s);
@@ -271,9 +320,10 @@ static dip_status gemv_entry(dip_ctx *ctx, const dip_mlp_weights *w, int which, 
                              const int32_t *kept_idx, int n_kept, const uint32_t *mask_bits,
                              float *out, void *stream)
 {
-    if (!ctx || !weights_ok(w) || !v || !out) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx) || !weights_ok(w) || !v || !out) return DIP_ERR_INVALID_ARG;
     if (!kept_idx && !mask_bits) return DIP_ERR_INVALID_ARG;
-    if (!dip_aligned16(v) || !dip_aligned16(out)) return DIP_ERR_INVALID_ARG;
+    if (!dip_aligned16(v) || !dip_aligned16(out) || !opt_aligned16(mask_bits)) return DIP_ERR_INVALID_ARG;
+    if (!fits(ctx, w->d_model, w->d_ff, batch)) return DIP_ERR_WORKSPACE;
     const int d_in = which == 0 ? w->d_model : w->d_ff;
     if (batch < 1 || batch > DIP_MAX_BATCH || n_kept < 1 || n_kept > d_in) return DIP_ERR_INVALID_ARG;
     if (batch > 1 && !mask_bits) return DIP_ERR_INVALID_ARG;
@@ -315,9 +365,10 @@ static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
     const float *x = xb ? x_norm : xa;
     if (!ctx || !weights_ok(w) || !xa || !x || !y || !dip_aligned16(xa) || !dip_aligned16(x) || !dip_aligned16(y))
         return DIP_ERR_INVALID_ARG;
-    if (batch < 1 || batch > DIP_MAX_BATCH) return DIP_ERR_INVALID_ARG;
+    if (batch < 1 || batch > DIP_MAX_BATCH || !outputs_aligned(out)) return DIP_ERR_INVALID_ARG;
     if (k_x < 1 || k_x > w->d_model || k_h < 1 || k_h > w->d_ff) return DIP_ERR_INVALID_ARG;
     if (!(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
+    if (!fits(ctx, w->d_model, w->d_ff, batch)) return DIP_ERR_WORKSPACE;
     if (cache_gu && !cache_ok(cache_gu, w->d_model)) return DIP_ERR_INVALID_ARG;
     if (cache_d && !cache_ok(cache_d, w->d_ff)) return DIP_ERR_INVALID_ARG;
     if (batch > 1 && (cache_gu || cache_d)) return DIP_ERR_UNSUPPORTED;   // Algorithm 1 is per token
@@ -368,7 +419,7 @@ dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
                         const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
                         float *y, const dip_step_outputs *out, void *stream)
 {
-    if (!ctx) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx)) return DIP_ERR_INVALID_ARG;
     return step_impl(ctx, w, x, nullptr, nullptr, batch, k_x, k_h, gamma, cache_gu, cache_d, y, out,
                      ctx->mask, ctx->mask_h, false, stream);
 }
@@ -413,8 +464,10 @@ dip_status dip_mlp_step_tiered(dip_ctx *ctx, const dip_mlp_weights *w,
                                const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
                                float *y, const dip_step_outputs *out, void *stream)
 {
-    if (!ctx || !w || !dims_ok(w->wtype, w->d_model, w->d_ff) || !x || !y || !dip_aligned16(x) || !dip_aligned16(y))
+    if (!ctx_ok(ctx) || !w || !dims_ok(w->wtype, w->d_model, w->d_ff) || !x || !y || !dip_aligned16(x) ||
+        !dip_aligned16(y) || !outputs_aligned(out))
         return DIP_ERR_INVALID_ARG;
+    if (!fits(ctx, w->d_model, w->d_ff, 1)) return DIP_ERR_WORKSPACE;
     if (w->wtype == DIP_W_INT4_G128 &&
         (!w->gate_up_scales || !w->down_scales || !dip_aligned16(w->gate_up_scales) || !dip_aligned16(w->down_scales)))
         return DIP_ERR_INVALID_ARG;
@@ -454,9 +507,11 @@ dip_status dip_mlp_step_neuron_pruned(dip_ctx *ctx, const dip_neuron_weights *w,
                                       float *p_out, uint32_t *mask_out, int32_t *idx_out, float *h_out,
                                       void *stream)
 {
-    if (!ctx || !w || !x || !y || !dip_aligned16(x) || !dip_aligned16(y)) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx) || !w || !x || !y || !dip_aligned16(x) || !dip_aligned16(y) || !opt_aligned16(mask_out))
+        return DIP_ERR_INVALID_ARG;
     if (w->wtype == DIP_W_INT4_G128) return DIP_ERR_UNSUPPORTED;
     if (!dims_ok(w->wtype, w->d_model, w->d_ff)) return DIP_ERR_INVALID_ARG;
+    if (!fits(ctx, w->d_model, w->d_ff, 1)) return DIP_ERR_WORKSPACE;
     if (!w->gate || !w->up || !w->down || !dip_aligned16(w->gate) || !dip_aligned16(w->up) || !dip_aligned16(w->down))
         return DIP_ERR_INVALID_ARG;
     if (prune_by != DIP_PRUNE_BY_GATE && prune_by != DIP_PRUNE_BY_UP) return DIP_ERR_INVALID_ARG;
@@ -493,9 +548,65 @@ dip_status dip_mlp_step_neuron_pruned(dip_ctx *ctx, const dip_neuron_weights *w,
 dip_status dip_residual_rmsnorm(dip_ctx *ctx, const float *x, const float *y,
                                 int batch, int d, float *x_next, void *stream)
 {
-    if (!ctx || !x || !y || !x_next) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx) || !x || !y || !x_next) return DIP_ERR_INVALID_ARG;
+    if (!dip_aligned16(x) || !dip_aligned16(y) || !dip_aligned16(x_next)) return DIP_ERR_INVALID_ARG;
     if (batch < 1 || batch > DIP_MAX_BATCH || d < 1 || d > DIP_MAX_D) return DIP_ERR_INVALID_ARG;
     return dip_launch_residual_rmsnorm(ctx, x, y, batch, d, x_next, (cudaStream_t)stream);
+}
+
+static dip_status stack_impl(dip_ctx *ctx, int n_layers, const dip_mlp_weights *layers,
+                             const float *x_in, int batch, int k_x, int k_h, float gamma,
+                             const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                             float *x_out, float *y_last, const dip_stack_probe *probe, void *stream)
+{
+    if (!ctx_ok(ctx) || n_layers < 1 || !layers || !x_in || !x_out) return DIP_ERR_INVALID_ARG;
+    if (!dip_aligned16(x_in) || !dip_aligned16(x_out) || !opt_aligned16(y_last)) return DIP_ERR_INVALID_ARG;
+    if (batch < 1 || batch > DIP_MAX_BATCH) return DIP_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!weights_ok(&layers[l])) return DIP_ERR_INVALID_ARG;
+        if (layers[l].d_model != layers[0].d_model || layers[l].d_ff != layers[0].d_ff) return DIP_ERR_INVALID_ARG;
+    }
+    const int d = layers[0].d_model, d_ff = layers[0].d_ff;
+    if (!fits(ctx, d, d_ff, batch)) return DIP_ERR_WORKSPACE;
+    if (probe && (!probe->x || !probe->mask_x || !probe->h || !probe->mask_h || !probe->y || !dip_aligned16(probe->x) ||
+                  !dip_aligned16(probe->mask_x) || !dip_aligned16(probe->h) || !dip_aligned16(probe->mask_h) ||
+                  !dip_aligned16(probe->y) || (d & 127) || (d_ff & 127)))
+        return DIP_ERR_INVALID_ARG;      // (per-layer slices of the arrays stay 16-byte aligned)
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t ring_words = (size_t)ctx->max_d / 32;
+    // x_0 = x_in; for l > 0 the chaining x_l = rmsnorm(x_{l-1} + y_{l-1}) runs inside layer l's
+    // first mask launch.  x and y ping-pong between two workspace buffers each.
+    const float *x_prev = x_in;
+    const float *y_prev = nullptr;
+    const bool ca = cache_gu || cache_d;
+    if (probe) DIP_CUDA_TRY(ctx, cudaMemcpyAsync(probe->x, x_in, sizeof(float) * (size_t)batch * d, cudaMemcpyDeviceToDevice, s));
+    for (int l = 0; l < n_layers; ++l) {
+        float *y = (l == n_layers - 1 && y_last) ? y_last : ((l & 1) ? ctx->y2 : ctx->y);
+        float *x_l = (l & 1) ? ctx->xb : ctx->xa;
+        // with caches each layer's masks get their own slot: the updates that read them run
+        // beside later layers
+        const int slot = ca ? l % DIP_RING_LAYERS : 0;
+        uint32_t *slot_x = batch == 1 ? ctx->mask_ring + (size_t)slot * ring_words : ctx->mask;
+        uint32_t *slot_h = batch == 1 ? ctx->mask_ring + (size_t)(DIP_RING_LAYERS + slot) * ring_words : ctx->mask_h;
+        dip_step_outputs po = {};
+        if (probe) {
+            y = probe->y + (size_t)l * batch * d;
+            x_l = probe->x + (size_t)l * batch * d;
+            po.mask_x = probe->mask_x + (size_t)l * batch * (d / 32);
+            po.mask_h = probe->mask_h + (size_t)l * batch * (d_ff / 32);
+            po.h = probe->h + (size_t)l * batch * d_ff;
+        }
+        dip_status st = step_impl(ctx, &layers[l], x_prev, y_prev, y_prev ? x_l : nullptr, batch, k_x, k_h, gamma,
+                                  cache_gu ? &cache_gu[l] : nullptr, cache_d ? &cache_d[l] : nullptr,
+                                  y, probe ? &po : nullptr, slot_x, slot_h, true, stream);
+        if (st != DIP_OK) return st;
+        if (ca && slot == DIP_RING_LAYERS - 1 && (st = join_cache_updates(ctx, s)) != DIP_OK) return st;
+        if (y_prev) x_prev = x_l;
+        y_prev = y;
+    }
+    dip_status st = dip_residual_rmsnorm(ctx, x_prev, y_prev, batch, d, x_out, stream);
+    if (st != DIP_OK) return st;
+    return join_cache_updates(ctx, s);
 }
 
 dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *layers,
@@ -503,37 +614,18 @@ dip_status dip_stack_step(dip_ctx *ctx, int n_layers, const dip_mlp_weights *lay
                           const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
                           float *x_out, float *y_last, void *stream)
 {
-    if (!ctx || n_layers < 1 || !layers || !x_in || !x_out) return DIP_ERR_INVALID_ARG;
-    if (batch < 1 || batch > DIP_MAX_BATCH) return DIP_ERR_INVALID_ARG;
-    for (int l = 0; l < n_layers; ++l) {
-        if (!weights_ok(&layers[l])) return DIP_ERR_INVALID_ARG;
-        if (layers[l].d_model != layers[0].d_model || layers[l].d_ff != layers[0].d_ff) return DIP_ERR_INVALID_ARG;
-    }
-    const int d = layers[0].d_model;
-    // x_0 = x_in; for l > 0 the chaining x_l = rmsnorm(x_{l-1} + y_{l-1}) runs inside layer l's
-    // first mask launch.  x and y ping-pong between two workspace buffers each.
-    const float *x_prev = x_in;
-    const float *y_prev = nullptr;
-    const bool ca = cache_gu || cache_d;
-    for (int l = 0; l < n_layers; ++l) {
-        float *y = (l == n_layers - 1 && y_last) ? y_last : ((l & 1) ? ctx->y2 : ctx->y);
-        float *x_l = (l & 1) ? ctx->xb : ctx->xa;
-        // with caches each layer's masks get their own slot: the updates that read them run
-        // beside later layers
-        const int slot = ca ? l % DIP_RING_LAYERS : 0;
-        uint32_t *slot_x = batch == 1 ? ctx->mask_ring + (size_t)slot * (DIP_MAX_D / 32) : ctx->mask;
-        uint32_t *slot_h = batch == 1 ? ctx->mask_ring + (size_t)(DIP_RING_LAYERS + slot) * (DIP_MAX_D / 32) : ctx->mask_h;
-        dip_status st = step_impl(ctx, &layers[l], x_prev, y_prev, y_prev ? x_l : nullptr, batch, k_x, k_h, gamma,
-                                  cache_gu ? &cache_gu[l] : nullptr, cache_d ? &cache_d[l] : nullptr,
-                                  y, nullptr, slot_x, slot_h, true, stream);
-        if (st != DIP_OK) return st;
-        if (ca && slot == DIP_RING_LAYERS - 1 && (st = join_cache_updates(ctx, (cudaStream_t)stream)) != DIP_OK) return st;
-        if (y_prev) x_prev = x_l;
-        y_prev = y;
-    }
-    dip_status st = dip_residual_rmsnorm(ctx, x_prev, y_prev, batch, d, x_out, stream);
-    if (st != DIP_OK) return st;
-    return join_cache_updates(ctx, (cudaStream_t)stream);
+    return stack_impl(ctx, n_layers, layers, x_in, batch, k_x, k_h, gamma, cache_gu, cache_d, x_out, y_last, nullptr,
+                      stream);
+}
+
+dip_status dip_stack_step_probed(dip_ctx *ctx, int n_layers, const dip_mlp_weights *layers,
+                                 const float *x_in, int batch, int k_x, int k_h, float gamma,
+                                 const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                                 float *x_out, const dip_stack_probe *probe, void *stream)
+{
+    if (!probe) return DIP_ERR_INVALID_ARG;
+    return stack_impl(ctx, n_layers, layers, x_in, batch, k_x, k_h, gamma, cache_gu, cache_d, x_out, nullptr, probe,
+                      stream);
 }
 
 // ---- device-side timeline (diagnostics) ----
@@ -553,7 +645,7 @@ static dip_status trace_clear(dip_ctx *ctx)
 
 dip_status dip_trace_begin(dip_ctx *ctx)
 {
-    if (!ctx) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx)) return DIP_ERR_INVALID_ARG;
     ctx->trace_on = 1;
     ctx->trace_next = 0;
     return trace_clear(ctx);
@@ -561,13 +653,13 @@ dip_status dip_trace_begin(dip_ctx *ctx)
 
 dip_status dip_trace_reset(dip_ctx *ctx)
 {
-    if (!ctx) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx)) return DIP_ERR_INVALID_ARG;
     return trace_clear(ctx);
 }
 
 dip_status dip_trace_read(dip_ctx *ctx, dip_trace_record *out, int max_records, int *n_out)
 {
-    if (!ctx || !out || !n_out || max_records < 0) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx) || !out || !n_out || max_records < 0) return DIP_ERR_INVALID_ARG;
     static unsigned long long host[DIP_TRACE_SLOTS * DIP_TRACE_WORDS];
     DIP_CUDA_TRY(ctx, cudaDeviceSynchronize());
     DIP_CUDA_TRY(ctx, cudaMemcpy(host, ctx->trace, sizeof(host), cudaMemcpyDeviceToHost));
@@ -588,7 +680,7 @@ dip_status dip_trace_read(dip_ctx *ctx, dip_trace_record *out, int max_records, 
 
 dip_status dip_trace_end(dip_ctx *ctx)
 {
-    if (!ctx) return DIP_ERR_INVALID_ARG;
+    if (!ctx_ok(ctx)) return DIP_ERR_INVALID_ARG;
     ctx->trace_on = 0;
     return DIP_OK;
 }

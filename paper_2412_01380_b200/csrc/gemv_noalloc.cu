@@ -68,7 +68,7 @@ template <> __device__ __forceinline__ void na_decode<DIP_W_BF16>(uint4 a, uint4
 // order, parts in part order by the last CTA to arrive at the slab.
 template <int WT>
 __global__ void __launch_bounds__(NA_THREADS)
-down_noalloc_kernel(const char *__restrict__ W, size_t row_bytes, int d_model,
+down_noalloc_kernel(const char *__restrict__ W, size_t row_bytes, int d_model, int d_ff,
                     const float *__restrict__ h, const int32_t *__restrict__ kept_idx, int n_kept,
                     float *__restrict__ y, NaScratch *scratch)
 {
@@ -95,7 +95,9 @@ down_noalloc_kernel(const char *__restrict__ W, size_t row_bytes, int d_model,
         float my_v = 0.f;
         if (c0 + lane < n_mine) {
             my_idx = kept_idx[r_begin + warp + (c0 + lane) * NA_WARPS];
-            my_v = h[my_idx];
+            // an entry outside [0, d_ff) names no column: it contributes nothing and reads nothing
+            if ((unsigned)my_idx >= (unsigned)d_ff) my_idx = 0;
+            else my_v = h[my_idx];
         }
         const int n_here = min(32, n_mine - c0);
         for (int j0 = 0; j0 < n_here; j0 += NA_UNROLL) {
@@ -213,9 +215,9 @@ extern "C" dip_status dip_sparse_gemv_down_noalloc(const dip_mlp_weights *w, con
     const size_t row_bytes = (size_t)w->d_model * (w->wtype == DIP_W_F32 ? 4 : 2);
     if (w->wtype == DIP_W_F32)
         down_noalloc_kernel<DIP_W_F32><<<grid, NA_THREADS, 0, s>>>((const char *)w->down, row_bytes, w->d_model,
-                                                                    h, kept_idx, n_kept, y, nd->scratch);
+                                                                    w->d_ff, h, kept_idx, n_kept, y, nd->scratch);
     else
         down_noalloc_kernel<DIP_W_BF16><<<grid, NA_THREADS, 0, s>>>((const char *)w->down, row_bytes, w->d_model,
-                                                                     h, kept_idx, n_kept, y, nd->scratch);
+                                                                     w->d_ff, h, kept_idx, n_kept, y, nd->scratch);
     return cudaGetLastError() == cudaSuccess ? DIP_OK : DIP_ERR_CUDA;
 }

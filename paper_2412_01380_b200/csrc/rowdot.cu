@@ -125,20 +125,12 @@ dip_status dip_launch_rowdot(dip_ctx *ctx, int wtype, const void *W, int d_model
     if (blocks > ctx->sm_count) blocks = ctx->sm_count;
     if (blocks < 1) blocks = 1;
     if (wtype == DIP_W_F32) {
-        static bool set = false;
-        if (!set) {
-            DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(rowdot_kernel<DIP_W_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)(sizeof(float) * DIP_MAX_D)));
-            set = true;
-        }
+        static dip_per_device_once once;
+        DIP_CUDA_TRY(ctx, dip_raise_smem_limit(once, ctx->device, rowdot_kernel<DIP_W_F32>, sizeof(float) * DIP_MAX_D));
         DIP_CUDA_TRY(ctx, dip_launch_pdl(rowdot_kernel<DIP_W_F32>, dim3(blocks), dim3(RD_THREADS), smem, stream, p));
     } else {
-        static bool set = false;
-        if (!set) {
-            DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(rowdot_kernel<DIP_W_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)(sizeof(float) * DIP_MAX_D)));
-            set = true;
-        }
+        static dip_per_device_once once;
+        DIP_CUDA_TRY(ctx, dip_raise_smem_limit(once, ctx->device, rowdot_kernel<DIP_W_BF16>, sizeof(float) * DIP_MAX_D));
         DIP_CUDA_TRY(ctx, dip_launch_pdl(rowdot_kernel<DIP_W_BF16>, dim3(blocks), dim3(RD_THREADS), smem, stream, p));
     }
     return DIP_OK;

@@ -100,7 +100,7 @@ def check_step(dip, ctx, lw, w, x, k_x, k_h, gamma, ref_gu, ref_d, g_gu, g_d, ti
     assert np.array_equal(idx_x.cpu().numpy(), idx_x_ref)
     gg = oracle.masked_matvec(Wg, x, m_x)
     uu = oracle.masked_matvec(Wu, x, m_x)
-    h_ref = uu * gg / (1.0 + np.exp(-gg))
+    h_ref = oracle.glu(gg, uu)
     h_gpu = h.cpu().numpy()
     assert rel_err(h_gpu, h_ref) <= REL_TOL
     # second half, teacher-forced on the GPU's h

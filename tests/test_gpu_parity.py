@@ -202,7 +202,7 @@ def test_sparse_gemvs_match_oracle(dip, ctx, wtype, d_model, d_ff, rho):
     m_x, idx_x = oracle.dip_ca_mask(x, k_x)
     g = oracle.masked_matvec(Wg, x, m_x)
     u = oracle.masked_matvec(Wu, x, m_x)
-    h_ref = u * g / (1.0 + np.exp(-g))
+    h_ref = oracle.glu(g, u)
     h = torch.full((d_ff,), 7.0, device="cuda")
     dip.dip_sparse_gemv_gate_up(ctx, w, torch.from_numpy(x).cuda(), torch.from_numpy(idx_x).cuda(), k_x, None, h)
     torch.cuda.synchronize()
@@ -266,11 +266,10 @@ def test_mlp_step_matches_oracle(dip, ctx, wtype, d_model, d_ff, rho, beta):
     (di.W_BF16, 512, 1536, 1.0, 0.5),       # keep ratio 1: every column kept
     (di.W_BF16, 256, 32, 0.25, 0.5),        # a single mask word
 ])
-def test_mlp_step_ranking_h_from_the_gemv_keys(dip, wtype, d_model, d_ff, rho, beta, monkeypatch):
+def test_mlp_step_ranking_h_from_the_gemv_keys(dip, wtype, d_model, d_ff, rho, beta):
     """A context that ranks h from the 16-bit keys left by the gate/up product at every size
     (by default only wide layers do): same bit-exact masks and cache state."""
-    monkeypatch.setenv("DIP_COARSE_MIN_D", "0")
-    c = dip.Context(0)
+    c = dip.Context(0, coarse_min_d=-1)
     try:
         lw = _layer(31 + d_ff, d_model, d_ff, wtype)
         w = upload_layer(dip, c, lw)
@@ -423,7 +422,7 @@ def test_batched_step_matches_per_token_oracle(dip, ctx, batch):
         assert np.array_equal(mx[b], m_x)
         gg = oracle.masked_matvec(Wg, x[b], m_x)
         uu = oracle.masked_matvec(Wu, x[b], m_x)
-        assert rel_err(hg[b], uu * gg / (1 + np.exp(-gg))) <= REL_TOL
+        assert rel_err(hg[b], oracle.glu(gg, uu)) <= REL_TOL
         m_h, _ = oracle.dip_ca_mask(hg[b], k_h)
         assert np.array_equal(mh[b], m_h)
         assert rel_err(yg[b], oracle.masked_matvec(Wd, hg[b], m_h)) <= REL_TOL
@@ -460,7 +459,7 @@ def test_full_size_batched_layer(dip, ctx):
     for b in (0, 7, 15):
         gg = oracle.masked_matvec(Wg, x[b], mx[b])
         uu = oracle.masked_matvec(Wu, x[b], mx[b])
-        assert rel_err(hg[b], uu * gg / (1 + np.exp(-gg))) <= REL_TOL
+        assert rel_err(hg[b], oracle.glu(gg, uu)) <= REL_TOL
         assert rel_err(yg[b], oracle.masked_matvec(Wd, hg[b], mh[b])) <= REL_TOL
     assert counts.cpu().tolist() == [oracle.mask_union(mx)[1], oracle.mask_union(mh)[1]]
 

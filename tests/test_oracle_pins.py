@@ -66,6 +66,31 @@ def test_silu_closed_forms():
     assert min(vals) == pytest.approx(-0.2784645427610738, abs=1e-7)
 
 
+def test_glu_elementwise_pins():
+    """Eq. 2 for given pre-activations: u * silu(g).  Closed forms, the tanh form of the sigmoid,
+    oddness in u, and the dense oracle's GLU on the same pre-activations."""
+    g = np.array([0.0, 1.0, -1.0, 40.0, -40.0, 2.5], dtype=np.float64)
+    u = np.array([3.0, 2.0, 2.0, -1.5, 7.0, 0.0], dtype=np.float64)
+    h = oracle.glu(g, u)
+    assert h[0] == 0.0 and h[5] == 0.0
+    assert h[1] == pytest.approx(2.0 * 0.7310585786300049, rel=1e-15)
+    assert h[1] - h[2] == pytest.approx(2.0 * 1.0, rel=1e-15)       # silu(z) - silu(-z) = z, times u
+    assert h[3] == pytest.approx(-1.5 * 40.0, rel=1e-15)
+    assert h[4] == pytest.approx(7.0 * -40.0 * math.exp(-40.0), rel=1e-12)
+    rng = np.random.default_rng(8)
+    g, u = rng.standard_normal(200) * 3, rng.standard_normal(200)
+    np.testing.assert_allclose(oracle.glu(g, u), u * g * 0.5 * (1.0 + np.tanh(0.5 * g)), rtol=1e-11, atol=1e-15)
+    np.testing.assert_array_equal(oracle.glu(g, -u), -oracle.glu(g, u))
+    assert not np.allclose(oracle.glu(g, u), oracle.glu(u, g))           # the gate is the activated branch
+    lw = _rand_layer(21, 64, 96)
+    Wg, Wu, Wd = _oracle_mats(lw)
+    x = di.heavy_tail_vector(22, 64)
+    ones = np.ones(64, dtype=np.uint8)
+    glu_dense, _ = oracle.dense_mlp(Wg, Wu, Wd, x)
+    np.testing.assert_array_equal(oracle.glu(oracle.masked_matvec(Wg, x, ones), oracle.masked_matvec(Wu, x, ones)),
+                                  glu_dense)
+
+
 # --------------------------------------------------------------------------
 # stored formats
 # --------------------------------------------------------------------------
