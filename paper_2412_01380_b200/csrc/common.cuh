@@ -44,9 +44,6 @@ struct dip_ctx {
     uint32_t *mask_ring; // [2][DIP_RING_LAYERS][max_d/32] per-layer mask slots of the stack runner
     uint32_t *mask_tmp;  // [max_d/32] list-based GEMV entry points
     uint16_t *coarse;    // [max_d] top 16 bits of the rank keys of h, left by the gate/up GEMV
-    uint32_t *certain;   // [2][max_d/32] early part of the masks of x and of h (see dip_handoff)
-    unsigned int *ready; // [2][2] hand-over flags of the masks of x and of h
-    int handoff;         // single-token steps hand their masks over early
     int coarse_min_d;    // smallest d_ff for which the step ranks h from those
     int *status;         // sticky device status word (0 = fine)
     // the cache updates run beside the GEMVs: one side stream per cache kind
@@ -83,20 +80,6 @@ static inline unsigned long long *dip_trace_slot(dip_ctx *ctx, int kind)
         }                                                                              \
     } while (0)
 
-// Early hand-over of a mask from the select kernel to the product kernel that follows it in the
-// stream (both are resident at the same time under programmatic dependent launch; the select is
-// always launched first, so the product's wait below never holds up its producer).
-//   ready[0]: the "certain" part of the mask (every column whose rank key lies in a radix bin
-//             above the threshold's) is in `certain`, and the input vector is complete;
-//   ready[1]: the final mask is in the launch's mask buffer.
-// certain is a subset of the final mask, so the product can stream its rows at once and pick up
-// the few remaining rows (final AND NOT certain) at its end.  The flags are cleared by the next
-// select kernel of the other masked input, which starts only after this mask's product is done.
-struct dip_handoff {
-    unsigned int *ready;        // [2] flags of this masked input
-    uint32_t *certain;          // [words] the certain part of the mask
-    unsigned int *clear;        // [2] flags of the other masked input (select: zeroed at start), or nullptr
-};
 #ifdef __CUDACC__
 // Timeline stamps (nanoseconds of %globaltimer) taken by thread 0 of each CTA when tr != nullptr:
 // word 0 = earliest kernel entry, 1 = earliest return from the dependency wait, 2 = latest exit,
@@ -107,30 +90,6 @@ __device__ __forceinline__ unsigned long long dip_gtime()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ void dip_flag_release(unsigned int *flag, unsigned int v)
-{
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(v) : "memory");
-}
-__device__ __forceinline__ unsigned int dip_flag_acquire(const unsigned int *flag)
-{
-    unsigned int v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-    return v;
-}
-// Bounded spin until *flag != 0; false when limit_ns ran out.
-__device__ __forceinline__ bool dip_flag_wait(const unsigned int *flag, unsigned long long limit_ns)
-{
-    unsigned long long t0 = 0;
-    for (unsigned i = 0;; ++i) {
-        if (dip_flag_acquire(flag) != 0u) return true;
-        if ((i & 63u) == 63u) {
-            const unsigned long long now = dip_gtime();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > limit_ns) return false;
-        }
-    }
-}
-
 #define DIP_TRACE_MIN(tr, i) do { if ((tr) && threadIdx.x == 0) atomicMin(&(tr)[i], dip_gtime()); } while (0)
 #define DIP_TRACE_MAX(tr, i) do { if ((tr) && threadIdx.x == 0) atomicMax(&(tr)[i], dip_gtime()); } while (0)
 
@@ -186,10 +145,9 @@ static inline cudaError_t dip_raise_smem_limit(dip_per_device_once &once, int de
 // coarse != nullptr (one row, no xb, d % 32 == 0): the producer of xa has left the top 16 bits of
 // every column's rank key there (dip_gemv_keys), and the launch reads those instead of all of
 // xa and stamp.
-// ho != nullptr (one row): the launch hands its mask over early (see dip_handoff).
 dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d, int k,
                              float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream,
-                             const uint16_t *coarse = nullptr, const dip_handoff *ho = nullptr);
+                             const uint16_t *coarse = nullptr);
 
 // topk.cu: LRU cache update from (mask, state).
 // count != nullptr: LFU (use counters), else LRU.
@@ -231,14 +189,10 @@ struct dip_gemv_keys {
     float gamma;
     int written;             // out
 };
-// ho != nullptr: the mask comes from the select kernel launched just before on the same stream with
-// the same hand-over; ho_used (out) says whether this launch takes it (only the single-token
-// F32 / BF16 launch does; the caller asks with dip_gemv_takes_handoff before launching the select).
 dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                            const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
                            float *out, cudaStream_t stream, const dip_gemv_rows *rows = nullptr,
-                           dip_gemv_keys *keys = nullptr, const dip_handoff *ho = nullptr);
-bool dip_gemv_takes_handoff(const dip_ctx *ctx, const dip_mlp_weights *w, int batch);
+                           dip_gemv_keys *keys = nullptr);
 
 // gemv.cu: one tiny kernel whose bounded wait runs out (sets the status word to 1).
 dip_status dip_launch_bounded_wait_selftest(dip_ctx *ctx, unsigned long long limit_ns, unsigned long long *waited_ns,

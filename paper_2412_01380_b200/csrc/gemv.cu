@@ -61,11 +61,6 @@ struct GemvParams {
     uint16_t *key_coarse;
     const int32_t *key_stamp;
     float key_gamma;
-    // gemv_direct_kernel only: early hand-over of the mask by the select kernel launched just before
-    // (see dip_handoff): ho_ready != nullptr: wait for ho_ready[0], stream the rows of ho_certain,
-    // then, once ho_ready[1] is set, the rows of mask_bits that ho_certain lacks
-    const unsigned int *ho_ready;
-    const uint32_t *ho_certain;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -699,17 +694,10 @@ template <int NW> struct __align__(16) GemvDirectSmem {
     int wsum[GV_SCAN_THREADS / 32];
     int n_total;
     int last;
-    int fail;
     float red[NW][32 * 8];           // [warp][lane * E + e], E <= 8
     float sum[32 * 8];
 };
 
-// With an early hand-over the kernel does not wait for the select kernel to finish: it waits for
-// the flag that says the certain part of the mask is there, streams those rows exactly as it would
-// stream a whole mask, and appends the few rows that the finished mask adds: warp w of row part q
-// owns the mask words q + nparts * (w + NW * t) and takes the added rows of those words, in the
-// same batches as (and right behind) its last rows of the certain part.  The order of every sum is
-// a function of the two bit sets alone.
 template <int WT, int WHICH, int NW, int U>
 __global__ void __launch_bounds__(NW * 32, 1)
 gemv_direct_kernel(const GemvParams p)
@@ -727,21 +715,9 @@ gemv_direct_kernel(const GemvParams p)
     const int slab = blockIdx.x, part = blockIdx.y, nparts = gridDim.y;
     const size_t byte_off = (size_t)slab * GD_SEG + lane * 16;
     const bool lane_ok = byte_off < p.row_bytes;
-    const bool ho = p.ho_ready != nullptr;
-    bool failed = false;
-    if (ho) {
-        dip_launch_dependents();
-        if (tid == 0) s.fail = dip_flag_wait(p.ho_ready, p.wait_limit_ns) ? 0 : 1;
-        __syncthreads();
-        failed = s.fail != 0;
-        if (failed && tid == 0) atomicExch(p.status, 1);
-        DIP_TRACE_MIN(p.tr, 1);
-    } else {
-        dip_grid_dependency_wait();
-        DIP_TRACE_MIN(p.tr, 1);
-        dip_launch_dependents();
-    }
-    const uint32_t *first_bits = ho ? p.ho_certain : p.mask_bits;
+    dip_grid_dependency_wait();
+    DIP_TRACE_MIN(p.tr, 1);
+    dip_launch_dependents();
 
     // the stamp that the epilogue's rank key needs travels while the rows stream
     int key_stamp = 0;
@@ -755,7 +731,7 @@ gemv_direct_kernel(const GemvParams p)
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int w = 4 * tid + j;
-            if (w < p.mask_words && !failed) u[j] = __ldcg(first_bits + w);
+            if (w < p.mask_words) u[j] = p.mask_bits[w];
             if (w == p.mask_words - 1 && (p.d_in & 31)) u[j] &= (1u << (p.d_in & 31)) - 1u;
             c += __popc(u[j]);
         }
@@ -786,24 +762,15 @@ gemv_direct_kernel(const GemvParams p)
     const int n_total = s.n_total;
     const int r_begin = (int)(((long long)part * n_total) / nparts);
     const int r_end = (int)(((long long)(part + 1) * n_total) / nparts);
-    const int n_rounds = r_end > r_begin ? (r_end - r_begin + GV_MAX_ROWS - 1) / GV_MAX_ROWS : 1;
 
     float acc[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
     const char *base = p.W + byte_off;
-    // hand-over: this warp's walk over the mask words it owns, for the rows the finished mask adds
-    const int ext_step = nparts * NW;
-    int ext_next = ho && !failed ? part + nparts * warp : p.mask_words;   // next owned word to look at
-    int ext_word = 0;                                                       // word that ext_bits came from
-    uint32_t ext_bits = 0u;
-    bool ext_open = false;
 
-    for (int round = 0; round < n_rounds; ++round) {
-        const int round_begin = r_begin + round * GV_MAX_ROWS;
+    for (int round_begin = r_begin; round_begin < r_end; round_begin += GV_MAX_ROWS) {
         const int n_rows = min(r_end - round_begin, GV_MAX_ROWS);
-        const bool last_round = round == n_rounds - 1;
-        if (round) __syncthreads();
+        if (round_begin != r_begin) __syncthreads();
         // ---- 2. the round's rows in rank order ----
         {
             const int lo_rank = round_begin, hi_rank = round_begin + n_rows;
@@ -822,47 +789,20 @@ gemv_direct_kernel(const GemvParams p)
         __syncthreads();
         // ---- 3. stream: warp w takes rows w, w + NW, ...; U of them in flight per lane.  The
         //         first batch of loads goes out before the vector's values are fetched ----
-        for (int r0 = warp;; r0 += NW * U) {
+        for (int r0 = warp; r0 < n_rows; r0 += NW * U) {
             uint4 q[U];
             float xv[U];
-            bool any = false;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int r = r0 + u * NW;
-                int idx = -1;
-                if (r < n_rows) {
-                    idx = s.idx[r];
-                } else if (last_round && ext_next < p.mask_words + ext_step) {
-                    // past this warp's share of the certain rows: the rows that the finished mask adds
-                    if (!ext_open) {
-                        ext_open = true;
-                        if (!dip_flag_wait(p.ho_ready + 1, p.wait_limit_ns)) {
-                            if (lane == 0) atomicExch(p.status, 1);
-                            ext_next = p.mask_words;
-                        }
-                    }
-                    while (ext_bits == 0u && ext_next < p.mask_words) {
-                        ext_word = ext_next;
-                        ext_bits = __ldcg(p.mask_bits + ext_word) & ~s.words[ext_word];
-                        if (ext_word == p.mask_words - 1 && (p.d_in & 31)) ext_bits &= (1u << (p.d_in & 31)) - 1u;
-                        ext_next += ext_step;
-                    }
-                    if (ext_bits) {
-                        idx = ext_word * 32 + __ffs(ext_bits) - 1;
-                        ext_bits &= ext_bits - 1;
-                    } else {
-                        ext_next = p.mask_words + ext_step;           // walked through: nothing more to add
-                    }
-                }
                 q[u] = make_uint4(0u, 0u, 0u, 0u);
                 xv[u] = 0.f;
-                if (idx >= 0) {
-                    any = true;
+                if (r < n_rows) {
+                    const int idx = s.idx[r];
                     if (lane_ok) q[u] = __ldcs(reinterpret_cast<const uint4 *>(base + (size_t)idx * p.row_bytes));
-                    xv[u] = __ldcg(p.v + idx);
+                    xv[u] = __ldg(p.v + idx);
                 }
             }
-            if (!any) break;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 float w[E];
@@ -873,9 +813,6 @@ gemv_direct_kernel(const GemvParams p)
         }
     }
     DIP_TRACE_MAX(p.tr, 3);            // streaming done
-    // the select kernel has published its last flag, so this returns at once; it keeps "this kernel
-    // has finished" meaning "so has everything before it in the stream" for the kernels that follow
-    if (ho) dip_grid_dependency_wait();
 
     // ---- 4. the warps' sums, in warp order ----
 #pragma unroll
@@ -1143,18 +1080,10 @@ dip_status launch_bt(dip_ctx *ctx, GemvParams &p, int n_kept_max, int mode, cuda
 
 }  // namespace
 
-bool dip_gemv_takes_handoff(const dip_ctx *ctx, const dip_mlp_weights *w, int batch)
-{
-    return ctx->handoff && ctx->gemv_direct && batch == 1 && w->wtype != DIP_W_INT4_G128;
-}
-
 dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                            const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
-                           float *out, cudaStream_t stream, const dip_gemv_rows *rows, dip_gemv_keys *keys,
-                           const dip_handoff *ho)
+                           float *out, cudaStream_t stream, const dip_gemv_rows *rows, dip_gemv_keys *keys)
 {
-    // a mask that is handed over early has to be taken: its select kernel's successor is this launch
-    if (ho && (rows || !dip_gemv_takes_handoff(ctx, w, batch))) return DIP_ERR_INVALID_ARG;
     const int mode = rows ? rows->mode : 0;
     if (keys) keys->written = 0;
     if (mode && batch != 1) return DIP_ERR_UNSUPPORTED;
@@ -1177,8 +1106,7 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
     p.key_coarse = nullptr;
     p.key_stamp = nullptr;
     p.key_gamma = 1.0f;
-    p.ho_ready = nullptr;
-    p.ho_certain = nullptr;
+
     // all tokens of the batch in one launch (up to 16 sets of accumulators in registers): the
     // union of their rows is read once
     for (int b0 = 0; b0 < batch; b0 += 16) {
@@ -1194,10 +1122,6 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                 p.key_stamp = keys->stamp;
                 p.key_gamma = keys->gamma;
                 keys->written = 1;
-            }
-            if (ho) {
-                p.ho_ready = ho->ready;
-                p.ho_certain = ho->certain;
             }
             if (w->wtype == DIP_W_F32)
                 st = which == 0 ? launch_direct<DIP_W_F32, 0>(ctx, p, n_kept_max, stream)

@@ -319,35 +319,6 @@ __device__ void general_select(const uint32_t *keys, int d, int k, TkShared &s, 
     }
 }
 
-// Early hand-over (see dip_handoff).  Called by all threads of the CTA.
-// start: the flags of the other masked input are cleared (its product has finished: this kernel's
-// dependency wait has returned).
-__device__ __forceinline__ void handoff_start(const dip_handoff &ho)
-{
-    if (ho.clear && threadIdx.x == 0) {
-        ho.clear[0] = 0u;
-        ho.clear[1] = 0u;
-    }
-}
-// certain: s_maskw holds the columns that are kept whatever the refinement decides, and the
-// input vector has been written out.
-__device__ __forceinline__ void handoff_certain(const dip_handoff &ho, const unsigned int *s_maskw, int n_words)
-{
-    if (!ho.ready) return;
-    for (int w = threadIdx.x; w < n_words; w += TK_THREADS) ho.certain[w] = s_maskw[w];
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) dip_flag_release(ho.ready, 1u);
-}
-// final: the whole mask is in the launch's mask buffer.
-__device__ __forceinline__ void handoff_final(const dip_handoff &ho)
-{
-    if (!ho.ready) return;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) dip_flag_release(ho.ready + 1, 1u);
-}
-
 // ---------------------------------------------------------------------------------------
 // select_kernel: the mask of one row.
 //   CA == false: key = bits(|x|)                              (DIP, Eq. 7-8)
@@ -362,7 +333,7 @@ template <bool CA, bool NORM>
 __global__ void __launch_bounds__(TK_THREADS, 1)
 select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *__restrict__ x_out,
               int d, int k, float gamma, const int32_t *__restrict__ stamp,
-              uint32_t *__restrict__ mask_bits, unsigned long long *tr, const dip_handoff ho)
+              uint32_t *__restrict__ mask_bits, unsigned long long *tr)
 {
     DIP_TRACE_MIN(tr, 0);
     extern __shared__ uint32_t keys[];
@@ -387,7 +358,6 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
     dip_grid_dependency_wait();        // the inputs come from the previous kernel in the stream
     DIP_TRACE_MIN(tr, 1);
     dip_launch_dependents();
-    handoff_start(ho);
 
     float scale = 1.0f;
     if (NORM)
@@ -488,14 +458,11 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
         }
     }
     __syncthreads();
-    handoff_certain(ho, s_maskw, n_words);
     if (refine_candidates(keys, s, s_maskw, s_candw, n_words, krem1, mask_bits)) {
-        handoff_final(ho);
         DIP_TRACE_MAX(tr, 2);
         return;
     }
     general_select(keys, d, k, s, mask_bits);
-    handoff_final(ho);
     DIP_TRACE_MAX(tr, 2);
 }
 
@@ -521,8 +488,7 @@ __device__ __forceinline__ uint32_t rank_key(float v, int stamp, float gamma)
 template <bool CA>
 __global__ void __launch_bounds__(TK_THREADS, 1)
 select_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ coarse, int d, int k, float gamma,
-                     const int32_t *__restrict__ stamp, uint32_t *__restrict__ mask_bits, unsigned long long *tr,
-                     const dip_handoff ho)
+                     const int32_t *__restrict__ stamp, uint32_t *__restrict__ mask_bits, unsigned long long *tr)
 {
     DIP_TRACE_MIN(tr, 0);
     extern __shared__ uint32_t keys[];
@@ -539,7 +505,6 @@ select_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ c
     dip_grid_dependency_wait();
     DIP_TRACE_MIN(tr, 1);
     dip_launch_dependents();
-    handoff_start(ho);
 
     // coarse keys to registers (all loads in flight together)
     uint4 ck[TK_COARSE_ITERS];
@@ -598,7 +563,6 @@ select_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ c
         }
     }
     __syncthreads();
-    handoff_certain(ho, s_maskw, n_words);
     // the full rank keys of the candidates (a word's candidates belong to one thread, here and in
     // the refinement)
     for (int w = tid; w < n_words; w += TK_THREADS) {
@@ -623,7 +587,6 @@ select_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ c
         }
     }
     if (refine_candidates(keys, s, s_maskw, s_candw, n_words, krem1, mask_bits)) {
-        handoff_final(ho);
         DIP_TRACE_MAX(tr, 2);
         return;
     }
@@ -631,7 +594,6 @@ select_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ c
     for (int e = tid; e < d; e += TK_THREADS) keys[e] = rank_key<CA>(x[e], CA ? stamp[e] : 0, gamma);
     __syncthreads();
     general_select(keys, d, k, s, mask_bits);
-    handoff_final(ho);
     DIP_TRACE_MAX(tr, 2);
 }
 
@@ -826,35 +788,33 @@ residual_rmsnorm_kernel(const float *x, const float *y, int d, float *x_next)
 // ---------------------------------------------------------------------------------------
 dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d, int k,
                              float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream,
-                             const uint16_t *coarse, const dip_handoff *ho_in)
+                             const uint16_t *coarse)
 {
     const size_t smem = (size_t)((d + 3) & ~3) * sizeof(uint32_t);
     const dim3 grid(batch), block(TK_THREADS);
     unsigned long long *tr = dip_trace_slot(ctx, d <= 0 ? 0 : (stamp ? 2 : 1));
-    if (ho_in && batch != 1) return DIP_ERR_INVALID_ARG;
-    const dip_handoff ho = ho_in ? *ho_in : dip_handoff{nullptr, nullptr, nullptr};
     cudaError_t e;
     if (coarse) {
         if (xb || batch != 1 || (d & 31)) return DIP_ERR_INVALID_ARG;
         if (stamp)
             e = dip_launch_pdl(select_coarse_kernel<true>, grid, block, smem, stream, xa, coarse, d, k, gamma, stamp,
-                               mask_bits, tr, ho);
+                               mask_bits, tr);
         else
             e = dip_launch_pdl(select_coarse_kernel<false>, grid, block, smem, stream, xa, coarse, d, k, 1.0f,
-                               (const int32_t *)nullptr, mask_bits, tr, ho);
+                               (const int32_t *)nullptr, mask_bits, tr);
     } else if (xb) {
         if (stamp)
-            e = dip_launch_pdl(select_kernel<true, true>, grid, block, smem, stream, xa, xb, x_out, d, k, gamma, stamp, mask_bits, tr, ho);
+            e = dip_launch_pdl(select_kernel<true, true>, grid, block, smem, stream, xa, xb, x_out, d, k, gamma, stamp, mask_bits, tr);
         else
             e = dip_launch_pdl(select_kernel<false, true>, grid, block, smem, stream, xa, xb, x_out, d, k, 1.0f,
-                               (const int32_t *)nullptr, mask_bits, tr, ho);
+                               (const int32_t *)nullptr, mask_bits, tr);
     } else {
         if (stamp)
             e = dip_launch_pdl(select_kernel<true, false>, grid, block, smem, stream, xa, (const float *)nullptr,
-                               (float *)nullptr, d, k, gamma, stamp, mask_bits, tr, ho);
+                               (float *)nullptr, d, k, gamma, stamp, mask_bits, tr);
         else
             e = dip_launch_pdl(select_kernel<false, false>, grid, block, smem, stream, xa, (const float *)nullptr,
-                               (float *)nullptr, d, k, 1.0f, (const int32_t *)nullptr, mask_bits, tr, ho);
+                               (float *)nullptr, d, k, 1.0f, (const int32_t *)nullptr, mask_bits, tr);
     }
     DIP_CUDA_TRY(ctx, e);
     return DIP_OK;

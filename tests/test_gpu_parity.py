@@ -292,6 +292,30 @@ def test_mlp_step_ranking_h_from_the_gemv_keys(dip, wtype, d_model, d_ff, rho, b
         c.close()
 
 
+@pytest.mark.parametrize("d_model,d_ff", [(256, 4096), (1024, 8192)])
+def test_step_when_one_radix_bin_holds_every_rank_key(dip, ctx, d_model, d_ff):
+    """Inputs whose magnitudes all share their top 11 key bits: no column is certainly kept after the
+    first radix digit, so the products receive their whole masks at the very end of the early
+    hand-over (x within a factor 1.06; h_j = silu(a.x) (b.x) (1 + eps_j) with tiny eps_j)."""
+    rng = np.random.default_rng(d_ff)
+    a = (rng.standard_normal(d_model) * 0.05).astype(np.float32)
+    b = (rng.standard_normal(d_model) * 0.05).astype(np.float32)
+    eps = (1.0 + 0.03 * rng.random(d_ff)).astype(np.float32)
+    gate = np.ascontiguousarray(np.broadcast_to(a, (d_ff, d_model))).astype(np.float32)
+    up = (eps[:, None] * b[None, :]).astype(np.float32)
+    down = (rng.standard_normal((d_model, d_ff)) * 0.02).astype(np.float32)
+    lw = di.LayerWeights(di.W_F32, d_model, d_ff, gate, up, down, None, None, None)
+    w = upload_layer(dip, ctx, lw)
+    k_x, k_h = d_model // 2, d_ff // 4
+    ref_gu, ref_d = oracle.Cache(d_model, d_model // 2), oracle.Cache(d_ff, d_ff // 2)
+    g_gu, g_d = dip.CacheState(d_model, d_model // 2, "cuda"), dip.CacheState(d_ff, d_ff // 2, "cuda")
+    for t in range(4):
+        x = ((1.0 + 0.06 * rng.random(d_model)) * np.where(rng.random(d_model) < 0.5, -1, 1)).astype(np.float32)
+        # gamma = 1: resident or not, the keys stay in one bin
+        _check_step(dip, ctx, lw, w, x, k_x, k_h, 1.0, ref_gu, ref_d, g_gu, g_d)
+    assert ctx.device_status() == 0
+
+
 def test_full_size_phi3_medium_layer(dip, ctx):
     """One Phi-3-Medium-shaped block at the benchmark's keep ratios, all outputs checked."""
     wl = di.WORKLOADS["phi3_medium"]
