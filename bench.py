@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--policy", default="lru", choices=["lru", "lfu"], help="eviction policy of the column caches")
     ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging; not a valid bench)")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--min-timed-s", type=float, default=0.5,
+                    help="repeat the timed region of --steps steps until this much time has been timed (profiling runs: 0)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--report", default=None, metavar="FILE",
                     help="run every workload of the five configurations (fewer steps) and write a markdown table")
@@ -920,7 +922,8 @@ def main():
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ
                            else int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])) if rank == 0 else None
     head = run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, args.steps, args.warmup,
-                      sampler=sampler, dist=dist, policy=args.policy)
+                      sampler=sampler, dist=dist, policy=args.policy, min_timed_s=args.min_timed_s,
+                      min_repeats=3 if args.min_timed_s > 0 else 1)
 
     sweep = []
     if not args.no_sweep and world == 1 and w.name == "phi3_medium":

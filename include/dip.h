@@ -156,18 +156,23 @@ dip_status dip_trace_end(dip_ctx *ctx);
  * Weights.  The paper's unit of selection is a column W[:, i] of a matrix
  * W in R^{d_out x d_in} (Eq. 4, 7, 8), so the library stores each matrix
  * column-contiguous: row i of the packed array holds column i.  Gate and up
- * always share one mask (Eq. 7), so their columns are bundled: packed row i
- * holds W^g[:, i] and W^u[:, i] interleaved in chunks of C outputs (piece 2c =
- * gate outputs of chunk c, piece 2c+1 = up outputs of chunk c), C = 4 for F32
- * and 8 for BF16 (16-byte pieces), C = 16 for INT4 (8-byte pieces).
+ * always share one mask (Eq. 7), so their columns are bundled in one packed row.
  *
- *   gate_up        [d_model][2 * d_ff] elements, interleaved as above
+ *   gate_up        [d_model][2 * d_ff] elements
  *   down           [d_ff][d_model]     elements
- *   INT4 codes     two per byte, element e of a row in bits 4*(e&1).. of byte e>>1;
- *                  value = (code - 8) * scale
- *   gate_up_scales [d_model/128][2 * d_ff] binary16, element for element like a
- *                  gate_up row (16 gate scales, 16 up scales, ...)
- *   down_scales    [d_ff/128][d_model] binary16
+ * F32 / BF16: a gate_up row interleaves gate and up in chunks of C outputs (piece
+ * 2c = gate outputs of chunk c, piece 2c+1 = up outputs of chunk c), C = 4 for
+ * F32 and 8 for BF16 (16-byte pieces); a down row is the column as it is.
+ * INT4: value = (code - 8) * scale.  A packed row is a sequence of chunks of 128
+ * codes = 64 bytes = 16 little-endian 32-bit words.  Local element e of a chunk is
+ * nibble (e >> 4) of word (e & 15) (nibble n = bits 4n .. 4n+3), and the words are
+ * stored in the order 0, 8, 1, 9, ..., 7, 15.  Chunk c of a down row holds outputs
+ * 128 c + e; chunk c of a gate_up row holds gate output 64 c + e for e < 64 and up
+ * output 64 c + (e - 64) for e >= 64.  (In this order the eight bytes at offset 8 g
+ * of a chunk are one thread's operand share of eight 16 x 16 tensor-core tiles.)
+ *   gate_up_scales [d_model/128][2 * d_ff] binary16, chunk for chunk like a
+ *                  gate_up row, local element e at position (e & 15) * 8 + (e >> 4)
+ *   down_scales    [d_ff/128][d_model] binary16, likewise
  *
  * Requirements: d_model % 32 == 0, d_ff % 32 == 0 (all formats); INT4 also
  * needs d_model % 128 == 0 and d_ff % 128 == 0.

@@ -23,45 +23,16 @@
 #include <cuda_fp16.h>
 
 #include "common.cuh"
+#include "gemv_common.cuh"
 
 namespace {
 
 constexpr int GV_CONSUMER_WARPS = 8;
 constexpr int GV_THREADS = (GV_CONSUMER_WARPS + 1) * 32;   // + one producer warp
 constexpr int GV_STAGES = 5;
-constexpr int GV_MAX_ROWS = 2048;                          // kept rows per round (index list in smem)
 // Rows per round for BT tokens: the tokens' values of a round's rows stay in shared memory
 // (BT x rows floats, at most 32 KB).
 template <int BT> struct GvRound { static constexpr int ROWS = BT <= 4 ? GV_MAX_ROWS : (BT == 8 ? 1024 : 512); };
-constexpr int GV_SCAN_THREADS = 256;                       // threads that scan the mask words
-
-struct GemvParams {
-    const char *W;             // packed rows
-    size_t row_bytes;          // bytes of one packed row
-    const uint16_t *scales;    // INT4: binary16 scales [d_in/128][row elements], laid out like a row
-    size_t scale_row_elems;    // INT4: elements of one scale row
-    const float *v;            // [batch][d_in]
-    int d_in;
-    const uint32_t *mask_bits; // [batch][mask_words]; rows read = OR over the batch
-    int mask_words;
-    float *out;                // [batch][d_out]
-    int d_out;
-    int batch;                 // tokens in this launch (<= BT)
-    float *partials;
-    unsigned int *tickets;
-    int *status;               // device status word (0 = fine)
-    unsigned long long wait_limit_ns;   // a wait on a copy's arrival gives up after this long
-    unsigned long long *tr;    // timeline slot or nullptr
-    const int32_t *loc;        // two-tier: packed row of column i is W + loc[i] * row_bytes (nullptr: row i)
-    int defer;                 // 1: leave the row parts in `partials` for combine_parts_kernel
-    int part_base;             // first part index of this launch inside `partials`
-    // gate/up, gemv_direct_kernel only: top 16 bits of the rank key of every h_j for the select
-    // that follows (nullptr: not wanted); the key is |h_j| * (key_stamp[j] >= 0 ? 1 : key_gamma),
-    // or |h_j| without stamps
-    uint16_t *key_coarse;
-    const int32_t *key_stamp;
-    float key_gamma;
-};
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -102,13 +73,10 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ float silu_f32(float g) { return g / (1.0f + expf(-g)); }
-
 template <int WT> struct WTraits;
 // E = weights in a lane's 16 bytes; C = gate/up interleave chunk of the bundled rows (weights)
 template <> struct WTraits<DIP_W_F32>       { static constexpr int E = 4;  static constexpr int C = 4; };
 template <> struct WTraits<DIP_W_BF16>      { static constexpr int E = 8;  static constexpr int C = 8; };
-template <> struct WTraits<DIP_W_INT4_G128> { static constexpr int E = 32; static constexpr int C = 16; };
 
 template <int WT> __device__ __forceinline__ void decode16(const uint4 &r, float (&w)[WTraits<WT>::E]);
 template <> __device__ __forceinline__ void decode16<DIP_W_F32>(const uint4 &r, float (&w)[4])
@@ -127,22 +95,7 @@ template <> __device__ __forceinline__ void decode16<DIP_W_BF16>(const uint4 &r,
     }
 }
 
-// Eight 4-bit codes of one word as (code - 8) in binary32: OR-ing a code into the mantissa of
-// 2^23 gives 8388608 + code exactly; subtracting 8388616 leaves code - 8.
-__device__ __forceinline__ void decode_int4_word(uint32_t w, float *out)
-{
-#pragma unroll
-    for (int n = 0; n < 8; ++n)
-        out[n] = __uint_as_float(0x4b000000u | ((w >> (4 * n)) & 15u)) - 8388616.0f;
-}
-
-__device__ __forceinline__ float half_bits_to_float(uint16_t h)
-{
-    return __half2float(__ushort_as_half(h));
-}
-
 constexpr int GV_STAGE_BYTES = 32768;
-constexpr int GV_SCALE_STAGE_BYTES = 32768;                // INT4: shared memory for staged scale rows
 
 static_assert(DIP_MAX_D <= 32768, "the row lists in shared memory are 16-bit");
 template <int SEG> struct __align__(16) GemvSmem {
@@ -185,10 +138,6 @@ gemv_kernel(const GemvParams p)
     // tensor-core path: the same bytes hold the values as bfloat16 pairs, [BT][XS] each
     __nv_bfloat16 *s_xh = reinterpret_cast<__nv_bfloat16 *>(s_v);
     __nv_bfloat16 *s_xl = s_xh + BT * XS;
-    // INT4: the scale rows of the round's groups for this slab, staged once per round
-    uint16_t *s_sc = reinterpret_cast<uint16_t *>(smem_raw + sizeof(GemvSmem<SEG>) + sizeof(float) * BT * (ROWS + 8));
-    constexpr int SC_GROUPS = GV_SCALE_STAGE_BYTES / (SLAB * 2);   // groups that fit
-    int sc_first = 0, sc_count = 0;                                  // staged groups (uniform over the CTA)
 
     DIP_TRACE_MIN(p.tr, 0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -269,13 +218,6 @@ gemv_kernel(const GemvParams p)
     for (int b = 0; b < BT; ++b)
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[b][e] = 0.f;
-    // INT4 only: sums of the current scale group, its scales, and which group that is
-    float accg[WT == DIP_W_INT4_G128 ? E : 1], sc[WT == DIP_W_INT4_G128 ? E : 1];
-    int cur_group = -1;
-    if (WT == DIP_W_INT4_G128) {
-#pragma unroll
-        for (int e = 0; e < (WT == DIP_W_INT4_G128 ? E : 1); ++e) accg[e] = sc[e] = 0.f;
-    }
     bool failed = false;
     int it_base = 0;                                          // stages issued in earlier rounds
 
@@ -381,19 +323,6 @@ gemv_kernel(const GemvParams p)
                     s_xl[b * XS + r] = __float2bfloat16_rn(0.f);
                 }
             }
-            if constexpr (WT == DIP_W_INT4_G128) {
-                // rows are ascending, so the round touches the groups first .. last; stage their
-                // scale segments if they fit (otherwise the consumers read them from global memory)
-                sc_first = s.idx[0] >> 7;
-                const int ng = (s.idx[n_rows - 1] >> 7) - sc_first + 1;
-                sc_count = ng <= SC_GROUPS ? ng : 0;
-                for (int t = tid; t < sc_count * (SLAB / 8); t += GV_CONSUMER_WARPS * 32) {
-                    const int g = t / (SLAB / 8), o = (t % (SLAB / 8)) * 8;
-                    if ((size_t)slab * SLAB + o < p.scale_row_elems)
-                        *reinterpret_cast<uint4 *>(s_sc + g * SLAB + o) = __ldg(reinterpret_cast<const uint4 *>(
-                            p.scales + (size_t)(sc_first + g) * p.scale_row_elems + (size_t)slab * SLAB + o));
-                }
-            }
             asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
 
             for (int i = 0; i < n_stages; ++i) {
@@ -453,50 +382,7 @@ gemv_kernel(const GemvParams p)
                         }
                     }
                 } else if (lane_ok) {
-                    if constexpr (WT == DIP_W_INT4_G128) {
-                        // W = (code - 8) * scale[group of 128 rows]: sum (code - 8) * v within a
-                        // group, multiply by the group's scales when the group changes
-                        for (int rr = 0; rr < R / RG; ++rr) {
-                            const int r = rr * RG + rg;
-                            if (r >= rows_here) break;
-                            const int g = s.idx[i * R + r] >> 7;
-                            if (g != cur_group) {
-                                if (cur_group >= 0) {
-#pragma unroll
-                                    for (int e = 0; e < E; ++e) {
-                                        acc[0][e] = fmaf(sc[e], accg[e], acc[0][e]);
-                                        accg[e] = 0.f;
-                                    }
-                                }
-                                const bool staged = g - sc_first < sc_count;
-                                const uint4 *sp = staged
-                                    ? reinterpret_cast<const uint4 *>(s_sc + (g - sc_first) * SLAB + (cw * 32 + lane) * E)
-                                    : reinterpret_cast<const uint4 *>(p.scales + (size_t)g * p.scale_row_elems +
-                                                                      (size_t)slab * SLAB + (cw * 32 + lane) * E);
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    const uint4 sv = sp[q];
-                                    const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
-#pragma unroll
-                                    for (int t = 0; t < 4; ++t) {
-                                        sc[q * 8 + 2 * t] = half_bits_to_float((uint16_t)(sw[t] & 0xffffu));
-                                        sc[q * 8 + 2 * t + 1] = half_bits_to_float((uint16_t)(sw[t] >> 16));
-                                    }
-                                }
-                                cur_group = g;
-                            }
-                            const uint4 raw = *reinterpret_cast<const uint4 *>(&s.ring[st][r * RS + byte_off]);
-                            const float xv = s_v[i * R + r];
-                            const uint32_t cwd[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                float w8[8];
-                                decode_int4_word(cwd[q], w8);
-#pragma unroll
-                                for (int n = 0; n < 8; ++n) accg[q * 8 + n] = fmaf(w8[n], xv, accg[q * 8 + n]);
-                            }
-                        }
-                    } else {
+                    {
 #pragma unroll
                         for (int rr = 0; rr < R / RG; ++rr) {
                             const int r = rr * RG + rg;
@@ -535,12 +421,6 @@ gemv_kernel(const GemvParams p)
     }
 
     DIP_TRACE_MAX(p.tr, 3);            // streaming done
-    if constexpr (WT == DIP_W_INT4_G128) {
-        if (cur_group >= 0) {
-#pragma unroll
-            for (int e = 0; e < E; ++e) acc[0][e] = fmaf(sc[e], accg[e], acc[0][e]);
-        }
-    }
     // ---- 5. combine the row groups through the (now idle) ring, in group order ----
     __syncthreads();
     if (s.abort) {
@@ -1003,6 +883,33 @@ combine_parts_kernel(const float *__restrict__ partials, int nparts, int n_slabs
     }
 }
 
+}  // namespace
+
+dip_status dip_launch_combine_parts(dip_ctx *ctx, int which, int total_parts, int n_slabs, int bt, int slab_elems, int c,
+                                    int batch, int d_out, float *out, cudaStream_t stream)
+{
+    const long long groups = (long long)n_slabs * batch * ((which == 0 ? slab_elems / 2 : slab_elems) / 4);
+    const float *partials = ctx->partials;
+    // eight lanes per group of outputs pay when there are many parts
+    const bool wide = total_parts >= 16;
+    const int blocks = (int)(((wide ? groups * 8 : groups) + 255) / 256);
+    cudaError_t e;
+    if (which == 0)
+        e = wide ? dip_launch_pdl(combine_parts_kernel<0, 8>, dim3(blocks), dim3(256), 0, stream, partials, total_parts,
+                                  n_slabs, bt, slab_elems, c, batch, d_out, out)
+                 : dip_launch_pdl(combine_parts_kernel<0, 1>, dim3(blocks), dim3(256), 0, stream, partials, total_parts,
+                                  n_slabs, bt, slab_elems, c, batch, d_out, out);
+    else
+        e = wide ? dip_launch_pdl(combine_parts_kernel<1, 8>, dim3(blocks), dim3(256), 0, stream, partials, total_parts,
+                                  n_slabs, bt, slab_elems, c, batch, d_out, out)
+                 : dip_launch_pdl(combine_parts_kernel<1, 1>, dim3(blocks), dim3(256), 0, stream, partials, total_parts,
+                                  n_slabs, bt, slab_elems, c, batch, d_out, out);
+    DIP_CUDA_TRY(ctx, e);
+    return DIP_OK;
+}
+
+namespace {
+
 template <int WT, int WHICH, int BT, int SEG>
 dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, int mode, cudaStream_t stream)
 {
@@ -1013,26 +920,14 @@ dip_status launch_seg(dip_ctx *ctx, GemvParams &p, int n_slabs, int nparts, int 
     if ((nparts > 1 || mode) && (size_t)total_parts * per_part > ctx->partials_floats) return DIP_ERR_WORKSPACE;
     p.defer = mode != 0;
     p.part_base = mode == 2 ? nparts : 0;
-    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * (GvRound<BT>::ROWS + 8) * sizeof(float) +
-                        (WT == DIP_W_INT4_G128 ? GV_SCALE_STAGE_BYTES : 0);
+    const size_t smem = sizeof(GemvSmem<SEG>) + (size_t)BT * (GvRound<BT>::ROWS + 8) * sizeof(float);
     static dip_per_device_once once;   // per instantiation
     DIP_CUDA_TRY(ctx, dip_raise_smem_limit(once, ctx->device, gemv_kernel<WT, WHICH, BT, SEG>, smem));
     dim3 grid(n_slabs, nparts);
     DIP_CUDA_TRY(ctx, dip_launch_pdl(gemv_kernel<WT, WHICH, BT, SEG>, grid, dim3(GV_THREADS), smem, stream, p));
-    if ((BT >= 8 && nparts > 1 && !mode) || mode == 2) {
-        const long long groups = (long long)n_slabs * p.batch * ((WHICH == 0 ? SLAB / 2 : SLAB) / 4);
-        if (total_parts >= 16) {
-            const int blocks = (int)((groups * 8 + 255) / 256);
-            DIP_CUDA_TRY(ctx, dip_launch_pdl(combine_parts_kernel<WHICH, 8>, dim3(blocks), dim3(256), 0, stream,
-                                             (const float *)p.partials, total_parts, n_slabs, BT, SLAB, WTraits<WT>::C,
-                                             p.batch, p.d_out, p.out));
-        } else {
-            const int blocks = (int)((groups + 255) / 256);
-            DIP_CUDA_TRY(ctx, dip_launch_pdl(combine_parts_kernel<WHICH, 1>, dim3(blocks), dim3(256), 0, stream,
-                                             (const float *)p.partials, total_parts, n_slabs, BT, SLAB, WTraits<WT>::C,
-                                             p.batch, p.d_out, p.out));
-        }
-    }
+    if ((BT >= 8 && nparts > 1 && !mode) || mode == 2)
+        return dip_launch_combine_parts(ctx, WHICH, total_parts, n_slabs, BT, SLAB, WTraits<WT>::C, p.batch, p.d_out,
+                                        p.out, stream);
     return DIP_OK;
 }
 
@@ -1129,9 +1024,15 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
             else
                 st = which == 0 ? launch_direct<DIP_W_BF16, 0>(ctx, p, n_kept_max, stream)
                                 : launch_direct<DIP_W_BF16, 1>(ctx, p, n_kept_max, stream);
-        } else if (int4)
-            st = which == 0 ? launch_one<DIP_W_INT4_G128, 0, 1>(ctx, p, n_kept_max, mode, stream)
-                            : launch_one<DIP_W_INT4_G128, 1, 1>(ctx, p, n_kept_max, mode, stream);
+        } else if (int4) {
+            if (keys && which == 0 && keys->coarse) {
+                p.key_coarse = keys->coarse;
+                p.key_stamp = keys->stamp;
+                p.key_gamma = keys->gamma;
+            }
+            st = dip_launch_gemv_int4(ctx, p, which, n_kept_max, mode, stream);
+            if (st == DIP_OK && p.key_coarse && !mode) keys->written = 1;
+        }
         else if (w->wtype == DIP_W_F32)
             st = which == 0 ? launch_bt<DIP_W_F32, 0>(ctx, p, n_kept_max, mode, stream)
                             : launch_bt<DIP_W_F32, 1>(ctx, p, n_kept_max, mode, stream);

@@ -1,0 +1,53 @@
+// Declarations shared by the product kernels (gemv.cu, gemv_int4.cu).
+#pragma once
+
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+
+constexpr int GV_MAX_ROWS = 2048;                          // kept rows per round (index list in smem)
+constexpr int GV_SCAN_THREADS = 256;                       // threads that scan the mask words
+
+struct GemvParams {
+    const char *W;             // packed rows
+    size_t row_bytes;          // bytes of one packed row
+    const uint16_t *scales;    // INT4: binary16 scales [d_in/128][row elements], laid out like a row
+    size_t scale_row_elems;    // INT4: elements of one scale row
+    const float *v;            // [batch][d_in]
+    int d_in;
+    const uint32_t *mask_bits; // [batch][mask_words]; rows read = OR over the batch
+    int mask_words;
+    float *out;                // [batch][d_out]
+    int d_out;
+    int batch;                 // tokens in this launch (<= BT)
+    float *partials;
+    unsigned int *tickets;
+    int *status;               // device status word (0 = fine)
+    unsigned long long wait_limit_ns;   // a wait on a copy's arrival gives up after this long
+    unsigned long long *tr;    // timeline slot or nullptr
+    const int32_t *loc;        // two-tier: packed row of column i is W + loc[i] * row_bytes (nullptr: row i)
+    int defer;                 // 1: leave the row parts in `partials` for combine_parts_kernel
+    int part_base;             // first part index of this launch inside `partials`
+    // gate/up, single-token launches only: top 16 bits of the rank key of every h_j for the select
+    // that follows (nullptr: not wanted); the key is |h_j| * (key_stamp[j] >= 0 ? 1 : key_gamma),
+    // or |h_j| without stamps
+    uint16_t *key_coarse;
+    const int32_t *key_stamp;
+    float key_gamma;
+};
+
+
+__device__ __forceinline__ float silu_f32(float g) { return g / (1.0f + expf(-g)); }
+
+__device__ __forceinline__ float half_bits_to_float(uint16_t h)
+{
+    return __half2float(__ushort_as_half(h));
+}
+
+// gemv.cu: sum of the row parts left in ctx->partials ([parts][n_slabs][bt][slab_elems]; gate/up
+// elements interleaved in chunks of c) and the epilogue, spread over the device.
+dip_status dip_launch_combine_parts(dip_ctx *ctx, int which, int total_parts, int n_slabs, int bt, int slab_elems, int c,
+                                    int batch, int d_out, float *out, cudaStream_t stream);
+
+// gemv_int4.cu: the single-token product for INT4-g128 weights.  mode as dip_gemv_rows.mode.
+dip_status dip_launch_gemv_int4(dip_ctx *ctx, GemvParams &p, int which, int n_kept_max, int mode, cudaStream_t stream);

@@ -28,34 +28,49 @@ __global__ void pack_transpose_kernel(const T *__restrict__ src, T *__restrict__
     }
 }
 
-// 4-bit codes.  src: [d_out][d_in/2] bytes, even i in the low nibble.  One thread writes one
-// destination byte = the codes of outputs j, j+1 (j even) for input column i.
-// mode 0: dst[i][j/2];  mode 1/2: 8-byte pieces of 16 codes, gate piece then up piece.
+// 4-bit codes.  src: [d_out][d_in/2] bytes, even i in the low nibble.  A packed row is a sequence
+// of chunks of 128 codes (64 bytes): local element e of a chunk is nibble (e >> 4) of the 32-bit
+// word w = e & 15, and the 16 words are stored in the order 0, 8, 1, 9, ..., 7, 15 (so that the
+// eight bytes at offset 8 g hold words g and g + 8: one lane's share of eight 16 x 16 MMA tiles).
+// mode 0 (down): chunk c holds outputs 128 c + e.  mode 1 (gate) / 2 (up): chunk c holds gate
+// outputs 64 c + e for e < 64 and up outputs 64 c + (e - 64) for e >= 64.
+// One thread writes one destination byte: nibbles m and m + 1 (m even) of a word, i.e. two
+// outputs 16 apart of the same source matrix.
 __global__ void pack_int4_kernel(const uint8_t *__restrict__ src, uint8_t *__restrict__ dst,
                                  int d_out, int d_in, int dst_row_bytes, int mode)
 {
-    const size_t n = (size_t)d_in * (d_out / 2);
-    for (size_t t = blockIdx.x * (size_t)blockDim.x + threadIdx.x; t < n; t += (size_t)gridDim.x * blockDim.x) {
-        const int i = (int)(t / (d_out / 2));
-        const int j = 2 * (int)(t % (d_out / 2));
+    const int per_chunk = mode == 0 ? 64 : 32;                    // destination bytes of this matrix per chunk
+    const int out_per_chunk = mode == 0 ? 128 : 64;
+    const int chunks = d_out / out_per_chunk;
+    const size_t n = (size_t)d_in * chunks * per_chunk;
+    for (size_t tt = blockIdx.x * (size_t)blockDim.x + threadIdx.x; tt < n; tt += (size_t)gridDim.x * blockDim.x) {
+        const int i = (int)(tt / ((size_t)chunks * per_chunk));
+        const int rem = (int)(tt % ((size_t)chunks * per_chunk));
+        const int c = rem / per_chunk, b = rem % per_chunk;
+        const int bytes_per_word = mode == 0 ? 4 : 2;             // of this matrix
+        const int wp = b / bytes_per_word, bl = b % bytes_per_word;
+        const int w = (wp >> 1) + 8 * (wp & 1);                   // word stored at position wp
+        const int j = c * out_per_chunk + 32 * bl + w;            // output in the low nibble; j + 16 in the high one
         const int sh = 4 * (i & 1);
         const uint8_t lo = (src[(size_t)j * (d_in / 2) + (i >> 1)] >> sh) & 15;
-        const uint8_t hi = (src[(size_t)(j + 1) * (d_in / 2) + (i >> 1)] >> sh) & 15;
-        size_t col = mode == 0 ? (size_t)(j >> 1)
-                               : (size_t)(j / 16) * 16 + ((j % 16) >> 1) + (mode == 2 ? 8 : 0);
-        dst[(size_t)i * dst_row_bytes + col] = (uint8_t)(lo | (hi << 4));
+        const uint8_t hi = (src[(size_t)(j + 16) * (d_in / 2) + (i >> 1)] >> sh) & 15;
+        const int byte_in_word = mode == 2 ? 2 + bl : bl;
+        dst[(size_t)i * dst_row_bytes + (size_t)c * 64 + wp * 4 + byte_in_word] = (uint8_t)(lo | (hi << 4));
     }
 }
 
-// binary16 scales [groups][d_out] -> same rows, interleaved per 16-output chunk for gate/up.
+// binary16 scales [groups][d_out] -> rows laid out element for element like the code chunks, with
+// local element e of a chunk at position (e & 15) * 8 + (e >> 4): eight consecutive scales are the
+// eight tiles of one fragment row.
 __global__ void pack_scales_kernel(const uint16_t *__restrict__ src, uint16_t *__restrict__ dst,
                                    int groups, int d_out, int dst_row_elems, int mode)
 {
     const size_t n = (size_t)groups * d_out;
     for (size_t t = blockIdx.x * (size_t)blockDim.x + threadIdx.x; t < n; t += (size_t)gridDim.x * blockDim.x) {
         const int g = (int)(t / d_out), j = (int)(t % d_out);
-        size_t col = mode == 0 ? (size_t)j : (size_t)(j / 16) * 32 + (j % 16) + (mode == 2 ? 16 : 0);
-        dst[(size_t)g * dst_row_elems + col] = src[t];
+        const int c = mode == 0 ? j / 128 : j / 64;
+        const int e = mode == 0 ? j % 128 : (j % 64) + (mode == 2 ? 64 : 0);
+        dst[(size_t)g * dst_row_elems + (size_t)c * 128 + (e & 15) * 8 + (e >> 4)] = src[t];
     }
 }
 
