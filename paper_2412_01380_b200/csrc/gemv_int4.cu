@@ -67,14 +67,15 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
 
 // Local element e of a chunk of a gate/up row: e < 64 gate output e, else up output e - 64.
 // WHICH = 0: grid.x segments of seg_chunks chunks of the bundled rows; WHICH = 1: of the down rows.
-template <int WHICH>
+template <int WHICH, int SEGC>
 __global__ void __launch_bounds__(I4_THREADS, 1)
-gemv_int4_kernel(const GemvParams p, int seg_chunks, int n_chunks)
+gemv_int4_kernel(const GemvParams p, int n_chunks)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     I4Smem &s = *reinterpret_cast<I4Smem *>(smem_raw);
-    const int seg_elems = seg_chunks * 128;
-    const int kgroups = I4_WARPS / seg_chunks;
+    constexpr int seg_chunks = SEGC;                            // chunks of 128 codes per segment
+    constexpr int seg_elems = seg_chunks * 128;
+    constexpr int kgroups = I4_WARPS / seg_chunks;
     float *s_sums = reinterpret_cast<float *>(smem_raw + sizeof(I4Smem));      // [kgroups][seg_elems]
     float *s_total = s_sums + kgroups * seg_elems;                             // [seg_elems]
     uint16_t *s_scale = reinterpret_cast<uint16_t *>(s_total + seg_elems);     // [staged groups][seg_elems]
@@ -101,10 +102,7 @@ gemv_int4_kernel(const GemvParams p, int seg_chunks, int n_chunks)
             if (o < seg_chunks * 64 && j < p.d_out) key_stamp[i] = __ldcg(p.key_stamp + j);
         }
     }
-    // ---- 1. the mask words and their popcount prefix; beside them (same round trip) the largest
-    //         magnitude of the vector, which fixes the power of two that lifts the values to the
-    //         top of the binary16 range ----
-    float amax = 0.f;
+    // ---- 1. the mask words and their popcount prefix ----
     uint32_t u[4] = {0u, 0u, 0u, 0u};
     if (tid < GV_SCAN_THREADS) {
 #pragma unroll
@@ -113,13 +111,6 @@ gemv_int4_kernel(const GemvParams p, int seg_chunks, int n_chunks)
             if (w < p.mask_words) u[j] = p.mask_bits[w];
         }
     }
-    for (int i = tid; i < p.d_in / 4; i += I4_THREADS) {
-        const float4 v = __ldg(reinterpret_cast<const float4 *>(p.v) + i);
-        amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    if (lane == 0) s.wmax[warp] = amax;
     if (tid < GV_SCAN_THREADS) {
         int c = 0;
 #pragma unroll
@@ -148,20 +139,40 @@ gemv_int4_kernel(const GemvParams p, int seg_chunks, int n_chunks)
         if (tid == GV_SCAN_THREADS - 1) s.n_total = pre;
     }
     __syncthreads();
-    float scale_up;
-    {
-        float m = s.wmax[lane & (I4_WARPS - 1)];
-#pragma unroll
-        for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        // the largest value lands in [2^14, 2^15)
-        int e = 0;
-        if (m > 0.f && m < 3.0e38f) (void)frexpf(m, &e);
-        scale_up = ldexpf(1.0f, max(-100, min(100, 15 - e)));
-    }
-    const float scale_down = 1.0f / scale_up;
     const int n_total = s.n_total;
     const int r_begin = (int)(((long long)part * n_total) / nparts);
     const int r_end = (int)(((long long)(part + 1) * n_total) / nparts);
+    // The largest magnitude among the values of the columns that the mask words of this part's
+    // rank range cover (a superset of the part's rows) fixes the power of two that lifts the
+    // values to the top of the binary16 range: the largest lands in [2^14, 2^15).
+    float scale_up, scale_down;
+    {
+        float amax = 0.f;
+        for (int w = tid; w < p.mask_words; w += I4_THREADS) {
+            const int lo = s.pre[w];
+            if (lo < r_end && lo + __popc(s.words[w]) > r_begin) {
+                const float4 *v4 = reinterpret_cast<const float4 *>(p.v + 32 * w);
+                float4 v[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = __ldg(v4 + i);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v[i].x), fabsf(v[i].y))), fmaxf(fabsf(v[i].z), fabsf(v[i].w)));
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        if (lane == 0) s.wmax[warp] = amax;
+        __syncthreads();
+        float m = s.wmax[lane & (I4_WARPS - 1)];
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        // binary32 exponent field of the largest magnitude (0 or a non-finite value: no scaling)
+        const int ef = (int)((__float_as_uint(m) >> 23) & 0xffu);
+        const int e = (ef == 0 || ef == 255) ? 0 : max(-100, min(100, 141 - ef));   // 2^e * m lies in [2^14, 2^15)
+        scale_up = __uint_as_float((uint32_t)(127 + e) << 23);
+        scale_down = __uint_as_float((uint32_t)(127 - e) << 23);
+    }
 
     // binary32 sums of this lane: tile m, fragment rows g and g + 8, still split over the four
     // groups of a quad (lane's t)
@@ -381,20 +392,30 @@ gemv_int4_kernel(const GemvParams p, int seg_chunks, int n_chunks)
             return;
         }
         __threadfence();
+        // all parts' loads in flight together: R = I4_THREADS / (seg_elems / 4) threads share four
+        // outputs, thread r of them adds the parts r, r + R, ...; the R sums meet in shared memory in
+        // order of r
         const size_t stride = (size_t)gridDim.x * seg_elems;
-        for (int e4 = tid; e4 < seg_elems / 4; e4 += I4_THREADS) {
-            const float *pp = p.partials + (size_t)slab * seg_elems + 4 * e4;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int q0 = 0; q0 < nparts; q0 += 8) {
-                float4 a[8];
+        constexpr int n4 = seg_elems / 4, R = I4_THREADS / n4;
+        const int e4 = tid % n4, r = tid / n4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float *pp = p.partials + (size_t)slab * seg_elems + 4 * e4;
+        for (int q0 = r; q0 < nparts; q0 += 8 * R) {
+            float4 a[8];
 #pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    a[q] = q0 + q < nparts ? __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(q0 + q) * stride))
+            for (int q = 0; q < 8; ++q)
+                a[q] = q0 + q * R < nparts ? __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(q0 + q * R) * stride))
                                            : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int q = 0; q < 8; ++q) { v.x += a[q].x; v.y += a[q].y; v.z += a[q].z; v.w += a[q].w; }
-            }
-            *reinterpret_cast<float4 *>(s_total + 4 * e4) = v;
+            for (int q = 0; q < 8; ++q) { v.x += a[q].x; v.y += a[q].y; v.z += a[q].z; v.w += a[q].w; }
+        }
+        *reinterpret_cast<float4 *>(s_sums + (size_t)r * seg_elems + 4 * e4) = v;
+        __syncthreads();
+        for (int e = tid; e < seg_elems; e += I4_THREADS) {
+            float t4 = 0.f;
+#pragma unroll
+            for (int k = 0; k < R; ++k) t4 += s_sums[(size_t)k * seg_elems + e];
+            s_total[e] = t4;
         }
         if (tid == 0) p.tickets[slab] = 0;                      // ready for the next launch
     }
@@ -430,22 +451,39 @@ gemv_int4_kernel(const GemvParams p, int seg_chunks, int n_chunks)
 // Segment width and row parts: one CTA per SM.  The CTA that completes a segment adds up
 // nparts x (segment outputs) partial sums alone, so the segment is narrowed (and the warps of a
 // CTA split the K-blocks instead) until that tail is short.
+namespace {
+
+template <int WHICH, int SEGC>
+dip_status launch_int4(dip_ctx *ctx, GemvParams &p, int n_chunks, int n_slabs, int nparts, size_t smem, cudaStream_t stream)
+{
+    static dip_per_device_once once;
+    constexpr size_t smem_max = sizeof(I4Smem) + (size_t)2 * I4_WARPS * 128 * sizeof(float) + I4_SCALE_BYTES;
+    DIP_CUDA_TRY(ctx, dip_raise_smem_limit(once, ctx->device, gemv_int4_kernel<WHICH, SEGC>, smem_max));
+    DIP_CUDA_TRY(ctx, dip_launch_pdl(gemv_int4_kernel<WHICH, SEGC>, dim3(n_slabs, nparts), dim3(I4_THREADS), smem, stream, p,
+                                     n_chunks));
+    return DIP_OK;
+}
+
+template <int WHICH>
+dip_status launch_int4_seg(dip_ctx *ctx, GemvParams &p, int seg_chunks, int n_chunks, int n_slabs, int nparts, size_t smem,
+                           cudaStream_t stream)
+{
+    switch (seg_chunks) {
+    case 16: return launch_int4<WHICH, 16>(ctx, p, n_chunks, n_slabs, nparts, smem, stream);
+    case 8: return launch_int4<WHICH, 8>(ctx, p, n_chunks, n_slabs, nparts, smem, stream);
+    case 4: return launch_int4<WHICH, 4>(ctx, p, n_chunks, n_slabs, nparts, smem, stream);
+    case 2: return launch_int4<WHICH, 2>(ctx, p, n_chunks, n_slabs, nparts, smem, stream);
+    default: return launch_int4<WHICH, 1>(ctx, p, n_chunks, n_slabs, nparts, smem, stream);
+    }
+}
+
+}  // namespace
+
 dip_status dip_launch_gemv_int4(dip_ctx *ctx, GemvParams &p, int which, int n_kept_max, int mode, cudaStream_t stream)
 {
     const int n_chunks = (int)(p.row_bytes / 64);
     int seg_chunks = 16, n_slabs = 0, nparts = 1;
-    // wide rows: the widest segment with which the segments alone occupy most of the SMs, so that
-    // one CTA sees all kept rows of its segment and nothing is combined across CTAs
-    bool whole = false;
-    for (int sc = 16; sc >= 1 && !whole; sc >>= 1) {
-        const int ns = (n_chunks + sc - 1) / sc;
-        if (ns <= ctx->sm_count && 5 * ns >= 3 * ctx->sm_count) {
-            seg_chunks = sc;
-            n_slabs = ns;
-            whole = true;
-        }
-    }
-    for (; !whole; seg_chunks >>= 1) {
+    for (;; seg_chunks >>= 1) {
         n_slabs = (n_chunks + seg_chunks - 1) / seg_chunks;
         nparts = ctx->sm_count / n_slabs;
         if (nparts > n_kept_max / 16) nparts = n_kept_max / 16;     // at least one K-block of rows per part
@@ -461,16 +499,9 @@ dip_status dip_launch_gemv_int4(dip_ctx *ctx, GemvParams &p, int which, int n_ke
     p.part_base = mode == 2 ? nparts : 0;
     const int kgroups = I4_WARPS / seg_chunks;
     const size_t smem = sizeof(I4Smem) + (size_t)(kgroups + 1) * seg_elems * sizeof(float) + I4_SCALE_BYTES;
-    const size_t smem_max = sizeof(I4Smem) + (size_t)2 * I4_WARPS * 128 * sizeof(float) + I4_SCALE_BYTES;
-    static dip_per_device_once once[2];
-    dim3 grid(n_slabs, nparts);
-    if (which == 0) {
-        DIP_CUDA_TRY(ctx, dip_raise_smem_limit(once[0], ctx->device, gemv_int4_kernel<0>, smem_max));
-        DIP_CUDA_TRY(ctx, dip_launch_pdl(gemv_int4_kernel<0>, grid, dim3(I4_THREADS), smem, stream, p, seg_chunks, n_chunks));
-    } else {
-        DIP_CUDA_TRY(ctx, dip_raise_smem_limit(once[1], ctx->device, gemv_int4_kernel<1>, smem_max));
-        DIP_CUDA_TRY(ctx, dip_launch_pdl(gemv_int4_kernel<1>, grid, dim3(I4_THREADS), smem, stream, p, seg_chunks, n_chunks));
-    }
+    const dip_status st = which == 0 ? launch_int4_seg<0>(ctx, p, seg_chunks, n_chunks, n_slabs, nparts, smem, stream)
+                                     : launch_int4_seg<1>(ctx, p, seg_chunks, n_chunks, n_slabs, nparts, smem, stream);
+    if (st != DIP_OK) return st;
     if (mode == 2)
         return dip_launch_combine_parts(ctx, which, total_parts, n_slabs, 1, seg_elems, 64, 1, p.d_out, p.out, stream);
     return DIP_OK;
