@@ -155,6 +155,7 @@ dip_status dip_create_ex(dip_ctx **out, int device, const dip_options *opt)
     if ((st = dev_alloc(ctx, &ctx->mask_ring, (size_t)2 * DIP_RING_LAYERS * (ctx->max_d / 32))) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask_tmp, (size_t)(ctx->max_d / 32))) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->coarse, (size_t)ctx->max_d)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->xt, (size_t)ctx->max_d * 32)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->status, (size_t)1)) != DIP_OK) return fail(st);
     if (cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
     if ((st = dev_alloc(ctx, &ctx->trace, (size_t)DIP_TRACE_SLOTS * DIP_TRACE_WORDS)) != DIP_OK) return fail(st);
@@ -198,6 +199,7 @@ dip_status dip_destroy(dip_ctx *ctx)
     cudaFree(ctx->mask_ring);
     cudaFree(ctx->mask_tmp);
     cudaFree(ctx->coarse);
+    cudaFree(ctx->xt);
     cudaFree(ctx->status);
     cudaFree(ctx->trace);
     for (int i = 0; i < 2; ++i) {

@@ -44,6 +44,7 @@ struct dip_ctx {
     uint32_t *mask_ring; // [2][DIP_RING_LAYERS][max_d/32] per-layer mask slots of the stack runner
     uint32_t *mask_tmp;  // [max_d/32] list-based GEMV entry points
     uint16_t *coarse;    // [max_d] top 16 bits of the rank keys of h, left by the gate/up GEMV
+    uint16_t *xt;        // [max_d][32] batched decode: per row of the union, the tokens' values as bfloat16 (16 high, 16 low halves)
     int coarse_min_d;    // smallest d_ff for which the step ranks h from those
     int *status;         // sticky device status word (0 = fine)
     // the cache updates run beside the GEMVs: one side stream per cache kind

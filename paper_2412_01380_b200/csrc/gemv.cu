@@ -1004,6 +1004,8 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
         else if (w->wtype == DIP_W_F32)
             st = which == 0 ? launch_bt<DIP_W_F32, 0>(ctx, p, n_kept_max, mode, stream)
                             : launch_bt<DIP_W_F32, 1>(ctx, p, n_kept_max, mode, stream);
+        else if (p.batch >= 3 && !mode)
+            st = dip_launch_gemv_tc(ctx, p, which, n_kept_max, stream);       // a dense contraction: tensor cores
         else
             st = which == 0 ? launch_bt<DIP_W_BF16, 0>(ctx, p, n_kept_max, mode, stream)
                             : launch_bt<DIP_W_BF16, 1>(ctx, p, n_kept_max, mode, stream);

@@ -82,5 +82,8 @@ __device__ __forceinline__ float half_bits_to_float(uint16_t h)
 dip_status dip_launch_combine_parts(dip_ctx *ctx, int which, int total_parts, int n_slabs, int bt, int slab_elems, int c,
                                     int batch, int d_out, float *out, cudaStream_t stream);
 
+// gemv_tc.cu: BF16 weights, 8 to 16 tokens: the product over the union of the tokens' rows on tcgen05 tensor cores.
+dip_status dip_launch_gemv_tc(dip_ctx *ctx, GemvParams &p, int which, int n_kept_max, cudaStream_t stream);
+
 // gemv_int4.cu: the single-token product for INT4-g128 weights.  mode as dip_gemv_rows.mode.
 dip_status dip_launch_gemv_int4(dip_ctx *ctx, GemvParams &p, int which, int n_kept_max, int mode, cudaStream_t stream);
