@@ -15,7 +15,9 @@
 // The order of every sum is fixed, so results are bit-reproducible; no float atomics.
 //
 // One token with F32 / BF16 weights takes gemv_direct_kernel further down instead: plain loads, a
-// 512-byte segment per CTA, and for gate/up no row parts at all.
+// 512-byte segment per CTA, and for gate/up no row parts at all.  INT4 weights (gemv_int4.cu) and
+// BF16 batches of three or more tokens (gemv_tc.cu) run on the tensor cores; this kernel serves
+// batches of F32 weights, two BF16 tokens, and the two-tier step.
 //
 // which = 0 (gate/up bundle): the epilogue applies silu(gate) * up (Eq. 2).  which = 1: down.
 // Every wait on an mbarrier is bounded; on expiry the kernel records a status word and leaves.
@@ -67,8 +69,8 @@ constexpr int GV_STAGE_BYTES = 32768;
 
 static_assert(DIP_MAX_D <= 32768, "the row lists in shared memory are 16-bit");
 template <int SEG> struct __align__(16) GemvSmem {
-    // [stage][row][SEG + 16]: rows are 16 bytes apart from a multiple of 2 KB, so that the 8 row
-    // addresses of a transposing matrix load fall into different banks
+    // [stage][row][SEG + 16]: rows are 16 bytes apart from a multiple of 2 KB, so that the row groups'
+    // 16-byte reads of neighbouring rows fall into different banks
     unsigned char ring[GV_STAGES][GV_STAGE_BYTES + (GV_STAGE_BYTES / SEG) * 16];
     uint64_t full[GV_STAGES];
     uint64_t empty[GV_STAGES];
@@ -97,15 +99,10 @@ gemv_kernel(const GemvParams p)
     constexpr int RG = GV_CONSUMER_WARPS / CG;                // row groups
     constexpr int R = GV_STAGE_BYTES / SEG;                   // rows per stage
     constexpr int RS = SEG + 16;                              // row stride inside a stage
-    constexpr bool MMA = WT == DIP_W_BF16 && BT >= 8;         // many tokens: tensor-core path
-    constexpr int XS = GvRound<BT>::ROWS + 8;                 // MMA: stride of a token's row of values
     extern __shared__ __align__(128) unsigned char smem_raw[];
     GemvSmem<SEG> &s = *reinterpret_cast<GemvSmem<SEG> *>(smem_raw);
     constexpr int ROWS = GvRound<BT>::ROWS;                   // rows per round
     float *s_v = reinterpret_cast<float *>(smem_raw + sizeof(GemvSmem<SEG>));   // [ROWS][BT]
-    // tensor-core path: the same bytes hold the values as bfloat16 pairs, [BT][XS] each
-    __nv_bfloat16 *s_xh = reinterpret_cast<__nv_bfloat16 *>(s_v);
-    __nv_bfloat16 *s_xl = s_xh + BT * XS;
 
     DIP_TRACE_MIN(p.tr, 0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -269,26 +266,8 @@ gemv_kernel(const GemvParams p)
 #pragma unroll
                     for (int b = 0; b < GB; ++b) {
                         const float val = ((mw[b] >> (idx & 31)) & 1u) ? vv[b] : 0.f;
-                        if constexpr (MMA) {
-                            // binary32 value as two bfloat16 (value = hi + lo up to 2^-17 relative),
-                            // stored [token][row] for the B operand of the tensor-core product
-                            const __nv_bfloat16 hi = __float2bfloat16_rn(val);
-                            const __nv_bfloat16 lo = __float2bfloat16_rn(val - __bfloat162float(hi));
-                            s_xh[(b0 + b) * XS + r] = hi;
-                            s_xl[(b0 + b) * XS + r] = lo;
-                        } else {
-                            s_v[r * BT + b0 + b] = val;
-                        }
+                        s_v[r * BT + b0 + b] = val;
                     }
-                }
-            }
-            if constexpr (MMA) {
-                // zero the values up to the next multiple of 16 rows (the last K step is partial)
-                const int n_pad = (n_rows + 15) & ~15;
-                for (int t = tid; t < (n_pad - n_rows) * BT; t += GV_CONSUMER_WARPS * 32) {
-                    const int b = t / (n_pad - n_rows), r = n_rows + t % (n_pad - n_rows);
-                    s_xh[b * XS + r] = __float2bfloat16_rn(0.f);
-                    s_xl[b * XS + r] = __float2bfloat16_rn(0.f);
                 }
             }
             asm volatile("bar.sync 2, %0;" ::"n"(GV_CONSUMER_WARPS * 32) : "memory");
@@ -299,57 +278,7 @@ gemv_kernel(const GemvParams p)
                 if (!mbar_wait(&s.full[st], (it / GV_STAGES) & 1, p.wait_limit_ns)) failed = true;
                 if (failed || s.abort) { failed = true; break; }
                 const int rows_here = min(R, n_rows - i * R);
-                if constexpr (MMA) {
-                    // Tensor cores: per 16 rows, D[16 outputs][8 tokens] += A[16 outputs][16 rows] * B[16 rows][8 tokens]
-                    // with A = the stage's weights (read transposed out of shared memory) and
-                    // B = the tokens' values, once for their high and once for their low halves.
-                    constexpr int MT = SEG / 256;             // 16-output tiles per warp
-                    constexpr int NT = BT / 8;                // 8-token tiles
-                    float *macc = &acc[0][0];                 // [MT][NT][4]
-                    const int g = lane >> 2, t4 = lane & 3;
-                    for (int kb = 0; kb < rows_here; kb += 16) {
-                        uint32_t bh[NT][2], bl[NT][2];
-#pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) {
-                            const int o = (nt * 8 + g) * XS + i * R + kb + 2 * t4;
-                            bh[nt][0] = *reinterpret_cast<const uint32_t *>(s_xh + o);
-                            bh[nt][1] = *reinterpret_cast<const uint32_t *>(s_xh + o + 8);
-                            bl[nt][0] = *reinterpret_cast<const uint32_t *>(s_xl + o);
-                            bl[nt][1] = *reinterpret_cast<const uint32_t *>(s_xl + o + 8);
-                        }
-                        const int left = rows_here - kb;      // valid rows of this K step
-#pragma unroll
-                        for (int mt = 0; mt < MT; ++mt) {
-                            const int m0 = (warp * MT + mt) * 16;
-                            // lane L addresses row (L & 7) of matrix L >> 3: rows kb..kb+7 / kb+8..kb+15,
-                            // outputs m0..m0+7 / m0+8..m0+15
-                            const int mrow = kb + ((lane >> 4) << 3) + (lane & 7);
-                            const int mcol = m0 + (((lane >> 3) & 1) << 3);
-                            uint32_t a0, a1, a2, a3;
-                            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3)
-                                         : "r"(smem_u32(&s.ring[st][mrow * RS + mcol * 2])));
-                            if (left < 16) {
-                                // rows past the end of the list hold stale bytes: clear them
-                                const int k0 = 2 * t4;
-                                if (k0 >= left) a0 = a1 = 0u; else if (k0 + 1 >= left) { a0 &= 0xffffu; a1 &= 0xffffu; }
-                                if (k0 + 8 >= left) a2 = a3 = 0u; else if (k0 + 9 >= left) { a2 &= 0xffffu; a3 &= 0xffffu; }
-                            }
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt) {
-                                float *c = macc + (mt * NT + nt) * 4;
-                                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
-                                             "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                             : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                                             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bh[nt][0]), "r"(bh[nt][1]));
-                                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
-                                             "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                                             : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                                             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bl[nt][0]), "r"(bl[nt][1]));
-                            }
-                        }
-                    }
-                } else if (lane_ok) {
+                if (lane_ok) {
                     {
 #pragma unroll
                         for (int rr = 0; rr < R / RG; ++rr) {
@@ -403,26 +332,7 @@ gemv_kernel(const GemvParams p)
     float *red = reinterpret_cast<float *>(&s.ring[0][0]);    // [RG-1][CG*32 lanes][BT][E]
     float *own = red + (RG - 1) * CG * 32 * BT * E;           // [BT][SLAB] sums of this CTA, after red
     static_assert(((RG - 1) * CG * 32 * BT * E + BT * SLAB) * sizeof(float) <= sizeof(s.ring), "ring too small");
-    if constexpr (MMA) {
-        // the accumulator fragments hold whole sums already (the warps split the outputs, not the rows)
-        if (warp < GV_CONSUMER_WARPS) {
-            constexpr int MT = SEG / 256, NT = BT / 8;
-            float *dst = (nparts > 1 || p.defer) ? p.partials + ((size_t)(p.part_base + part) * gridDim.x + slab) * (BT * SLAB) : own;
-            const float *macc = &acc[0][0];
-            const int g = lane >> 2, t4 = lane & 3;
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const float *c = macc + (mt * NT + nt) * 4;
-                    const int m = (warp * MT + mt) * 16 + g, n = nt * 8 + 2 * t4;
-                    dst[n * SLAB + m] = c[0];
-                    dst[(n + 1) * SLAB + m] = c[1];
-                    dst[n * SLAB + m + 8] = c[2];
-                    dst[(n + 1) * SLAB + m + 8] = c[3];
-                }
-        }
-    } else {
+    {
     if (warp < GV_CONSUMER_WARPS && rg > 0) {
 #pragma unroll
             for (int b = 0; b < BT; ++b)

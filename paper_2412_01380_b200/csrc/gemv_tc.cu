@@ -9,8 +9,8 @@
 //     MN-major operand descriptor names: the outputs of a row are contiguous, so the weights are the
 //     B operand (N = 256) as they arrive, untransposed, and each byte is read by one MMA only;
 //   * the tokens' values of the union's rows, zeroed where a token drops the row and split into two
-//     bfloat16, are gathered ONCE per product by xt_build_kernel (16 scattered loads per row) into
-//     rank order, 64 bytes per row; the loaders copy them as the MN-major A operand: row n = the
+//     bfloat16, are gathered ONCE per product by xt_build_kernel (16 scattered loads per row), 64
+//     bytes per column of the union; the loaders copy them as the MN-major A operand: row n = the
 //     high halves of token n, row 16 + n the low halves, the other rows of the M = 128 tile zero;
 //   * one thread of a seventeenth warp issues one tcgen05.mma (M = 128, N = 256, K = 16) per 16 rows
 //     once the loader warps have arrived on the buffer's "full" barrier; the accumulator lives in
@@ -102,57 +102,31 @@ __device__ __forceinline__ void tc_ld64(uint32_t taddr, float (&v)[64])
 
 namespace {
 
-// The tokens' values of every row of the union, in rank order, ready for the tensor core: xt[rank][n] =
-// bfloat16 high half of token n's value at that row (zero where the token's own mask drops the row
-// or n >= batch), xt[rank][16 + n] = the low half.  Built once per product instead of once per CTA
-// (the values are 16 scattered 4-byte loads per row).  Each CTA recomputes the prefix of the union's
-// mask words and fills the rows of its slice of the ranks.
+// The tokens' values of every column of the union, ready for the tensor core: xt[i][n] = bfloat16 high
+// half of token n's value at column i (zero where the token's own mask drops the column or
+// n >= batch), xt[i][16 + n] = the low half; columns outside the union are not written (and never
+// read).  Built once per product instead of once per CTA (the values are 16 scattered 4-byte loads
+// per column).  A block takes two mask words per pass; 16 consecutive threads are the 16 tokens of
+// one column.
 __global__ void __launch_bounds__(1024, 1)
 xt_build_kernel(const uint32_t *__restrict__ mask_bits, const float *__restrict__ v, int batch, int d_in, int mask_words,
                 uint16_t *__restrict__ xt)
 {
-    __shared__ uint32_t words[DIP_MAX_D / 32];
-    __shared__ int pre[DIP_MAX_D / 32];
-    __shared__ int wsum[32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
+    const int n = tid & 15, bit = (tid >> 4) & 31, half = tid >> 9;
     dip_grid_dependency_wait();
     dip_launch_dependents();
-    {
-        uint32_t u = 0u;
-        if (tid < mask_words)
-            for (int b = 0; b < batch; ++b) u |= mask_bits[(size_t)b * mask_words + tid];
-        if (tid == mask_words - 1 && (d_in & 31)) u &= (1u << (d_in & 31)) - 1u;
-        const int c = __popc(u);
-        int incl = c;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int n = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += n;
-        }
-        if (lane == 31) wsum[warp] = incl;
-        __syncthreads();
-        int before = 0;
-        for (int w = 0; w < warp; ++w) before += wsum[w];
-        if (tid < mask_words) {
-            words[tid] = u;
-            pre[tid] = before + incl - c;
-        }
-    }
-    __syncthreads();
-    // the mask words are shared out over the CTAs, two words per CTA and pass (one per half of the
-    // block); 16 consecutive threads (the tokens) take a row: a word's up to 32 rows at once
-    const int n = tid & 15, half = tid >> 9, j = (tid >> 4) & 31;
     for (int w = 2 * blockIdx.x + half; w < mask_words; w += 2 * gridDim.x) {
-        const uint32_t u = words[w];
-        if (j >= __popc(u)) continue;
-        const int bit = __fns(u, 0, j + 1);                      // the j-th set bit
         const int idx = w * 32 + bit;
-        const uint32_t mine = n < batch ? mask_bits[(size_t)n * mask_words + w] : 0u;
-        const float x = ((mine >> bit) & 1u) ? __ldg(v + (size_t)n * d_in + idx) : 0.f;
+        const bool mine = n < batch && idx < d_in && ((mask_bits[(size_t)n * mask_words + w] >> bit) & 1u);
+        // in the union if any of the 16 tokens (a half-warp) keeps the column
+        const unsigned any = __ballot_sync(0xffffffffu, mine) & (0xffffu << (tid & 16));
+        if (!any) continue;
+        const float x = mine ? __ldg(v + (size_t)n * d_in + idx) : 0.f;
         const __nv_bfloat16 hi = __float2bfloat16_rn(x);
         const __nv_bfloat16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
-        xt[(size_t)(pre[w] + j) * 32 + n] = __bfloat16_as_ushort(hi);
-        xt[(size_t)(pre[w] + j) * 32 + 16 + n] = __bfloat16_as_ushort(lo);
+        xt[(size_t)idx * 32 + n] = __bfloat16_as_ushort(hi);
+        xt[(size_t)idx * 32 + 16 + n] = __bfloat16_as_ushort(lo);
     }
 }
 
@@ -291,7 +265,7 @@ gemv_tc_kernel(const GemvParams p, const uint16_t *__restrict__ xt)
                     if (tid < TC_ROUND_ROWS * 4) {
                         const int r = mr * TC_ROUND_ROWS + bb_row;
                         const bool ok = r < n_rows;
-                        const uint16_t *src = ok ? xt + (size_t)(list_begin + r) * 32 + bb_mg * 8 : xt;
+                        const uint16_t *src = ok ? xt + (size_t)s.idx[r] * 32 + bb_mg * 8 : xt;
                         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(bb), "l"(src), "r"(ok ? 16 : 0) : "memory");
                     }
                 }
