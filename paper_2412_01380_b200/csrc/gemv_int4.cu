@@ -483,7 +483,18 @@ dip_status dip_launch_gemv_int4(dip_ctx *ctx, GemvParams &p, int which, int n_ke
 {
     const int n_chunks = (int)(p.row_bytes / 64);
     int seg_chunks = 16, n_slabs = 0, nparts = 1;
-    for (;; seg_chunks >>= 1) {
+    // wide rows: the widest segment with which the segments alone occupy most of the SMs, so that
+    // one CTA sees all kept rows of its segment and nothing is combined across CTAs
+    bool whole = false;
+    for (int sc = 16; sc >= 1 && !whole; sc >>= 1) {
+        const int ns = (n_chunks + sc - 1) / sc;
+        if (ns <= ctx->sm_count && 5 * ns >= 3 * ctx->sm_count) {
+            seg_chunks = sc;
+            n_slabs = ns;
+            whole = true;
+        }
+    }
+    for (; !whole; seg_chunks >>= 1) {
         n_slabs = (n_chunks + seg_chunks - 1) / seg_chunks;
         nparts = ctx->sm_count / n_slabs;
         if (nparts > n_kept_max / 16) nparts = n_kept_max / 16;     // at least one K-block of rows per part
