@@ -81,8 +81,14 @@ typedef struct dip_ctx dip_ctx;   /* opaque; owns scratch workspace on one devic
  *   coarse_min_d       smallest d_ff for which a single-token step ranks h from the 16-bit keys
  *                      that the gate/up product leaves behind: 0 = default (4096), negative =
  *                      every size.  Either way the masks are the same bits.
- *   wait_limit_us      bound of every in-kernel wait on an asynchronous copy, in microseconds
- *                      (0 = one second); see dip_device_status. */
+ *   wait_limit_us      bound of every in-kernel wait (on an asynchronous copy, on another thread
+ *                      block's flag), in microseconds (0 = one second); see dip_device_status.
+ *   select_in_product  0 = default: in a single-token step with F32 / BF16 weights each product
+ *                      kernel builds the mask of its own input (every thread block finds the
+ *                      columns that are certainly kept and streams them at once, one extra block
+ *                      completes the mask meanwhile); negative: a select kernel runs in front of
+ *                      each product instead.  The masks are the same bits either way; the
+ *                      products add the same rows in a different order. */
 typedef struct {
     int32_t max_d;
     int32_t max_batch;
@@ -90,7 +96,8 @@ typedef struct {
     int32_t gemv_copy_ring;
     int32_t coarse_min_d;
     int32_t wait_limit_us;
-    int32_t reserved[4];          /* keep zero */
+    int32_t select_in_product;
+    int32_t reserved[3];          /* keep zero */
 } dip_options;
 
 /* Create a context on `device` (a CUDA ordinal).  Allocates the scratch

@@ -47,7 +47,7 @@ class StepOutputsStruct(C.Structure):
 class OptionsStruct(C.Structure):
     _fields_ = [("max_d", C.c_int32), ("max_batch", C.c_int32), ("gemv_segment_bytes", C.c_int32),
                 ("gemv_copy_ring", C.c_int32), ("coarse_min_d", C.c_int32), ("wait_limit_us", C.c_int32),
-                ("reserved", C.c_int32 * 4)]
+                ("select_in_product", C.c_int32), ("reserved", C.c_int32 * 3)]
 
 
 class StackProbeStruct(C.Structure):
@@ -165,13 +165,14 @@ class Context:
     """A dip_ctx: scratch workspace on one device.  Not for concurrent use from several streams."""
 
     def __init__(self, device: int = 0, max_d: int = 0, max_batch: int = 0, gemv_segment_bytes: int = 0,
-                 gemv_copy_ring: bool = False, coarse_min_d: int = 0, wait_limit_us: int = 0):
+                 gemv_copy_ring: bool = False, coarse_min_d: int = 0, wait_limit_us: int = 0,
+                 select_in_product: int = 0):
         """The keyword arguments are the fields of dip_options (0 = the library's default)."""
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2412_01380_b200 needs a CUDA device; there is no CPU path")
         h = _vp()
         opt = OptionsStruct(int(max_d), int(max_batch), int(gemv_segment_bytes), int(bool(gemv_copy_ring)),
-                            int(coarse_min_d), int(wait_limit_us))
+                            int(coarse_min_d), int(wait_limit_us), int(select_in_product))
         st = _lib.dip_create_ex(C.byref(h), int(device), C.byref(opt))
         if st != OK:
             raise DipError(st, "dip_create_ex")

@@ -13,8 +13,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdip.so")
-SOURCES = ["api.cu", "topk.cu", "gemv.cu", "gemv_int4.cu", "gemv_tc.cu", "gemv_noalloc.cu", "pack.cu", "tier.cu", "rowdot.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "gemv_common.cuh"), os.path.join(ROOT, "include", "dip.h")]
+SOURCES = ["api.cu", "topk.cu", "gemv.cu", "gemv_fused.cu", "gemv_int4.cu", "gemv_tc.cu", "gemv_noalloc.cu", "pack.cu", "tier.cu", "rowdot.cu"]
+HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "gemv_common.cuh"), os.path.join(CSRC, "select_core.cuh"), os.path.join(ROOT, "include", "dip.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

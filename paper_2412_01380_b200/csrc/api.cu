@@ -133,6 +133,7 @@ dip_status dip_create_ex(dip_ctx **out, int device, const dip_options *opt)
     ctx->gemv_direct = o.gemv_copy_ring ? 0 : 1;
     // below ~4096 columns the whole of h and its stamps is a few KB and the plain select is as fast
     ctx->coarse_min_d = o.coarse_min_d == 0 ? 4096 : (o.coarse_min_d < 0 ? 0 : o.coarse_min_d);
+    ctx->fuse_select = o.select_in_product < 0 ? 0 : 1;
     ctx->wait_limit_ns = o.wait_limit_us ? 1000ull * (unsigned long long)o.wait_limit_us : 1000000000ull;
     // split-row partial sums: up to one part per SM of a whole output row per token
     ctx->partials_floats = PARTIALS_FLOATS;
@@ -384,26 +385,39 @@ static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
     const int nmax_h = cap_h < w->d_ff ? (int)cap_h : w->d_ff;
     dip_status st;
 
-    // m_x = topK(score(x))            (Eq. 7; the ranking of Algorithm 1 when a cache is given)
-    st = dip_launch_select(ctx, xa, xb, x_norm, batch, w->d_model, k_x, gamma,
-                           cache_gu ? cache_gu->stamp : nullptr, mask_x, s);
-    if (st != DIP_OK) return st;
-    // c' = cache_update(c, m_x)       (Algorithm 1; beside the products, which do not need it)
-    if (cache_gu && (st = fork_cache_update(ctx, 0, mask_x, cache_gu, s)) != DIP_OK) return st;
-    // h = (W~u x) * silu(W~g x)       (Eq. 2 inside Eq. 3)
-    // (a single-token product also leaves the top bits of the rank keys of h for the next launch)
-    dip_gemv_keys hk = {ctx->coarse, cache_d ? cache_d->stamp : nullptr, gamma, 0};
-    st = dip_launch_gemv(ctx, w, 0, x, batch, mask_x, nmax_x, h, s, nullptr,
-                         batch == 1 && w->d_ff >= ctx->coarse_min_d ? &hk : nullptr);
-    if (st != DIP_OK) return st;
-    // m_h = topK(score(h))            (Eq. 8: the GLU of the already sparsified gate/up)
-    st = dip_launch_select(ctx, h, nullptr, nullptr, batch, w->d_ff, k_h, gamma,
-                           cache_d ? cache_d->stamp : nullptr, mask_h, s, hk.written ? ctx->coarse : nullptr);
-    if (st != DIP_OK) return st;
-    if (cache_d && (st = fork_cache_update(ctx, 1, mask_h, cache_d, s)) != DIP_OK) return st;
-    // y = W~d h                       (Eq. 1 inside Eq. 3)
-    st = dip_launch_gemv(ctx, w, 1, h, batch, mask_h, nmax_h, y, s);
-    if (st != DIP_OK) return st;
+    if (batch == 1 && dip_gemv_fused_supported(ctx, w, 0, xb != nullptr) && dip_gemv_fused_supported(ctx, w, 1, false)) {
+        // The same four operations in two launches: each product builds the mask of its own input
+        // (Eq. 7 / Eq. 8, or the ranking of Algorithm 1) while it already streams the rows that are
+        // certain to be kept; the cache updates follow the launch that wrote their mask.
+        dip_gemv_keys hk = {ctx->coarse, cache_d ? cache_d->stamp : nullptr, gamma, 0};
+        const dip_fused_select sx = {xa, xb, x_norm, nullptr, k_x, gamma, cache_gu ? cache_gu->stamp : nullptr, mask_x};
+        if ((st = dip_launch_gemv_fused(ctx, w, 0, &sx, h, s, &hk)) != DIP_OK) return st;
+        if (cache_gu && (st = fork_cache_update(ctx, 0, mask_x, cache_gu, s)) != DIP_OK) return st;
+        const dip_fused_select sh = {h, nullptr, nullptr, ctx->coarse, k_h, gamma, cache_d ? cache_d->stamp : nullptr, mask_h};
+        if ((st = dip_launch_gemv_fused(ctx, w, 1, &sh, y, s, nullptr)) != DIP_OK) return st;
+        if (cache_d && (st = fork_cache_update(ctx, 1, mask_h, cache_d, s)) != DIP_OK) return st;
+    } else {
+        // m_x = topK(score(x))            (Eq. 7; the ranking of Algorithm 1 when a cache is given)
+        st = dip_launch_select(ctx, xa, xb, x_norm, batch, w->d_model, k_x, gamma,
+                               cache_gu ? cache_gu->stamp : nullptr, mask_x, s);
+        if (st != DIP_OK) return st;
+        // c' = cache_update(c, m_x)       (Algorithm 1; beside the products, which do not need it)
+        if (cache_gu && (st = fork_cache_update(ctx, 0, mask_x, cache_gu, s)) != DIP_OK) return st;
+        // h = (W~u x) * silu(W~g x)       (Eq. 2 inside Eq. 3)
+        // (a single-token product also leaves the top bits of the rank keys of h for the next launch)
+        dip_gemv_keys hk = {ctx->coarse, cache_d ? cache_d->stamp : nullptr, gamma, 0};
+        st = dip_launch_gemv(ctx, w, 0, x, batch, mask_x, nmax_x, h, s, nullptr,
+                             batch == 1 && w->d_ff >= ctx->coarse_min_d ? &hk : nullptr);
+        if (st != DIP_OK) return st;
+        // m_h = topK(score(h))            (Eq. 8: the GLU of the already sparsified gate/up)
+        st = dip_launch_select(ctx, h, nullptr, nullptr, batch, w->d_ff, k_h, gamma,
+                               cache_d ? cache_d->stamp : nullptr, mask_h, s, hk.written ? ctx->coarse : nullptr);
+        if (st != DIP_OK) return st;
+        if (cache_d && (st = fork_cache_update(ctx, 1, mask_h, cache_d, s)) != DIP_OK) return st;
+        // y = W~d h                       (Eq. 1 inside Eq. 3)
+        st = dip_launch_gemv(ctx, w, 1, h, batch, mask_h, nmax_h, y, s);
+        if (st != DIP_OK) return st;
+    }
 
     if (out && out->idx_x && (st = dip_launch_mask_to_idx(ctx, mask_x, batch, 1, w->d_model, out->idx_x, k_x, nullptr, s)) != DIP_OK)
         return st;

@@ -47,6 +47,7 @@ struct dip_ctx {
     uint16_t *xt;        // [max_d][32] batched decode: per row of the union, the tokens' values as bfloat16 (16 high, 16 low halves)
     int coarse_min_d;    // smallest d_ff for which the step ranks h from those
     int *status;         // sticky device status word (0 = fine)
+    int fuse_select;     // single-token F32 / BF16 steps: the products build their own masks
     // the cache updates run beside the GEMVs: one side stream per cache kind
     cudaStream_t side[2];
     cudaEvent_t ev_fork[2], ev_join[2];
@@ -194,6 +195,21 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
                            const float *v, int batch, const uint32_t *mask_bits, int n_kept_max,
                            float *out, cudaStream_t stream, const dip_gemv_rows *rows = nullptr,
                            dip_gemv_keys *keys = nullptr);
+
+// gemv_fused.cu: the product `which` of a single-token step together with the select of its input.
+struct dip_fused_select {
+    const float *xa;         // gate/up: x, or the previous layer's x when xb is given; down: h
+    const float *xb;         // gate/up, chained layers: the previous layer's y (else nullptr)
+    float *x_out;            // gate/up with xb: receives x = (xa + xb) / rms(xa + xb)
+    const uint16_t *coarse;  // down: the 16-bit rank keys that the gate/up product left
+    int k;
+    float gamma;
+    const int32_t *stamp;    // cache state of the input (cache-aware ranking) or nullptr
+    uint32_t *mask_out;      // receives the mask
+};
+bool dip_gemv_fused_supported(const dip_ctx *ctx, const dip_mlp_weights *w, int which, bool norm);
+dip_status dip_launch_gemv_fused(dip_ctx *ctx, const dip_mlp_weights *w, int which, const dip_fused_select *sel,
+                                 float *out, cudaStream_t stream, dip_gemv_keys *keys);
 
 // gemv.cu: one tiny kernel whose bounded wait runs out (sets the status word to 1).
 dip_status dip_launch_bounded_wait_selftest(dip_ctx *ctx, unsigned long long limit_ns, unsigned long long *waited_ns,

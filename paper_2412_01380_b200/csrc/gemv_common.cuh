@@ -1,4 +1,4 @@
-// Declarations shared by the product kernels (gemv.cu, gemv_int4.cu).
+// Declarations shared by the product kernels (gemv.cu, gemv_fused.cu, gemv_int4.cu, gemv_tc.cu).
 #pragma once
 
 #include <cuda_fp16.h>
@@ -76,6 +76,32 @@ __device__ __forceinline__ float half_bits_to_float(uint16_t h)
 {
     return __half2float(__ushort_as_half(h));
 }
+
+namespace {
+
+template <int WT> struct WTraits;
+// E = weights in a lane's 16 bytes; C = gate/up interleave chunk of the bundled rows (weights)
+template <> struct WTraits<DIP_W_F32>       { static constexpr int E = 4;  static constexpr int C = 4; };
+template <> struct WTraits<DIP_W_BF16>      { static constexpr int E = 8;  static constexpr int C = 8; };
+
+template <int WT> __device__ __forceinline__ void decode16(const uint4 &r, float (&w)[WTraits<WT>::E]);
+template <> __device__ __forceinline__ void decode16<DIP_W_F32>(const uint4 &r, float (&w)[4])
+{
+    w[0] = __uint_as_float(r.x); w[1] = __uint_as_float(r.y);
+    w[2] = __uint_as_float(r.z); w[3] = __uint_as_float(r.w);
+}
+// bfloat16 is the upper half of a binary32: widening is a shift or a mask.
+template <> __device__ __forceinline__ void decode16<DIP_W_BF16>(const uint4 &r, float (&w)[8])
+{
+    const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        w[2 * i] = __uint_as_float(u[i] << 16);
+        w[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+    }
+}
+
+}  // namespace
 
 // gemv.cu: sum of the row parts left in ctx->partials ([parts][n_slabs][bt][slab_elems]; gate/up
 // elements interleaved in chunks of c) and the epilogue, spread over the device.
