@@ -166,9 +166,13 @@ def median_repeat(ms_list):
     return s[len(s) // 2]
 
 
-def GATE_UP_KERNEL(w, batch):
+def GATE_UP_KERNEL(w, batch, select_in_product=True):
     """Name of the kernel that computes the gate/up product for this workload."""
-    return "gemv_direct_kernel" if batch == 1 and w.wtype != di.W_INT4_G128 else "gemv_kernel"
+    if w.wtype == di.W_INT4_G128:
+        return "gemv_int4_kernel"
+    if batch == 1:
+        return "gemv_fused_kernel" if select_in_product else "gemv_direct_kernel"
+    return "gemv_kernel" if batch == 2 else "gemv_tc_kernel"
 
 
 def max_over_ranks(ms, dist, torch, device):
@@ -355,40 +359,66 @@ def run_config(dip, ctx, torch, w, layers, xs_host, keep_ratio, budget, steps, w
         h = torch.empty(d_ff, device="cuda")
         y = torch.empty(d_model, device="cuda")
         n_pass_tok = 6
-        names = ["mask_x", "gate_up", "mask_h", "down", "rmsnorm"]   # mask_* = select (+ cache update when on)
+        # A step of this configuration runs each mask together with its product (one launch each) when the
+        # library supports that for the weights and shape; otherwise a select kernel precedes each product.
+        try:
+            dip.dip_select_gemv_gate_up(ctx, layers[0], xs_dev[0].clone(), k_x, gamma,
+                                        st2.cache_gu[0] if ca else None, st2.cache_d[0] if ca else None, mask_x, h)
+            fused = True
+        except dip.DipError:
+            fused = False
+        res["select_in_product"] = fused
+        cg = (lambda l: st2.cache_gu[l]) if ca else (lambda l: None)
+        cd = (lambda l: st2.cache_d[l]) if ca else (lambda l: None)
+        if fused:
+            names = ["select_gate_up", "select_down", "rmsnorm"]
+        else:
+            names = ["mask_x", "gate_up", "mask_h", "down", "rmsnorm"]   # mask_* = select (+ cache update when on)
         evs = []
         for t in range(n_pass_tok):
             cur = xs_dev[t % n_tok].clone()
             for l in range(L):
-                ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)]
                 ev[0].record(stream)
-                if ca:
-                    dip.dip_ca_mask(ctx, cur, k_x, gamma, st2.cache_gu[l], mask_x, None)
+                if fused:
+                    dip.dip_select_gemv_gate_up(ctx, layers[l], cur, k_x, gamma, cg(l), cd(l), mask_x, h)
+                    ev[1].record(stream)
+                    dip.dip_select_gemv_down(ctx, layers[l], h, k_h, gamma, cd(l), mask_h, y)
+                    ev[2].record(stream)
                 else:
-                    dip.dip_mask_topk(ctx, cur, k_x, mask_x, None)
-                ev[1].record(stream)
-                dip.dip_sparse_gemv_gate_up(ctx, layers[l], cur, None, k_x, mask_x, h)
-                ev[2].record(stream)
-                if ca:
-                    dip.dip_ca_mask(ctx, h, k_h, gamma, st2.cache_d[l], mask_h, None)
-                else:
-                    dip.dip_mask_topk(ctx, h, k_h, mask_h, None)
-                ev[3].record(stream)
-                dip.dip_sparse_gemv_down(ctx, layers[l], h, None, k_h, mask_h, y)
-                ev[4].record(stream)
+                    if ca:
+                        dip.dip_ca_mask(ctx, cur, k_x, gamma, st2.cache_gu[l], mask_x, None)
+                    else:
+                        dip.dip_mask_topk(ctx, cur, k_x, mask_x, None)
+                    ev[1].record(stream)
+                    dip.dip_sparse_gemv_gate_up(ctx, layers[l], cur, None, k_x, mask_x, h)
+                    ev[2].record(stream)
+                    if ca:
+                        dip.dip_ca_mask(ctx, h, k_h, gamma, st2.cache_d[l], mask_h, None)
+                    else:
+                        dip.dip_mask_topk(ctx, h, k_h, mask_h, None)
+                    ev[3].record(stream)
+                    dip.dip_sparse_gemv_down(ctx, layers[l], h, None, k_h, mask_h, y)
+                    ev[4].record(stream)
                 dip.dip_residual_rmsnorm(ctx, cur, y, cur)
-                ev[5].record(stream)
+                ev[len(names)].record(stream)
                 if t >= 2:
                     evs.append(ev)
         torch.cuda.synchronize()
         kern = {}
         for i, n in enumerate(names):
             kern[n + "_us"] = float(np.mean([e[i].elapsed_time(e[i + 1]) for e in evs])) * 1e3
-        # The GEMVs again as a train of launches: one event pair around the product of every
+        # The products again as a train of launches: one event pair around the launch of every
         # layer (distinct weights, so each launch streams from HBM), twice.  The mean is the
-        # kernel's launch duration without the event pair's own overhead on every launch.
-        for name, call in (("gate_up", lambda l: dip.dip_sparse_gemv_gate_up(ctx, layers[l], cur, None, k_x, mask_x, h)),
-                           ("down", lambda l: dip.dip_sparse_gemv_down(ctx, layers[l], h, None, k_h, mask_h, y))):
+        # kernel's launch duration without the event pair's own overhead on every launch.  With
+        # select_in_product the launch is the step's own kernel: the select of the input and the product.
+        if fused:
+            calls = (("gate_up", lambda l: dip.dip_select_gemv_gate_up(ctx, layers[l], cur, k_x, gamma, cg(l), cd(l), mask_x, h)),
+                     ("down", lambda l: dip.dip_select_gemv_down(ctx, layers[l], h, k_h, gamma, cd(l), mask_h, y)))
+        else:
+            calls = (("gate_up", lambda l: dip.dip_sparse_gemv_gate_up(ctx, layers[l], cur, None, k_x, mask_x, h)),
+                     ("down", lambda l: dip.dip_sparse_gemv_down(ctx, layers[l], h, None, k_h, mask_h, y)))
+        for name, call in calls:
             for l in range(min(L, 3)):
                 call(l)
             ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -947,8 +977,11 @@ def main():
         # batched decode: no per-kernel pass; the whole step on the bytes of the union of the masks
         gu_us = None
         achieved = head.get("union_gbs", head["step_gbs"])
-    launches_per_step = L * (4 + (2 if budget is not None else 0)) + 1
-    kernel_name = GATE_UP_KERNEL(w, args.batch) + " (gate/up bundle)"
+    fused = bool(head.get("select_in_product"))
+    # per layer: two selects and two products (or two launches that do both), two cache updates when a
+    # cache is on; one residual + rmsnorm closes the stack
+    launches_per_step = L * ((2 if fused else 4) + (2 if budget is not None else 0)) + 1
+    kernel_name = GATE_UP_KERNEL(w, args.batch, fused) + (" (select of x + gate/up bundle)" if fused else " (gate/up bundle)")
     line = {
         "metric": METRIC, "value": whole_job_rate(L * args.steps, world, head["ms_total"]), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["ms_per_step"],

@@ -308,6 +308,36 @@ dip_status dip_sparse_gemv_down(dip_ctx *ctx, const dip_mlp_weights *w,
                                 const uint32_t *mask_bits,
                                 float *y, void *stream);
 
+/* ------------------------------------------------------------------------
+ * dip_select_gemv_gate_up / dip_select_gemv_down — a mask and its product in
+ * ONE launch, for one token and F32 / BF16 weights: the two halves of
+ * dip_mlp_step as that step itself runs them (Eq. 7 + Eq. 2 in Eq. 3, then
+ * Eq. 8 + Eq. 1 in Eq. 3).  Every thread block of the product selects for
+ * itself and goes straight on to its rows, so nothing waits for a select kernel.
+ *   gate_up: x [d_model] in;  mask_x [ceil(d_model/32)] out;  h [d_ff] out.
+ *   down:    h [d_ff] in;     mask_h [ceil(d_ff/32)] out;     y [d_model] out.
+ *   cache    optional state of that input: the ranking of Algorithm 1 with
+ *            gamma; the state is only READ (no cache_update here).  NULL: plain
+ *            magnitude top-k, gamma ignored.
+ * The paper names no such operation: it is a fusion of dip_mask_topk /
+ * dip_ca_mask's ranking with dip_sparse_gemv_*, and gives their results (the
+ * mask bit for bit, the product up to the order of the binary32 sums).
+ * dip_select_gemv_down ranks h from 16-bit keys that dip_select_gemv_gate_up
+ * left in the context: call it right after dip_select_gemv_gate_up on the same
+ * context and stream, with that call's h, and pass the SAME cache_d and gamma to
+ * both (gate_up needs them to form the keys; NULL there means NULL here).
+ * DIP_ERR_UNSUPPORTED for INT4 weights, for shapes whose working set does not
+ * fit a thread block's shared memory, and when the context was created with
+ * select_in_product < 0.
+ * ------------------------------------------------------------------------ */
+dip_status dip_select_gemv_gate_up(dip_ctx *ctx, const dip_mlp_weights *w, const float *x,
+                                   int k_x, float gamma, const dip_cache_state *cache_gu,
+                                   const dip_cache_state *cache_d,
+                                   uint32_t *mask_x, float *h, void *stream);
+dip_status dip_select_gemv_down(dip_ctx *ctx, const dip_mlp_weights *w, const float *h,
+                                int k_h, float gamma, const dip_cache_state *cache_d,
+                                uint32_t *mask_h, float *y, void *stream);
+
 /* Optional outputs of a step; any pointer may be NULL (the step then keeps the
  * intermediate in its own workspace). */
 typedef struct {

@@ -84,6 +84,12 @@ _lib.dip_ca_mask.argtypes = [_vp, _vp, _i32, _i32, _f32, C.POINTER(CacheStateStr
 for _name in ("dip_sparse_gemv_gate_up", "dip_sparse_gemv_down"):
     getattr(_lib, _name).restype = _i32
     getattr(_lib, _name).argtypes = [_vp, C.POINTER(MlpWeightsStruct), _vp, _i32, _vp, _i32, _vp, _vp, _vp]
+_lib.dip_select_gemv_gate_up.restype = _i32
+_lib.dip_select_gemv_gate_up.argtypes = [_vp, C.POINTER(MlpWeightsStruct), _vp, _i32, _f32, C.POINTER(CacheStateStruct),
+                                         C.POINTER(CacheStateStruct), _vp, _vp, _vp]
+_lib.dip_select_gemv_down.restype = _i32
+_lib.dip_select_gemv_down.argtypes = [_vp, C.POINTER(MlpWeightsStruct), _vp, _i32, _f32, C.POINTER(CacheStateStruct),
+                                      _vp, _vp, _vp]
 _lib.dip_mlp_step.restype = _i32
 _lib.dip_mlp_step.argtypes = [_vp, C.POINTER(MlpWeightsStruct), _vp, _i32, _i32, _i32, _f32,
                               C.POINTER(CacheStateStruct), C.POINTER(CacheStateStruct), _vp,
@@ -127,7 +133,8 @@ EXPORTED = ["dip_create", "dip_create_ex", "dip_destroy", "dip_status_string", "
             "dip_device_status", "dip_reset_device_status", "dip_selftest_bounded_wait", "dip_stack_step_probed",
             "dip_trace_begin", "dip_trace_reset", "dip_trace_read", "dip_trace_end",
             "dip_packed_bytes", "dip_pack_weights", "dip_mask_topk", "dip_ca_mask",
-            "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_mlp_step",
+            "dip_sparse_gemv_gate_up", "dip_sparse_gemv_down", "dip_select_gemv_gate_up", "dip_select_gemv_down",
+            "dip_mlp_step",
             "dip_residual_rmsnorm", "dip_stack_step", "dip_mlp_step_tiered", "dip_mlp_step_neuron_pruned",
             "dip_sparse_gemv_down_noalloc"]
 
@@ -316,6 +323,22 @@ def dip_sparse_gemv_down(ctx: Context, w: MlpWeights, h: torch.Tensor, kept_idx:
     batch = 1 if h.dim() == 1 else h.shape[0]
     ctx.check(_lib.dip_sparse_gemv_down(ctx.handle, C.byref(w.struct), _ptr(h), batch, _ptr(kept_idx),
                                         int(n_kept), _ptr(mask_bits), _ptr(y), _stream()))
+
+
+def dip_select_gemv_gate_up(ctx: Context, w: MlpWeights, x: torch.Tensor, k_x: int, gamma: float,
+                            cache_gu: Optional[CacheState], cache_d: Optional[CacheState],
+                            mask_x: torch.Tensor, h: torch.Tensor) -> None:
+    ctx.check(_lib.dip_select_gemv_gate_up(ctx.handle, C.byref(w.struct), _ptr(x), int(k_x), float(gamma),
+                                           C.byref(cache_gu.struct) if cache_gu else None,
+                                           C.byref(cache_d.struct) if cache_d else None,
+                                           _ptr(mask_x), _ptr(h), _stream()))
+
+
+def dip_select_gemv_down(ctx: Context, w: MlpWeights, h: torch.Tensor, k_h: int, gamma: float,
+                         cache_d: Optional[CacheState], mask_h: torch.Tensor, y: torch.Tensor) -> None:
+    ctx.check(_lib.dip_select_gemv_down(ctx.handle, C.byref(w.struct), _ptr(h), int(k_h), float(gamma),
+                                        C.byref(cache_d.struct) if cache_d else None,
+                                        _ptr(mask_h), _ptr(y), _stream()))
 
 
 def dip_mlp_step(ctx: Context, w: MlpWeights, x: torch.Tensor, k_x: int, k_h: int, gamma: float,

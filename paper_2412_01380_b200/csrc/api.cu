@@ -354,6 +354,35 @@ dip_status dip_sparse_gemv_down(dip_ctx *ctx, const dip_mlp_weights *w, const fl
     return gemv_entry(ctx, w, 1, h, batch, kept_idx, n_kept, mask_bits, y, stream);
 }
 
+dip_status dip_select_gemv_gate_up(dip_ctx *ctx, const dip_mlp_weights *w, const float *x, int k_x, float gamma,
+                                   const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
+                                   uint32_t *mask_x, float *h, void *stream)
+{
+    if (!ctx_ok(ctx) || !weights_ok(w) || !x || !mask_x || !h) return DIP_ERR_INVALID_ARG;
+    if (!dip_aligned16(x) || !dip_aligned16(mask_x) || !dip_aligned16(h)) return DIP_ERR_INVALID_ARG;
+    if (k_x < 1 || k_x > w->d_model || !(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
+    if (cache_gu && !cache_ok(cache_gu, w->d_model)) return DIP_ERR_INVALID_ARG;
+    if (cache_d && !cache_ok(cache_d, w->d_ff)) return DIP_ERR_INVALID_ARG;
+    if (!fits(ctx, w->d_model, w->d_ff, 1)) return DIP_ERR_WORKSPACE;
+    if (!dip_gemv_fused_supported(ctx, w, 0, false) || !dip_gemv_fused_supported(ctx, w, 1, false)) return DIP_ERR_UNSUPPORTED;
+    dip_gemv_keys hk = {ctx->coarse, cache_d ? cache_d->stamp : nullptr, gamma, 0};
+    const dip_fused_select sx = {x, nullptr, nullptr, nullptr, k_x, gamma, cache_gu ? cache_gu->stamp : nullptr, mask_x};
+    return dip_launch_gemv_fused(ctx, w, 0, &sx, h, (cudaStream_t)stream, &hk);
+}
+
+dip_status dip_select_gemv_down(dip_ctx *ctx, const dip_mlp_weights *w, const float *h, int k_h, float gamma,
+                                const dip_cache_state *cache_d, uint32_t *mask_h, float *y, void *stream)
+{
+    if (!ctx_ok(ctx) || !weights_ok(w) || !h || !mask_h || !y) return DIP_ERR_INVALID_ARG;
+    if (!dip_aligned16(h) || !dip_aligned16(mask_h) || !dip_aligned16(y)) return DIP_ERR_INVALID_ARG;
+    if (k_h < 1 || k_h > w->d_ff || !(gamma >= 0.0f) || !isfinite(gamma)) return DIP_ERR_INVALID_ARG;
+    if (cache_d && !cache_ok(cache_d, w->d_ff)) return DIP_ERR_INVALID_ARG;
+    if (!fits(ctx, w->d_model, w->d_ff, 1)) return DIP_ERR_WORKSPACE;
+    if (!dip_gemv_fused_supported(ctx, w, 1, false)) return DIP_ERR_UNSUPPORTED;
+    const dip_fused_select sh = {h, nullptr, nullptr, ctx->coarse, k_h, gamma, cache_d ? cache_d->stamp : nullptr, mask_h};
+    return dip_launch_gemv_fused(ctx, w, 1, &sh, y, (cudaStream_t)stream, nullptr);
+}
+
 // One sparse MLP step.  xb != nullptr: the step's input is formed first as
 // x = (xa + xb) / rms(xa + xb), written to x_norm, in the same launch as its mask.
 // slot_x / slot_h: where the masks go when the caller did not ask for them.  defer_join: leave

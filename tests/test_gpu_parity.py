@@ -294,9 +294,9 @@ def test_mlp_step_ranking_h_from_the_gemv_keys(dip, wtype, d_model, d_ff, rho, b
 
 @pytest.mark.parametrize("d_model,d_ff", [(256, 4096), (1024, 8192)])
 def test_step_when_one_radix_bin_holds_every_rank_key(dip, ctx, d_model, d_ff):
-    """Inputs whose magnitudes all share their top 11 key bits: no column is certainly kept after the
-    first radix digit, so the products receive their whole masks at the very end of the early
-    hand-over (x within a factor 1.06; h_j = silu(a.x) (b.x) (1 + eps_j) with tiny eps_j)."""
+    """Inputs whose magnitudes all share their leading key bits, so that the bin of the k-th key holds
+    most columns and the selects take their general path (x within a factor 1.06; h_j = silu(a.x)
+    (b.x) (1 + eps_j) with tiny eps_j)."""
     rng = np.random.default_rng(d_ff)
     a = (rng.standard_normal(d_model) * 0.05).astype(np.float32)
     b = (rng.standard_normal(d_model) * 0.05).astype(np.float32)
@@ -314,6 +314,125 @@ def test_step_when_one_radix_bin_holds_every_rank_key(dip, ctx, d_model, d_ff):
         # gamma = 1: resident or not, the keys stay in one bin
         _check_step(dip, ctx, lw, w, x, k_x, k_h, 1.0, ref_gu, ref_d, g_gu, g_d)
     assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("levels", [6, 64, 1500])
+@pytest.mark.parametrize("beta", [None, 0.5])
+def test_step_with_tied_magnitudes(dip, ctx, levels, beta):
+    """x takes few distinct magnitudes, so many rank keys are EQUAL: ties go to the lower column.  With 6
+    levels hundreds of keys tie at the threshold (general path), with 64 some dozens (ranked inside the
+    threshold's bin), with 1500 a few."""
+    d_model, d_ff = 4096, 8192
+    lw = _layer(5 + levels, d_model, d_ff, di.W_BF16)
+    w = upload_layer(dip, ctx, lw)
+    k_x, k_h = di.keep_count(0.25, d_model), di.keep_count(0.25, d_ff)
+    gamma = 0.2 if beta is not None else 1.0
+    ref_gu = ref_d = g_gu = g_d = None
+    if beta is not None:
+        ref_gu, ref_d = oracle.Cache(d_model, int(beta * d_model)), oracle.Cache(d_ff, int(beta * d_ff))
+        g_gu, g_d = dip.CacheState(d_model, ref_gu.capacity, "cuda"), dip.CacheState(d_ff, ref_d.capacity, "cuda")
+    rng = np.random.default_rng(levels)
+    mags = np.sort(np.abs(rng.standard_normal(levels)).astype(np.float32) + np.float32(0.05))
+    for t in range(3):
+        x = (mags[rng.integers(0, levels, d_model)] * np.where(rng.random(d_model) < 0.5, -1, 1)).astype(np.float32)
+        _check_step(dip, ctx, lw, w, x, k_x, k_h, gamma, ref_gu, ref_d, g_gu, g_d)
+    assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("wtype,d_model,d_ff,rho,beta", [
+    (di.W_F32, 1024, 2816, 0.5, None),
+    (di.W_BF16, 3072, 8192, 0.25, 0.5),
+    (di.W_BF16, 1056, 4096, 0.1, 0.25),     # d_model not a multiple of 128
+])
+def test_select_gemv_pair(dip, ctx, wtype, d_model, d_ff, rho, beta):
+    """dip_select_gemv_gate_up + dip_select_gemv_down (mask and product in one launch each): masks bit-exact
+    against the oracle's ranking, products within tolerance, cache states only read."""
+    lw = _layer(71 + d_ff, d_model, d_ff, wtype)
+    w = upload_layer(dip, ctx, lw)
+    Wg, Wu, Wd = oracle_mats(lw)
+    k_x, k_h = di.keep_count(rho, d_model), di.keep_count(rho, d_ff)
+    gamma = 0.2 if beta is not None else 1.0
+    ref_gu = ref_d = g_gu = g_d = None
+    wl = di.WORKLOADS["phi3_mini"].scaled(seed=d_ff + 3)
+    xs = di.token_inputs(wl, n_tokens=4, batch=1, d=d_model)[:, 0]
+    if beta is not None:
+        # warm caches: a few tokens through the oracle, then copied to the device
+        ref_gu = oracle.Cache(d_model, di.cache_capacity(beta, d_model))
+        ref_d = oracle.Cache(d_ff, di.cache_capacity(beta, d_ff))
+        for x in xs[:3]:
+            oracle.mlp_step(Wg, Wu, Wd, x, k_x, k_h, gamma, ref_gu, ref_d)
+        g_gu, g_d = gpu_cache_from_oracle(dip, ref_gu), gpu_cache_from_oracle(dip, ref_d)
+    x = xs[3]
+    mask_x = torch.zeros((d_model + 31) // 32, dtype=torch.int32, device="cuda")
+    mask_h = torch.zeros((d_ff + 31) // 32, dtype=torch.int32, device="cuda")
+    h = torch.empty(d_ff, device="cuda")
+    y = torch.empty(d_model, device="cuda")
+    dip.dip_select_gemv_gate_up(ctx, w, torch.from_numpy(x).cuda(), k_x, gamma, g_gu, g_d, mask_x, h)
+    dip.dip_select_gemv_down(ctx, w, h, k_h, gamma, g_d, mask_h, y)
+    torch.cuda.synchronize()
+    if beta is not None:
+        assert cache_equal(g_gu, ref_gu) and cache_equal(g_d, ref_d)          # untouched
+    import copy
+    m_x, _ = oracle.dip_ca_mask(x, k_x, gamma, copy.deepcopy(ref_gu))
+    assert np.array_equal(bits_to_mask(mask_x, d_model), m_x)
+    h_ref = oracle.glu(oracle.masked_matvec(Wg, x, m_x), oracle.masked_matvec(Wu, x, m_x))
+    h_gpu = h.cpu().numpy()
+    assert rel_err(h_gpu, h_ref) <= REL_TOL
+    m_h, _ = oracle.dip_ca_mask(h_gpu, k_h, gamma, copy.deepcopy(ref_d))
+    assert np.array_equal(bits_to_mask(mask_h, d_ff), m_h)
+    assert rel_err(y.cpu().numpy(), oracle.masked_matvec(Wd, h_gpu, m_h)) <= REL_TOL
+    # the step itself gives the same bits (it runs these two launches)
+    y2 = torch.empty_like(y)
+    h2 = torch.empty_like(h)
+    c_gu = gpu_cache_from_oracle(dip, ref_gu) if beta is not None else None
+    c_d = gpu_cache_from_oracle(dip, ref_d) if beta is not None else None
+    dip.dip_mlp_step(ctx, w, torch.from_numpy(x).cuda(), k_x, k_h, gamma, c_gu, c_d, y2, h=h2)
+    torch.cuda.synchronize()
+    assert torch.equal(h, h2) and torch.equal(y, y2)
+    assert ctx.device_status() == 0
+
+
+def test_select_gemv_refuses_int4(dip, ctx):
+    lw = _layer(3, 512, 1024, di.W_INT4_G128)
+    w = upload_layer(dip, ctx, lw)
+    x = torch.zeros(512, device="cuda")
+    with pytest.raises(dip.DipError):
+        dip.dip_select_gemv_gate_up(ctx, w, x, 128, 1.0, None, None, torch.zeros(16, dtype=torch.int32, device="cuda"),
+                                    torch.empty(1024, device="cuda"))
+
+
+@pytest.mark.parametrize("wtype,d_model,d_ff,rho,beta", [
+    (di.W_F32, 1024, 2816, 0.5, None),
+    (di.W_BF16, 3072, 8192, 0.25, 0.5),
+])
+def test_step_with_select_kernels_in_front(dip, ctx, wtype, d_model, d_ff, rho, beta):
+    """A context created with select_in_product < 0 runs a select kernel in front of each product:
+    same bit-exact masks and cache states, products within tolerance of the oracle and of the default path."""
+    c = dip.Context(0, select_in_product=-1)
+    try:
+        lw = _layer(91 + d_ff, d_model, d_ff, wtype)
+        w = upload_layer(dip, c, lw)
+        k_x, k_h = di.keep_count(rho, d_model), di.keep_count(rho, d_ff)
+        gamma = 0.2 if beta is not None else 1.0
+        ref_gu = ref_d = g_gu = g_d = None
+        if beta is not None:
+            ref_gu = oracle.Cache(d_model, di.cache_capacity(beta, d_model))
+            ref_d = oracle.Cache(d_ff, di.cache_capacity(beta, d_ff))
+            g_gu = dip.CacheState(d_model, ref_gu.capacity, "cuda")
+            g_d = dip.CacheState(d_ff, ref_d.capacity, "cuda")
+        wl = di.WORKLOADS["phi3_mini"].scaled(seed=d_ff + 7)
+        xs = di.token_inputs(wl, n_tokens=4, batch=1, d=d_model)[:, 0]
+        for x in xs:
+            y = _check_step(dip, c, lw, w, x, k_x, k_h, gamma, ref_gu, ref_d, g_gu, g_d)
+        # the default context on the last token, from the same cache states before that token
+        with pytest.raises(dip.DipError):
+            dip.dip_select_gemv_gate_up(c, w, torch.from_numpy(xs[0]).cuda(), k_x, gamma, None, None,
+                                        torch.zeros((d_model + 31) // 32, dtype=torch.int32, device="cuda"),
+                                        torch.empty(d_ff, device="cuda"))
+        assert np.all(np.isfinite(y))
+    finally:
+        torch.cuda.synchronize()
+        c.close()
 
 
 def test_full_size_phi3_medium_layer(dip, ctx):
