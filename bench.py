@@ -146,8 +146,8 @@ class ClockSampler:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up GEMV launch at Phi-3-Medium shapes, keep
 # ratio 0.25, one token, from the committed ncu capture (profiles/): bytes, and the kernel it is of.
-NCU_TRAFFIC = {"kernel": "gemv_direct_kernel", "bytes": 94.40e6,
-               "source": "profiles/kernels_phi3_medium_4layers_rho025.md"}
+NCU_TRAFFIC = {"kernel": "gemv_fused_kernel", "bytes": 94.1e6,
+               "source": "profiles/kernels_fused_phi3_medium_4layers_rho025.md"}
 
 
 def ncu_traffic(w, keep_ratio, batch, kernel_name):
