@@ -234,6 +234,8 @@ _check_step = check_step
     (di.W_BF16, 1024, 4096, 0.1, 0.25),
     (di.W_BF16, 1024, 2048, 0.5, 0.25),     # k > capacity: bypass
     (di.W_BF16, 512, 1536, 1.0, 0.5),       # keep ratio 1: dense
+    (di.W_BF16, 512, 32768, 0.1, 0.25),     # the widest h the library takes
+    (di.W_BF16, 32768, 512, 0.25, 0.5),     # the widest x
     (di.W_INT4_G128, 1024, 2816, 0.25, 0.4),
     (di.W_INT4_G128, 4096, 14336, 0.25, 0.4),   # a full Llama-3-8B-shaped block
     (di.W_INT4_G128, 512, 1024, 1.0, None),
