@@ -13,7 +13,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdip.so")
-SOURCES = ["api.cu", "topk.cu", "gemv.cu", "gemv_fused.cu", "gemv_int4.cu", "gemv_tc.cu", "gemv_noalloc.cu", "pack.cu", "tier.cu", "rowdot.cu"]
+SOURCES = ["api.cu", "topk.cu", "gemv.cu", "gemv_fused.cu", "gemv_direct_bt.cu", "gemv_int4.cu", "gemv_tc.cu", "gemv_noalloc.cu", "pack.cu", "tier.cu", "rowdot.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "gemv_common.cuh"), os.path.join(CSRC, "select_core.cuh"), os.path.join(ROOT, "include", "dip.h")]
 
 NVCC_FLAGS = [

@@ -889,6 +889,8 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
             st = dip_launch_gemv_int4(ctx, p, which, n_kept_max, mode, stream);
             if (st == DIP_OK && p.key_coarse && !mode) keys->written = 1;
         }
+        else if (ctx->gemv_direct && p.batch == 2 && !rows)
+            st = dip_launch_gemv_direct_bt(ctx, p, w->wtype, which, n_kept_max, stream);   // two tokens: plain loads and FMAs keep up
         else if (w->wtype == DIP_W_F32)
             st = which == 0 ? launch_bt<DIP_W_F32, 0>(ctx, p, n_kept_max, mode, stream)
                             : launch_bt<DIP_W_F32, 1>(ctx, p, n_kept_max, mode, stream);

@@ -1,4 +1,4 @@
-// Declarations shared by the product kernels (gemv.cu, gemv_fused.cu, gemv_int4.cu, gemv_tc.cu).
+// Declarations shared by the product kernels (gemv.cu, gemv_fused.cu, gemv_direct_bt.cu, gemv_int4.cu, gemv_tc.cu).
 #pragma once
 
 #include <cuda_fp16.h>
@@ -107,6 +107,10 @@ template <> __device__ __forceinline__ void decode16<DIP_W_BF16>(const uint4 &r,
 // elements interleaved in chunks of c) and the epilogue, spread over the device.
 dip_status dip_launch_combine_parts(dip_ctx *ctx, int which, int total_parts, int n_slabs, int bt, int slab_elems, int c,
                                     int batch, int d_out, float *out, cudaStream_t stream);
+
+// gemv_direct_bt.cu: F32 / BF16 weights, two tokens: the product over the union of the tokens' rows with
+// plain loads and FMAs.
+dip_status dip_launch_gemv_direct_bt(dip_ctx *ctx, GemvParams &p, int wtype, int which, int n_kept_max, cudaStream_t stream);
 
 // gemv_tc.cu: BF16 weights, 8 to 16 tokens: the product over the union of the tokens' rows on tcgen05 tensor cores.
 dip_status dip_launch_gemv_tc(dip_ctx *ctx, GemvParams &p, int which, int n_kept_max, cudaStream_t stream);
