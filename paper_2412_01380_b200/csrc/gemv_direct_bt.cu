@@ -12,9 +12,11 @@ namespace {
 
 constexpr int GB_SEG = 512;
 
+constexpr int GB_MAX_ROWS = 8192;          // rows of the union per round (a part's share of them)
+
 struct __align__(16) GemvBtSmem {
-    uint16_t idx[GV_MAX_ROWS];
-    unsigned char tok[GV_MAX_ROWS];        // bit b: token b keeps the row
+    uint16_t idx[GB_MAX_ROWS];
+    unsigned char tok[GB_MAX_ROWS];        // bit b: token b keeps the row
     uint32_t words[DIP_MAX_D / 32];        // the union of the masks
     int pre[DIP_MAX_D / 32];
     int wsum[GV_SCAN_THREADS / 32];
@@ -97,8 +99,8 @@ gemv_direct_bt_kernel(const GemvParams p)
         for (int e = 0; e < E; ++e) acc[b][e] = 0.f;
     const char *base = p.W + byte_off;
 
-    for (int round_begin = r_begin; round_begin < r_end; round_begin += GV_MAX_ROWS) {
-        const int n_rows = min(r_end - round_begin, GV_MAX_ROWS);
+    for (int round_begin = r_begin; round_begin < r_end; round_begin += GB_MAX_ROWS) {
+        const int n_rows = min(r_end - round_begin, GB_MAX_ROWS);
         if (round_begin != r_begin) __syncthreads();
         // ---- 2. the round's rows in rank order, each with the set of tokens that keep it ----
         {
