@@ -42,6 +42,10 @@ constexpr int TC_A_KB_BYTES = 16 * TC_SEG;       // one K-block of weights: [k g
 constexpr int TC_B_KB_BYTES = 128 * 16 * 2;      // one K-block of values: [row group 16][k group 2][8 rows][16 B]
 constexpr int TC_TMEM_COLS = 256;                // one accumulator: 128 lanes x 256 binary32 columns
 
+// Rows per in-kernel list: a list boundary drains the copy ring, so a part should be one list
+// (16 tokens at keep ratio 0.25 keep ~5100 of 5120 gate/up rows, ~2500 down rows per part).
+constexpr int TC_LIST_ROWS = 8192;
+
 struct __align__(1024) TcSmem {
     unsigned char a[TC_BUFS][TC_KB * TC_A_KB_BYTES];   // weights, 4 x 32 KB
     unsigned char b[TC_BUFS][TC_KB * TC_B_KB_BYTES];   // token values, 4 x 16 KB
@@ -53,7 +57,7 @@ struct __align__(1024) TcSmem {
     int wsum[GV_SCAN_THREADS / 32];
     uint32_t words[DIP_MAX_D / 32];
     int pre[DIP_MAX_D / 32];
-    uint16_t idx[GV_MAX_ROWS];
+    uint16_t idx[TC_LIST_ROWS];
 };
 
 // Shared-memory operand descriptor: start address, leading / stride byte offsets (in 16-byte units),
@@ -220,10 +224,10 @@ gemv_tc_kernel(const GemvParams p, const uint16_t *__restrict__ xt)
     int g = 0;                         // rounds so far (buffer g & 1)
     bool failed = false;
 
-    // The part's rows go through in lists of at most GV_MAX_ROWS (the in-kernel row list), a list in
+    // The part's rows go through in lists of at most TC_LIST_ROWS (the in-kernel row list), a list in
     // rounds of TC_ROUND_ROWS.  Warps 0-15 load and store; warp 16 issues the MMAs.
-    for (int list_begin = r_begin; list_begin < r_end; list_begin += GV_MAX_ROWS) {
-        const int n_rows = min(r_end - list_begin, GV_MAX_ROWS);
+    for (int list_begin = r_begin; list_begin < r_end; list_begin += TC_LIST_ROWS) {
+        const int n_rows = min(r_end - list_begin, TC_LIST_ROWS);
         if (list_begin != r_begin) __syncthreads();               // everyone is done with the previous list
         {
             const int lo_rank = list_begin, hi_rank = list_begin + n_rows;
@@ -401,6 +405,7 @@ dip_status dip_launch_gemv_tc(dip_ctx *ctx, GemvParams &p, int which, int n_kept
     p.defer = 0;
     p.part_base = 0;
     const size_t smem = sizeof(TcSmem) + 1024;
+    static_assert(sizeof(TcSmem) + 1024 <= 227 * 1024, "fits a CTA's shared memory");
     static dip_per_device_once once[2];
     // the tokens' values of the union's rows, once for all CTAs
     const int xt_ctas = min((p.mask_words + 1) / 2, 2 * ctx->sm_count);
