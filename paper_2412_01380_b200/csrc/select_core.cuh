@@ -1,8 +1,8 @@
-// The radix select that builds a top-k bit mask (Sec. 3.1, Eq. 7-8; the cache-aware ranking of Eq. 10), as
-// device functions for CTAs of 1024 threads: shared state, the histogram search, the first half
-// (rank keys, first radix digit, classification into certain / candidate columns) and the second
-// half (refinement of the candidates, or the general path under heavy ties).  Used by the stand-alone
-// select kernels and by the product kernels that select for themselves.
+// The select that builds a top-k bit mask (Sec. 3.1, Eq. 7-8; the cache-aware ranking of Eq. 10), as
+// device functions for CTAs of 1024 threads: the one-histogram select over the top 15 bits of the
+// rank keys with an exact ranking inside the threshold's bin, the general radix select for heavy
+// ties (also the cache update's victim search), and the residual scale of a chained layer.  Used by
+// the stand-alone select kernels and by the product kernels that select for themselves.
 #pragma once
 
 #include "common.cuh"
@@ -22,9 +22,6 @@ struct TkShared {
     int wc[TK_WARPS];
     float wf[TK_WARPS];
     float scale;
-    int n_cand2;
-    uint32_t last_key[32];
-    int last_idx[32];
 };
 
 __device__ __forceinline__ unsigned lanemask_lt()
@@ -213,65 +210,6 @@ __device__ float block_residual_scale(const float *__restrict__ xa, const float 
     return *scale_slot;
 }
 
-// Second half of the fast path.  s_maskw holds the columns whose key lies in a bin above the
-// threshold's, s_candw those in the threshold's bin (both in the mask's layout, complete and
-// visible), keys[] the rank key of every candidate column at least, s.hist is zero.  The krem1
-// largest candidates (lower column first among equals) complete the mask.  Returns false when
-// more than 32 candidates share the threshold's top 22 bits; nothing has been written then.
-__device__ bool refine_candidates(const uint32_t *keys, TkShared &s, unsigned int *s_maskw, const unsigned int *s_candw,
-                                  int n_words, int krem1, uint32_t *__restrict__ mask_bits)
-{
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // second digit (bits 19..9) of the candidates; a thread walks the candidate bits of a word
-    for (int w = tid; w < n_words; w += TK_THREADS) {
-        unsigned u = s_candw[w];
-        while (u) {
-            const int col = w * 32 + __ffs(u) - 1;
-            u &= u - 1;
-            atomicAdd(&s.hist[(keys[col] & 0xfffffu) >> 9], 1u);
-        }
-    }
-    __syncthreads();
-    find_bin(s, krem1);
-    const uint32_t b2 = (uint32_t)s.bcast[0];
-    const int krem2 = s.bcast[1], cnt2 = s.bcast[2];
-    if (cnt2 > 32) return false;
-    for (int w = tid; w < n_words; w += TK_THREADS) {
-        unsigned u = s_candw[w], keep = 0u;
-        while (u) {
-            const int bit = __ffs(u) - 1;
-            u &= u - 1;
-            const uint32_t low = keys[w * 32 + bit] & 0xfffffu;
-            const uint32_t dg = low >> 9;
-            if (dg > b2) {
-                keep |= 1u << bit;
-            } else if (dg == b2) {
-                const int pos = atomicAdd(&s.n_cand2, 1);
-                s.last_key[pos] = low & 0x1ffu;
-                s.last_idx[pos] = w * 32 + bit;
-            }
-        }
-        if (keep) s_maskw[w] |= keep;                  // the word is this thread's
-    }
-    __syncthreads();
-    if (warp == 0) {
-        // at most 32 keys share the threshold's top 22 bits: rank them by (key descending,
-        // column ascending) and keep the first krem2
-        const uint32_t kv = lane < cnt2 ? s.last_key[lane] : 0u;
-        const int iv = lane < cnt2 ? s.last_idx[lane] : 0x7fffffff;
-        int rank = 0;
-        for (int j = 0; j < cnt2; ++j) {
-            const uint32_t kj = __shfl_sync(0xffffffffu, kv, j);
-            const int ij = __shfl_sync(0xffffffffu, iv, j);
-            rank += (kj > kv) || (kj == kv && ij < iv);
-        }
-        if (lane < cnt2 && rank < krem2) atomicOr(&s_maskw[iv >> 5], 1u << (iv & 31));
-    }
-    __syncthreads();
-    for (int w = tid; w < n_words; w += TK_THREADS) mask_bits[w] = s_maskw[w];
-    return true;
-}
-
 // General path (very many keys tied around the threshold): full radix select on all d keys in
 // keys[], then an ordered sweep that ranks the ties by column.
 __device__ void general_select(const uint32_t *keys, int d, int k, TkShared &s, uint32_t *__restrict__ mask_bits)
@@ -323,220 +261,7 @@ __device__ __forceinline__ uint32_t rank_key(float v, int stamp, float gamma)
     return __float_as_uint(a) & 0x7fffffffu;
 }
 
-// First half of the select over full rank keys.  On entry s.hist is zero (and that is visible);
-// with NORM, keys[] holds the bits of r = xa + xb and `scale` is 1 / rms(r), without NORM the row
-// is xa.  Forms the row's values (written to x_out and / or x_keep when given), the rank keys
-// (left in keys[]) and the histogram of their top 11 bits, finds the bin b1 of the k-th largest
-// key and sorts the columns into s_maskw (bins above b1: certainly kept) and s_candw (bin b1),
-// both in the mask's layout.  Returns how many of the candidates complete the mask; s.hist is
-// zero again; ends with a barrier.
-//   CA == false: key = bits(|x|)                              (DIP, Eq. 7-8)
-//   CA == true : key = bits(|x| * (resident ? 1 : gamma))     (numerator of Eq. 10)
-template <bool CA, bool NORM>
-__device__ __forceinline__ int select_front(const float *__restrict__ xa, float *__restrict__ x_out, float *x_keep,
-                                            int d, int k, float gamma, const int32_t *__restrict__ stamp, float scale,
-                                            uint32_t *keys, TkShared &s, unsigned int *s_maskw, unsigned int *s_candw)
-{
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if ((d & 3) == 0) {
-        const int n4 = d >> 2;
-        for (int j0 = 0; j0 < TK_VEC_ITERS && tid + j0 * TK_THREADS < n4; j0 += TK_VEC_BATCH) {
-        float4 v4[TK_VEC_BATCH];
-        int4 st4[TK_VEC_BATCH];
-#pragma unroll
-        for (int j = 0; j < TK_VEC_BATCH; ++j) {
-            const int q = tid + (j0 + j) * TK_THREADS;
-            if (q < n4) {
-                if (NORM) {
-                    const uint4 r = *reinterpret_cast<const uint4 *>(keys + 4 * q);
-                    v4[j] = make_float4(__uint_as_float(r.x) * scale, __uint_as_float(r.y) * scale,
-                                        __uint_as_float(r.z) * scale, __uint_as_float(r.w) * scale);
-                } else {
-                    v4[j] = reinterpret_cast<const float4 *>(xa)[q];
-                }
-                if (CA) st4[j] = reinterpret_cast<const int4 *>(stamp)[q];
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < TK_VEC_BATCH; ++j) {
-            const int q = tid + (j0 + j) * TK_THREADS;
-            if (q < n4) {
-                if (x_out) reinterpret_cast<float4 *>(x_out)[q] = v4[j];
-                if (x_keep) reinterpret_cast<float4 *>(x_keep)[q] = v4[j];
-                const float vv[4] = {v4[j].x, v4[j].y, v4[j].z, v4[j].w};
-                const int sv[4] = {CA ? st4[j].x : 0, CA ? st4[j].y : 0, CA ? st4[j].z : 0, CA ? st4[j].w : 0};
-                uint32_t kk[4];
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    kk[t] = rank_key<CA>(vv[t], sv[t], gamma);
-                    atomicAdd(&s.hist[kk[t] >> 20], 1u);
-                }
-                *reinterpret_cast<uint4 *>(keys + 4 * q) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
-            }
-        }
-        }
-    } else {
-        for (int e = tid; e < d; e += TK_THREADS) {
-            float v;
-            if (NORM) v = __uint_as_float(keys[e]) * scale;
-            else v = xa[e];
-            if (x_out) x_out[e] = v;
-            if (x_keep) x_keep[e] = v;
-            const uint32_t key = rank_key<CA>(v, CA ? stamp[e] : 0, gamma);
-            keys[e] = key;
-            atomicAdd(&s.hist[key >> 20], 1u);
-        }
-    }
-    __syncthreads();
-    find_bin(s, k);
-    const uint32_t b1 = (uint32_t)s.bcast[0];
-    const int krem1 = s.bcast[1];
-
-    // Every key in a bin above b1 is kept, every key below is dropped; the krem1 largest of the
-    // keys in bin b1 (lower index first among equals) complete the mask.  One sweep, four keys
-    // per lane, builds two bit sets in the mask's layout: the certain columns and the columns of
-    // bin b1.  A lane's four flags are a nibble; eight neighbouring lanes OR theirs into a word.
-    s.hist[2 * tid] = 0;          // free again: refilled by the refinement with the candidates' next digit
-    s.hist[2 * tid + 1] = 0;
-    {
-        const int n4 = (d + 3) >> 2;
-        const int sh = (lane & 7) * 4;
-        for (int q0 = warp * 32; q0 < n4; q0 += TK_THREADS) {
-            const int q = q0 + lane;
-            uint4 kk = make_uint4(0u, 0u, 0u, 0u);
-            unsigned live = 0u;                                // which of the four columns exist
-            if (q < n4) {
-                kk = *reinterpret_cast<const uint4 *>(keys + 4 * q);
-                live = 4 * q + 4 <= d ? 0xfu : (1u << (d - 4 * q)) - 1u;
-            }
-            const uint32_t d0 = kk.x >> 20, d1 = kk.y >> 20, d2 = kk.z >> 20, d3 = kk.w >> 20;
-            unsigned gt = (d0 > b1 ? 1u : 0u) | (d1 > b1 ? 2u : 0u) | (d2 > b1 ? 4u : 0u) | (d3 > b1 ? 8u : 0u);
-            unsigned eq = (d0 == b1 ? 1u : 0u) | (d1 == b1 ? 2u : 0u) | (d2 == b1 ? 4u : 0u) | (d3 == b1 ? 8u : 0u);
-            gt = (gt & live) << sh;
-            eq = (eq & live) << sh;
-#pragma unroll
-            for (int o = 1; o < 8; o <<= 1) {
-                gt |= __shfl_xor_sync(0xffffffffu, gt, o);
-                eq |= __shfl_xor_sync(0xffffffffu, eq, o);
-            }
-            if ((lane & 7) == 0 && q < n4) {
-                s_maskw[q >> 3] = gt;
-                s_candw[q >> 3] = eq;
-            }
-        }
-    }
-    __syncthreads();
-    return krem1;
-}
-
-// First half of the select over coarse keys: coarse[] holds the top 16 bits of every rank key
-// (d % 8 == 0, d <= 8 * TK_COARSE_ITERS * TK_THREADS).  On entry s.hist is zero and visible.  Same
-// results as select_front (the first radix digit is the top 11 bits either way); no full key is
-// formed here.
-constexpr int TK_COARSE_ITERS = DIP_MAX_D / 8 / TK_THREADS;    // 16-byte loads per thread at the largest d
-
-__device__ __forceinline__ int select_coarse_front(const uint16_t *__restrict__ coarse, int d, int k, TkShared &s,
-                                                   unsigned int *s_maskw, unsigned int *s_candw)
-{
-    const int tid = threadIdx.x, lane = tid & 31;
-    const int n8 = d >> 3;
-    // coarse keys to registers (all loads in flight together)
-    uint4 ck[TK_COARSE_ITERS];
-#pragma unroll
-    for (int j = 0; j < TK_COARSE_ITERS; ++j) {
-        const int q = tid + j * TK_THREADS;
-        ck[j] = make_uint4(0u, 0u, 0u, 0u);
-        if (q < n8) ck[j] = __ldcg(reinterpret_cast<const uint4 *>(coarse) + q);
-    }
-#pragma unroll
-    for (int j = 0; j < TK_COARSE_ITERS; ++j) {
-        if (tid + j * TK_THREADS < n8) {
-            const uint32_t wv[4] = {ck[j].x, ck[j].y, ck[j].z, ck[j].w};
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                atomicAdd(&s.hist[(wv[t] & 0xffffu) >> 4], 1u);
-                atomicAdd(&s.hist[wv[t] >> 20], 1u);
-            }
-        }
-    }
-    __syncthreads();
-    find_bin(s, k);
-    const uint32_t b1 = (uint32_t)s.bcast[0];
-    const int krem1 = s.bcast[1];
-
-    // classification: a lane's eight flags are a byte, four neighbouring lanes make a mask word
-    s.hist[2 * tid] = 0;
-    s.hist[2 * tid + 1] = 0;
-    {
-        const int sh = (lane & 3) * 8;
-#pragma unroll
-        for (int j = 0; j < TK_COARSE_ITERS; ++j) {
-            const int q = tid + j * TK_THREADS;
-            if ((tid & ~31) + j * TK_THREADS < n8) {                  // the whole warp or none of it
-                const uint32_t wv[4] = {ck[j].x, ck[j].y, ck[j].z, ck[j].w};
-                unsigned gt = 0u, eq = 0u;
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const uint32_t lo = (wv[t] & 0xffffu) >> 4, hi = wv[t] >> 20;
-                    gt |= (lo > b1 ? 1u : 0u) << (2 * t) | (hi > b1 ? 2u : 0u) << (2 * t);
-                    eq |= (lo == b1 ? 1u : 0u) << (2 * t) | (hi == b1 ? 2u : 0u) << (2 * t);
-                }
-                if (q >= n8) gt = eq = 0u;
-                gt <<= sh;
-                eq <<= sh;
-                gt |= __shfl_xor_sync(0xffffffffu, gt, 1);
-                eq |= __shfl_xor_sync(0xffffffffu, eq, 1);
-                gt |= __shfl_xor_sync(0xffffffffu, gt, 2);
-                eq |= __shfl_xor_sync(0xffffffffu, eq, 2);
-                if ((lane & 3) == 0 && q < n8) {
-                    s_maskw[q >> 2] = gt;
-                    s_candw[q >> 2] = eq;
-                }
-            }
-        }
-    }
-    __syncthreads();
-    return krem1;
-}
-
-// Second half over coarse keys: the full rank keys of the candidates from x and the stamps, the
-// refinement, and under heavy ties all keys in full and the general path.  Writes the mask.
-template <bool CA>
-__device__ __forceinline__ void select_coarse_back(const float *__restrict__ x, const int32_t *__restrict__ stamp,
-                                                   float gamma, int d, int k, int krem1, uint32_t *keys, TkShared &s,
-                                                   unsigned int *s_maskw, const unsigned int *s_candw,
-                                                   uint32_t *__restrict__ mask_bits)
-{
-    const int tid = threadIdx.x;
-    const int n_words = d >> 5;
-    // (a word's candidates belong to one thread, here and in the refinement)
-    for (int w = tid; w < n_words; w += TK_THREADS) {
-        unsigned u = s_candw[w];
-        while (u) {
-            // four columns at a time, their loads in flight together
-            int col[4], sv[4];
-            float xv[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                col[i] = -1;
-                if (u) {
-                    col[i] = w * 32 + __ffs(u) - 1;
-                    u &= u - 1;
-                    xv[i] = __ldcg(x + col[i]);
-                    sv[i] = CA ? __ldcg(stamp + col[i]) : 0;
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (col[i] >= 0) keys[col[i]] = rank_key<CA>(xv[i], sv[i], gamma);
-        }
-    }
-    if (refine_candidates(keys, s, s_maskw, s_candw, n_words, krem1, mask_bits)) return;
-    // heavy ties: all keys in full, then the general path
-    for (int e = tid; e < d; e += TK_THREADS) keys[e] = rank_key<CA>(x[e], CA ? stamp[e] : 0, gamma);
-    __syncthreads();
-    general_select(keys, d, k, s, mask_bits);
-}
+constexpr int TK_COARSE_ITERS = DIP_MAX_D / 8 / TK_THREADS;    // 16-byte loads of 16-bit keys per thread at the largest d
 
 // ---------------------------------------------------------------------------------------------
 // The select in one histogram: the top 15 bits of the rank keys (8 exponent and 7 mantissa bits)

@@ -3,8 +3,8 @@
 // + RMS re-normalisation that chains layers.
 //
 // The step's critical path only needs the mask, so the work is split in two kernels:
-//   select_kernel        rank keys -> k-th largest key by radix select -> bit mask.  One CTA of
-//                        1024 threads per row; the keys live in shared memory.
+//   select_fine_kernel   rank keys -> k-th largest key by a histogram of their top 15 bits -> bit
+//                        mask.  One CTA of 1024 threads per row; the keys live in shared memory.
 //   cache_update_kernel  hits, misses, LRU victims and the new stamps from (mask, state).  It
 //                        does not feed the GEMVs and runs beside them on another stream.
 // Everything here is integer work on bit patterns, so results are exact and unique (ties go
@@ -15,26 +15,33 @@ namespace {
 
 
 // ---------------------------------------------------------------------------------------
-// select_kernel: the mask of one row.
+// select_fine_kernel: the mask of one row by the one-histogram select of select_core.cuh (the
+// select that the fused product kernels run), one CTA per row.
 //   CA == false: key = bits(|x|)                              (DIP, Eq. 7-8)
 //   CA == true : key = bits(|x| * (resident ? 1 : gamma))     (numerator of Eq. 10); the cache
 //                state is only read.
 //   NORM == true: the row is first formed as x = (xa + xb) / rms(xa + xb) (the layer chaining
 //                of a stack) and written to x_out; the summation order is that of
 //                residual_rmsnorm_kernel, so both give the same bits.
-// keys[] is dynamic shared memory: d words rounded up to a multiple of four.
+// select_fine_coarse_kernel: the same mask as select_fine_kernel<CA, false> for one row whose
+// producer has already left the top 16 bits of every rank key in coarse[] (the gate/up product
+// does, in its epilogue): one SM reads global memory at a fraction of the device's rate, so the
+// bytes this CTA has to pull in are its floor: two bytes per column instead of the eight of value +
+// stamp.  Needs d % 8 == 0 and d <= 8 * TK_COARSE_ITERS * TK_THREADS.
+// Dynamic shared memory: TkFine, then keys[] (d words rounded up to four).
 // ---------------------------------------------------------------------------------------
 template <bool CA, bool NORM>
 __global__ void __launch_bounds__(TK_THREADS, 1)
-select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *__restrict__ x_out,
-              int d, int k, float gamma, const int32_t *__restrict__ stamp,
-              uint32_t *__restrict__ mask_bits, unsigned long long *tr)
+select_fine_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float *__restrict__ x_out,
+                   int d, int k, float gamma, const int32_t *__restrict__ stamp,
+                   uint32_t *__restrict__ mask_bits, unsigned long long *tr)
 {
     DIP_TRACE_MIN(tr, 0);
-    extern __shared__ uint32_t keys[];
+    extern __shared__ __align__(16) unsigned char dyn[];
+    TkFine &f = *reinterpret_cast<TkFine *>(dyn);
+    uint32_t *keys = reinterpret_cast<uint32_t *>(dyn + sizeof(TkFine));
     __shared__ TkShared s;
-    __shared__ unsigned int s_maskw[DIP_MAX_D / 32];   // the mask being built
-    __shared__ unsigned int s_candw[DIP_MAX_D / 32];   // columns whose key falls in the threshold's bin
+    __shared__ unsigned int s_maskw[DIP_MAX_D / 32];
     const int tid = threadIdx.x;
     const int row = blockIdx.x;
     const int n_words = (d + 31) >> 5;
@@ -45,61 +52,45 @@ select_kernel(const float *__restrict__ xa, const float *__restrict__ xb, float 
     }
     mask_bits += (size_t)row * n_words;
 
-    s.hist[2 * tid] = 0;
-    s.hist[2 * tid + 1] = 0;
-    if (tid == 0) {
-        s.n_cand2 = 0;
-    }
-    dip_grid_dependency_wait();        // the inputs come from the previous kernel in the stream
-    DIP_TRACE_MIN(tr, 1);
-    dip_launch_dependents();
-
-    float scale = 1.0f;
-    if (NORM)
-        scale = block_residual_scale(xa, xb, d, keys, s.wf, &s.scale);   // ends with a barrier
-    else
-        __syncthreads();                                                  // histogram zeroed
-    const int krem1 = select_front<CA, NORM>(xa, NORM ? x_out : nullptr, nullptr, d, k, gamma, stamp, scale, keys, s,
-                                             s_maskw, s_candw);
-    if (refine_candidates(keys, s, s_maskw, s_candw, n_words, krem1, mask_bits)) {
-        DIP_TRACE_MAX(tr, 2);
-        return;
-    }
-    general_select(keys, d, k, s, mask_bits);
-    DIP_TRACE_MAX(tr, 2);
-}
-
-// ---------------------------------------------------------------------------------------
-// select_coarse_kernel: the same mask as select_kernel<CA, false> for one row whose producer has
-// already left the top 16 bits of every rank key in coarse[] (the gate/up GEMV does, in its
-// epilogue).  One SM reads global memory at a fraction of the device's rate, so the bytes this CTA
-// has to pull in are its floor: two bytes per column here instead of the eight of value + stamp.
-// The first radix digit (top 11 bits) and the classification sweep work on the coarse keys, eight
-// per lane, held in registers; the full key is formed only for the few hundred columns of the
-// threshold's bin.  Needs d % 8 == 0 and d <= 8 * TK_COARSE_ITERS * TK_THREADS.
-// ---------------------------------------------------------------------------------------
-template <bool CA>
-__global__ void __launch_bounds__(TK_THREADS, 1)
-select_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ coarse, int d, int k, float gamma,
-                     const int32_t *__restrict__ stamp, uint32_t *__restrict__ mask_bits, unsigned long long *tr)
-{
-    DIP_TRACE_MIN(tr, 0);
-    extern __shared__ uint32_t keys[];
-    __shared__ TkShared s;
-    __shared__ unsigned int s_maskw[DIP_MAX_D / 32];
-    __shared__ unsigned int s_candw[DIP_MAX_D / 32];
-    const int tid = threadIdx.x;
-
-    s.hist[2 * tid] = 0;
-    s.hist[2 * tid + 1] = 0;
-    if (tid == 0) s.n_cand2 = 0;
+    fine_zero(f);
     dip_grid_dependency_wait();
     DIP_TRACE_MIN(tr, 1);
     dip_launch_dependents();
-    __syncthreads();                                               // histogram zeroed
+    if (NORM && (d & 3) == 0 && d <= 8 * TK_THREADS) {
+        __syncthreads();                                              // histogram zeroed
+        select_fine_chained<CA>(xa, xb, x_out, nullptr, d, k, gamma, stamp, keys, s, f, s_maskw);
+    } else {
+        float scale = 1.0f;
+        if (NORM)
+            scale = block_residual_scale(xa, xb, d, keys, s.wf, &s.scale);   // ends with a barrier
+        else
+            __syncthreads();
+        select_fine<CA, NORM>(xa, NORM ? x_out : nullptr, nullptr, d, k, gamma, stamp, scale, keys, s, f, s_maskw);
+    }
+    for (int w = tid; w < n_words; w += TK_THREADS) mask_bits[w] = s_maskw[w];
+    DIP_TRACE_MAX(tr, 2);
+}
 
-    const int krem1 = select_coarse_front(coarse, d, k, s, s_maskw, s_candw);
-    select_coarse_back<CA>(x, stamp, gamma, d, k, krem1, keys, s, s_maskw, s_candw, mask_bits);
+template <bool CA>
+__global__ void __launch_bounds__(TK_THREADS, 1)
+select_fine_coarse_kernel(const float *__restrict__ x, const uint16_t *__restrict__ coarse, int d, int k, float gamma,
+                          const int32_t *__restrict__ stamp, uint32_t *__restrict__ mask_bits, unsigned long long *tr)
+{
+    DIP_TRACE_MIN(tr, 0);
+    extern __shared__ __align__(16) unsigned char dyn[];
+    TkFine &f = *reinterpret_cast<TkFine *>(dyn);
+    uint32_t *keys = reinterpret_cast<uint32_t *>(dyn + sizeof(TkFine));
+    __shared__ TkShared s;
+    __shared__ unsigned int s_maskw[DIP_MAX_D / 32];
+    const int tid = threadIdx.x;
+
+    fine_zero(f);
+    dip_grid_dependency_wait();
+    DIP_TRACE_MIN(tr, 1);
+    dip_launch_dependents();
+    __syncthreads();                                                  // histogram zeroed
+    select_fine_coarse<CA>(coarse, x, stamp, gamma, d, k, keys, s, f, s_maskw);
+    for (int w = tid; w < (d >> 5); w += TK_THREADS) mask_bits[w] = s_maskw[w];
     DIP_TRACE_MAX(tr, 2);
 }
 
@@ -296,30 +287,30 @@ dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, flo
                              float gamma, const int32_t *stamp, uint32_t *mask_bits, cudaStream_t stream,
                              const uint16_t *coarse)
 {
-    const size_t smem = (size_t)((d + 3) & ~3) * sizeof(uint32_t);
+    const size_t smem = sizeof(TkFine) + (size_t)((d + 3) & ~3) * sizeof(uint32_t);
     const dim3 grid(batch), block(TK_THREADS);
     unsigned long long *tr = dip_trace_slot(ctx, d <= 0 ? 0 : (stamp ? 2 : 1));
     cudaError_t e;
     if (coarse) {
         if (xb || batch != 1 || (d & 31)) return DIP_ERR_INVALID_ARG;
         if (stamp)
-            e = dip_launch_pdl(select_coarse_kernel<true>, grid, block, smem, stream, xa, coarse, d, k, gamma, stamp,
+            e = dip_launch_pdl(select_fine_coarse_kernel<true>, grid, block, smem, stream, xa, coarse, d, k, gamma, stamp,
                                mask_bits, tr);
         else
-            e = dip_launch_pdl(select_coarse_kernel<false>, grid, block, smem, stream, xa, coarse, d, k, 1.0f,
+            e = dip_launch_pdl(select_fine_coarse_kernel<false>, grid, block, smem, stream, xa, coarse, d, k, 1.0f,
                                (const int32_t *)nullptr, mask_bits, tr);
     } else if (xb) {
         if (stamp)
-            e = dip_launch_pdl(select_kernel<true, true>, grid, block, smem, stream, xa, xb, x_out, d, k, gamma, stamp, mask_bits, tr);
+            e = dip_launch_pdl(select_fine_kernel<true, true>, grid, block, smem, stream, xa, xb, x_out, d, k, gamma, stamp, mask_bits, tr);
         else
-            e = dip_launch_pdl(select_kernel<false, true>, grid, block, smem, stream, xa, xb, x_out, d, k, 1.0f,
+            e = dip_launch_pdl(select_fine_kernel<false, true>, grid, block, smem, stream, xa, xb, x_out, d, k, 1.0f,
                                (const int32_t *)nullptr, mask_bits, tr);
     } else {
         if (stamp)
-            e = dip_launch_pdl(select_kernel<true, false>, grid, block, smem, stream, xa, (const float *)nullptr,
+            e = dip_launch_pdl(select_fine_kernel<true, false>, grid, block, smem, stream, xa, (const float *)nullptr,
                                (float *)nullptr, d, k, gamma, stamp, mask_bits, tr);
         else
-            e = dip_launch_pdl(select_kernel<false, false>, grid, block, smem, stream, xa, (const float *)nullptr,
+            e = dip_launch_pdl(select_fine_kernel<false, false>, grid, block, smem, stream, xa, (const float *)nullptr,
                                (float *)nullptr, d, k, 1.0f, (const int32_t *)nullptr, mask_bits, tr);
     }
     DIP_CUDA_TRY(ctx, e);
@@ -339,13 +330,14 @@ dip_status dip_launch_cache_update(dip_ctx *ctx, const uint32_t *mask_bits, int 
 dip_status dip_init_mask_kernels(dip_ctx *ctx)
 {
     const int bytes = DIP_MAX_D * (int)sizeof(uint32_t);
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_coarse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_coarse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(cache_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    const int fine_bytes = bytes + (int)sizeof(TkFine);
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_fine_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, fine_bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_fine_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, fine_bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_fine_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, fine_bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_fine_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, fine_bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_fine_coarse_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, fine_bytes));
+    DIP_CUDA_TRY(ctx, cudaFuncSetAttribute(select_fine_coarse_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, fine_bytes));
     return DIP_OK;
 }
 
