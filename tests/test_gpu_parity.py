@@ -543,10 +543,11 @@ def test_stack_free_running_matches_oracle_up_to_near_ties(dip, ctx):
 # --------------------------------------------------------------------------------------
 # batched decode: per-token masks, union of kept columns read once
 # --------------------------------------------------------------------------------------
+@pytest.mark.parametrize("wtype", [di.W_BF16, di.W_F32])
 @pytest.mark.parametrize("batch", [2, 3, 4, 8, 16])
-def test_batched_step_matches_per_token_oracle(dip, ctx, batch):
+def test_batched_step_matches_per_token_oracle(dip, ctx, batch, wtype):
     d_model, d_ff = 1024, 2816
-    lw = _layer(41, d_model, d_ff, di.W_BF16)
+    lw = _layer(41, d_model, d_ff, wtype)
     w = upload_layer(dip, ctx, lw)
     Wg, Wu, Wd = oracle_mats(lw)
     wl = di.WORKLOADS["phi3_medium_batched"].scaled(d_model=d_model, d_ff=d_ff)
@@ -574,6 +575,36 @@ def test_batched_step_matches_per_token_oracle(dip, ctx, batch):
     _, n_ux = oracle.mask_union(mx)
     _, n_uh = oracle.mask_union(mh)
     assert counts.cpu().tolist() == [n_ux, n_uh]
+
+
+@pytest.mark.parametrize("batch", [2, 5])
+def test_batched_union_longer_than_one_row_list(dip, ctx, batch):
+    """A gate/up input of 16384 columns at keep ratio 0.9: the union of the tokens' rows (nearly all of them) is
+    longer than the products' in-kernel row lists of 8192, so they go through it in several rounds."""
+    d_model, d_ff = 16384, 512
+    lw = _layer(43, d_model, d_ff, di.W_BF16)
+    w = upload_layer(dip, ctx, lw)
+    Wg, Wu, Wd = oracle_mats(lw)
+    wl = di.WORKLOADS["phi3_medium_batched"].scaled(d_model=d_model, d_ff=d_ff)
+    x = di.token_inputs(wl, n_tokens=1, batch=batch)[0]
+    k_x, k_h = di.keep_count(0.9, d_model), di.keep_count(0.5, d_ff)
+    y = torch.empty((batch, d_model), device="cuda")
+    mask_x = torch.zeros((batch, d_model // 32), dtype=torch.int32, device="cuda")
+    mask_h = torch.zeros((batch, d_ff // 32), dtype=torch.int32, device="cuda")
+    h = torch.empty((batch, d_ff), device="cuda")
+    dip.dip_mlp_step(ctx, w, torch.from_numpy(x).cuda(), k_x, k_h, 1.0, None, None, y, mask_x=mask_x, h=h, mask_h=mask_h)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    mx, mh, hg, yg = bits_to_mask(mask_x, d_model), bits_to_mask(mask_h, d_ff), h.cpu().numpy(), y.cpu().numpy()
+    assert int(np.bitwise_or.reduce(mx, axis=0).sum()) > 8192
+    for b in range(batch):
+        m_x, _ = oracle.dip_ca_mask(x[b], k_x)
+        assert np.array_equal(mx[b], m_x)
+        h_ref = oracle.glu(oracle.masked_matvec(Wg, x[b], m_x), oracle.masked_matvec(Wu, x[b], m_x))
+        assert rel_err(hg[b], h_ref) <= REL_TOL
+        m_h, _ = oracle.dip_ca_mask(hg[b], k_h)
+        assert np.array_equal(mh[b], m_h)
+        assert rel_err(yg[b], oracle.masked_matvec(Wd, hg[b], m_h)) <= REL_TOL
 
 
 def test_full_size_batched_layer(dip, ctx):
