@@ -155,7 +155,7 @@ dip_status dip_create_ex(dip_ctx **out, int device, const dip_options *opt)
     if ((st = dev_alloc(ctx, &ctx->counts, (size_t)8)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask_ring, (size_t)2 * DIP_RING_LAYERS * (ctx->max_d / 32))) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->mask_tmp, (size_t)(ctx->max_d / 32))) != DIP_OK) return fail(st);
-    if ((st = dev_alloc(ctx, &ctx->coarse, (size_t)ctx->max_d)) != DIP_OK) return fail(st);
+    if ((st = dev_alloc(ctx, &ctx->coarse, vec)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->xt, (size_t)ctx->max_d * 32)) != DIP_OK) return fail(st);
     if ((st = dev_alloc(ctx, &ctx->status, (size_t)1)) != DIP_OK) return fail(st);
     if (cudaMemset(ctx->status, 0, sizeof(int)) != cudaSuccess) return fail(DIP_ERR_CUDA);
@@ -436,7 +436,7 @@ static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
         // (a single-token product also leaves the top bits of the rank keys of h for the next launch)
         dip_gemv_keys hk = {ctx->coarse, cache_d ? cache_d->stamp : nullptr, gamma, 0};
         st = dip_launch_gemv(ctx, w, 0, x, batch, mask_x, nmax_x, h, s, nullptr,
-                             batch == 1 && w->d_ff >= ctx->coarse_min_d ? &hk : nullptr);
+                             w->d_ff >= ctx->coarse_min_d && (w->d_ff & 31) == 0 ? &hk : nullptr);
         if (st != DIP_OK) return st;
         // m_h = topK(score(h))            (Eq. 8: the GLU of the already sparsified gate/up)
         st = dip_launch_select(ctx, h, nullptr, nullptr, batch, w->d_ff, k_h, gamma,

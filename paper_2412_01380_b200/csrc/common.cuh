@@ -43,7 +43,7 @@ struct dip_ctx {
     int32_t *counts;     // [8] device scalars (union sizes)
     uint32_t *mask_ring; // [2][DIP_RING_LAYERS][max_d/32] per-layer mask slots of the stack runner
     uint32_t *mask_tmp;  // [max_d/32] list-based GEMV entry points
-    uint16_t *coarse;    // [max_d] top 16 bits of the rank keys of h, left by the gate/up GEMV
+    uint16_t *coarse;    // [max_batch][max_d] top 16 bits of the rank keys of h, left by the gate/up product
     uint16_t *xt;        // [max_d][32] batched decode: per row of the union, the tokens' values as bfloat16 (16 high, 16 low halves)
     int coarse_min_d;    // smallest d_ff for which the step ranks h from those
     int *status;         // sticky device status word (0 = fine)
@@ -144,7 +144,7 @@ static inline cudaError_t dip_raise_smem_limit(dip_per_device_once &once, int de
 
 // topk.cu: mask of each row: k largest rank keys (|x|, or |x| * (resident ? 1 : gamma) when stamp
 // is given).  xb != nullptr: the row is first formed as (xa + xb) / rms(xa + xb), written to x_out.
-// coarse != nullptr (one row, no xb, d % 32 == 0): the producer of xa has left the top 16 bits of
+// coarse != nullptr (no xb, d % 32 == 0; several rows only without stamps): the producer of xa has left the top 16 bits of
 // every column's rank key there (dip_gemv_keys), and the launch reads those instead of all of
 // xa and stamp.
 dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, float *x_out, int batch, int d, int k,

@@ -889,13 +889,21 @@ dip_status dip_launch_gemv(dip_ctx *ctx, const dip_mlp_weights *w, int which,
             st = dip_launch_gemv_int4(ctx, p, which, n_kept_max, mode, stream);
             if (st == DIP_OK && p.key_coarse && !mode) keys->written = 1;
         }
-        else if (ctx->gemv_direct && p.batch == 2 && !rows)
+        else if (ctx->gemv_direct && p.batch == 2 && !rows) {
+            if (keys && which == 0 && keys->coarse && batch <= 16) {
+                p.key_coarse = keys->coarse;
+                keys->written = 1;
+            }
             st = dip_launch_gemv_direct_bt(ctx, p, w->wtype, which, n_kept_max, stream);   // two tokens: plain loads and FMAs keep up
+        }
         else if (w->wtype == DIP_W_F32)
             st = which == 0 ? launch_bt<DIP_W_F32, 0>(ctx, p, n_kept_max, mode, stream)
                             : launch_bt<DIP_W_F32, 1>(ctx, p, n_kept_max, mode, stream);
-        else if (p.batch >= 3 && !mode)
+        else if (p.batch >= 3 && !mode) {
+            if (keys && which == 0 && keys->coarse && batch <= 16) p.key_coarse = keys->coarse;
             st = dip_launch_gemv_tc(ctx, p, which, n_kept_max, stream);       // a dense contraction: tensor cores
+            if (st == DIP_OK && p.key_coarse) keys->written = 1;      // (the launcher drops the request when it splits the rows)
+        }
         else
             st = which == 0 ? launch_bt<DIP_W_BF16, 0>(ctx, p, n_kept_max, mode, stream)
                             : launch_bt<DIP_W_BF16, 1>(ctx, p, n_kept_max, mode, stream);

@@ -212,6 +212,9 @@ gemv_direct_bt_kernel(const GemvParams p)
                 r = s_sum[b * SLAB + o];
             }
             p.out[(size_t)b * p.d_out + j] = r;
+            // top 16 bits of the rank key |h_j| for the select that follows (no cache with several tokens)
+            if (WHICH == 0 && p.key_coarse)
+                p.key_coarse[(size_t)b * p.d_out + j] = (uint16_t)((__float_as_uint(r) & 0x7fffffffu) >> 16);
         }
     }
     DIP_TRACE_MAX(p.tr, 2);

@@ -359,6 +359,15 @@ gemv_tc_kernel(const GemvParams p, const uint16_t *__restrict__ xt)
                         if (j + 8 * c + 8 <= p.d_out) {
                             *reinterpret_cast<float4 *>(dst + 8 * c) = make_float4(h[0], h[1], h[2], h[3]);
                             *reinterpret_cast<float4 *>(dst + 8 * c + 4) = make_float4(h[4], h[5], h[6], h[7]);
+                            if (p.key_coarse) {
+                                // top 16 bits of the rank keys |h_j| for the select that follows (no cache with several tokens)
+                                uint32_t kk[4];
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)
+                                    kk[i] = ((__float_as_uint(h[2 * i]) & 0x7fffffffu) >> 16) |
+                                            ((__float_as_uint(h[2 * i + 1]) & 0x7fffffffu) & 0xffff0000u);
+                                *reinterpret_cast<uint4 *>(p.key_coarse + (size_t)n * p.d_out + j + 8 * c) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+                            }
                         } else {
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
@@ -404,6 +413,7 @@ dip_status dip_launch_gemv_tc(dip_ctx *ctx, GemvParams &p, int which, int n_kept
     if (nparts > 1 && (size_t)nparts * n_slabs * TC_N * 256 > ctx->partials_floats) return DIP_ERR_WORKSPACE;
     p.defer = 0;
     p.part_base = 0;
+    if (nparts > 1 || which != 0 || (p.d_out & 7)) p.key_coarse = nullptr;      // only the epilogue that sees whole sums forms the keys
     const size_t smem = sizeof(TcSmem) + 1024;
     static_assert(sizeof(TcSmem) + 1024 <= 227 * 1024, "fits a CTA's shared memory");
     static dip_per_device_once once[2];

@@ -83,6 +83,10 @@ select_fine_coarse_kernel(const float *__restrict__ x, const uint16_t *__restric
     __shared__ TkShared s;
     __shared__ unsigned int s_maskw[DIP_MAX_D / 32];
     const int tid = threadIdx.x;
+    const int row = blockIdx.x;                                       // (several rows only without a cache)
+    x += (size_t)row * d;
+    coarse += (size_t)row * d;
+    mask_bits += (size_t)row * (d >> 5);
 
     fine_zero(f);
     dip_grid_dependency_wait();
@@ -292,7 +296,7 @@ dip_status dip_launch_select(dip_ctx *ctx, const float *xa, const float *xb, flo
     unsigned long long *tr = dip_trace_slot(ctx, d <= 0 ? 0 : (stamp ? 2 : 1));
     cudaError_t e;
     if (coarse) {
-        if (xb || batch != 1 || (d & 31)) return DIP_ERR_INVALID_ARG;
+        if (xb || (batch != 1 && stamp) || (d & 31)) return DIP_ERR_INVALID_ARG;
         if (stamp)
             e = dip_launch_pdl(select_fine_coarse_kernel<true>, grid, block, smem, stream, xa, coarse, d, k, gamma, stamp,
                                mask_bits, tr);
