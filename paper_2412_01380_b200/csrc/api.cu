@@ -392,7 +392,7 @@ static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
                             int batch, int k_x, int k_h, float gamma,
                             const dip_cache_state *cache_gu, const dip_cache_state *cache_d,
                             float *y, const dip_step_outputs *out,
-                            uint32_t *slot_x, uint32_t *slot_h, bool defer_join, void *stream)
+                            uint32_t *slot_x, uint32_t *slot_h, bool defer_join, bool join_follows, void *stream)
 {
     const float *x = xb ? x_norm : xa;
     if (!ctx || !weights_ok(w) || !xa || !x || !y || !dip_aligned16(xa) || !dip_aligned16(x) || !dip_aligned16(y))
@@ -422,9 +422,19 @@ static dip_status step_impl(dip_ctx *ctx, const dip_mlp_weights *w,
         const dip_fused_select sx = {xa, xb, x_norm, nullptr, k_x, gamma, cache_gu ? cache_gu->stamp : nullptr, mask_x};
         if ((st = dip_launch_gemv_fused(ctx, w, 0, &sx, h, s, &hk)) != DIP_OK) return st;
         if (cache_gu && (st = fork_cache_update(ctx, 0, mask_x, cache_gu, s)) != DIP_OK) return st;
-        const dip_fused_select sh = {h, nullptr, nullptr, ctx->coarse, k_h, gamma, cache_d ? cache_d->stamp : nullptr, mask_h};
-        if ((st = dip_launch_gemv_fused(ctx, w, 1, &sh, y, s, nullptr)) != DIP_OK) return st;
-        if (cache_d && (st = fork_cache_update(ctx, 1, mask_h, cache_d, s)) != DIP_OK) return st;
+        if (cache_d && join_follows) {
+            // The caller waits for this step's cache updates right after it: the update of the down input
+            // (the long one) then has to run BESIDE the down product, which it can only with the mask
+            // from a select kernel of its own.
+            st = dip_launch_select(ctx, h, nullptr, nullptr, 1, w->d_ff, k_h, gamma, cache_d->stamp, mask_h, s, ctx->coarse);
+            if (st != DIP_OK) return st;
+            if ((st = fork_cache_update(ctx, 1, mask_h, cache_d, s)) != DIP_OK) return st;
+            if ((st = dip_launch_gemv(ctx, w, 1, h, 1, mask_h, nmax_h, y, s)) != DIP_OK) return st;
+        } else {
+            const dip_fused_select sh = {h, nullptr, nullptr, ctx->coarse, k_h, gamma, cache_d ? cache_d->stamp : nullptr, mask_h};
+            if ((st = dip_launch_gemv_fused(ctx, w, 1, &sh, y, s, nullptr)) != DIP_OK) return st;
+            if (cache_d && (st = fork_cache_update(ctx, 1, mask_h, cache_d, s)) != DIP_OK) return st;
+        }
     } else {
         // m_x = topK(score(x))            (Eq. 7; the ranking of Algorithm 1 when a cache is given)
         st = dip_launch_select(ctx, xa, xb, x_norm, batch, w->d_model, k_x, gamma,
@@ -466,7 +476,7 @@ dip_status dip_mlp_step(dip_ctx *ctx, const dip_mlp_weights *w,
 {
     if (!ctx_ok(ctx)) return DIP_ERR_INVALID_ARG;
     return step_impl(ctx, w, x, nullptr, nullptr, batch, k_x, k_h, gamma, cache_gu, cache_d, y, out,
-                     ctx->mask, ctx->mask_h, false, stream);
+                     ctx->mask, ctx->mask_h, false, true, stream);
 }
 
 // One masked input of the two-tier step.  On the step's path: the hit / miss split, the list of
@@ -643,7 +653,8 @@ static dip_status stack_impl(dip_ctx *ctx, int n_layers, const dip_mlp_weights *
         }
         dip_status st = step_impl(ctx, &layers[l], x_prev, y_prev, y_prev ? x_l : nullptr, batch, k_x, k_h, gamma,
                                   cache_gu ? &cache_gu[l] : nullptr, cache_d ? &cache_d[l] : nullptr,
-                                  y, probe ? &po : nullptr, slot_x, slot_h, true, stream);
+                                  y, probe ? &po : nullptr, slot_x, slot_h, true,
+                                  l == n_layers - 1 || (ca && slot == DIP_RING_LAYERS - 1), stream);
         if (st != DIP_OK) return st;
         if (ca && slot == DIP_RING_LAYERS - 1 && (st = join_cache_updates(ctx, s)) != DIP_OK) return st;
         if (y_prev) x_prev = x_l;
