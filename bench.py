@@ -980,7 +980,8 @@ def main():
     fused = bool(head.get("select_in_product"))
     # per layer: two selects and two products (or two launches that do both), two cache updates when a
     # cache is on; one residual + rmsnorm closes the stack
-    launches_per_step = L * ((2 if fused else 4) + (2 if budget is not None else 0)) + 1
+    # (with a cache the last layer's down half keeps its select kernel: one launch more per token)
+    launches_per_step = L * ((2 if fused else 4) + (2 if budget is not None else 0)) + 1 + (1 if fused and budget is not None else 0)
     kernel_name = GATE_UP_KERNEL(w, args.batch, fused) + (" (select of x + gate/up bundle)" if fused else " (gate/up bundle)")
     line = {
         "metric": METRIC, "value": whole_job_rate(L * args.steps, world, head["ms_total"]), "unit": UNIT, "n_gpus": world,
