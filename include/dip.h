@@ -78,9 +78,10 @@ typedef struct dip_ctx dip_ctx;   /* opaque; owns scratch workspace on one devic
  *                      row that one thread block of the copy-ring product kernel handles.
  *   gemv_copy_ring     non-zero: single-token F32 / BF16 products also go through the
  *                      copy-ring kernel (by default they use the plain-load kernel).
- *   coarse_min_d       smallest d_ff for which a single-token step ranks h from the 16-bit keys
- *                      that the gate/up product leaves behind: 0 = default (4096), negative =
- *                      every size.  Either way the masks are the same bits.
+ *   coarse_min_d       smallest d_ff for which a step that runs a select kernel in front of the
+ *                      down product (INT4 weights, several tokens, select_in_product < 0) ranks
+ *                      h from the 16-bit keys that the gate/up product leaves behind: 0 = default
+ *                      (4096), negative = every size.  Either way the masks are the same bits.
  *   wait_limit_us      bound of every in-kernel wait (on an asynchronous copy, on another thread
  *                      block's flag), in microseconds (0 = one second); see dip_device_status.
  *   select_in_product  0 = default: in a single-token step with F32 / BF16 weights each product
