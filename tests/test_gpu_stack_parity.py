@@ -182,6 +182,17 @@ def test_phi3_mini_stack_matches_oracle(dip, ctx):
     _run_stack_case(dip, ctx, wl, 3, 8, wl.keep_ratio, wl.cache_budget)
 
 
+def test_phi3_mini_stack_with_select_kernels_in_front(dip):
+    """The same stack on a context created with select_in_product < 0: four launches per layer."""
+    wl = di.WORKLOADS["phi3_mini"]
+    c = dip.Context(0, select_in_product=-1)
+    try:
+        _run_stack_case(dip, c, wl, 2, 4, wl.keep_ratio, wl.cache_budget)
+    finally:
+        torch.cuda.synchronize()
+        c.close()
+
+
 def test_llama3_8b_int4_stack_matches_oracle(dip, ctx):
     wl = di.WORKLOADS["llama3_8b_int4"]
     _run_stack_case(dip, ctx, wl, 2, 6, wl.keep_ratio, wl.cache_budget)
